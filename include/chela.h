@@ -1,0 +1,126 @@
+/*
+ * chela.h -- C ABI of the B200 (sm_100a) CHELA token-mixer hot path.
+ *
+ * The library evaluates, on one GPU, the forward pass of
+ *   - the short depthwise causal convolution + SiLU            (Eq. 7, inner part),
+ *   - the per-channel long convolution of length L via FFT       (Eq. 6, Sec. 2.2),
+ *   - chunked ("tiled, divide-and-conquer") causal linear attention with a carried
+ *     d_k x d_v state and a row normaliser                       (Eq. 2, Sec. 4.1),
+ *   - their composition with the Q/K/V formation                 (Eqs. 8, 10-12).
+ *
+ * Conventions common to every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller; the library never frees or
+ *     keeps it.  Pointers must be 16-byte aligned and the tensors contiguous in the stated
+ *     row-major layout (last index fastest).
+ *   - Work is enqueued on `stream`; calls return without synchronising the stream.
+ *   - `workspace` is caller-provided device scratch of at least the size the matching
+ *     `*_workspace_bytes` query returns (a query may return 0; then `workspace` may be NULL).
+ *     Its contents are undefined before and after a call.  Two calls that share a workspace
+ *     must be ordered on the GPU (same stream or an event).
+ *   - The library allocates no device memory in these calls.
+ *   - Return value: CHELA_OK or an error; arguments are validated before anything is
+ *     launched, so an error return means no kernel ran.  Nothing throws or aborts.
+ *   - dtype arguments take chela_dtype_t; bf16 tensors hold IEEE bfloat16 bit patterns.
+ *     All arithmetic accumulates in fp32.
+ */
+#ifndef CHELA_H_
+#define CHELA_H_
+
+#include <stddef.h>
+#include <cuda_runtime_api.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CHELA_OK = 0,
+    CHELA_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer          */
+    CHELA_ERR_UNSUPPORTED = 2, /* valid but outside the supported set (see each function)     */
+    CHELA_ERR_WORKSPACE = 3,   /* workspace missing or smaller than the query's answer        */
+    CHELA_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (launch, tensor map, ...) */
+    CHELA_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (reported asynchronously) */
+} chela_status_t;
+
+typedef enum { CHELA_F32 = 0, CHELA_BF16 = 1 } chela_dtype_t;
+
+/* CHELA_NORM_RMS: o = r * (mean_j r_j^2 + eps)^(-1/2) over the d_v entries of one head's output
+ * row, no learnable gain -- the library's reading of "Norm" in Eq. 2.  CHELA_NORM_NONE: o = r. */
+typedef enum { CHELA_NORM_NONE = 0, CHELA_NORM_RMS = 1 } chela_norm_t;
+
+const char *chela_status_string(chela_status_t status);
+int chela_version(void);
+
+/* Which linear-attention kernel a call with these arguments dispatches to:
+ * 0 = none (unsupported), 1 = fp32 SIMT kernel, 2 = tcgen05/TMEM/TMA bf16 kernel. */
+int chela_linattn_kernel_kind(int B, int H, int L, int d_k, int d_v, int chunk,
+                              chela_dtype_t in_dtype, chela_dtype_t out_dtype);
+
+/*
+ * Short depthwise causal convolution with optional SiLU (Eq. 7, inner part; Sec. 4.2):
+ *   y[b,t,c] = act( bias[c] + sum_{j=0}^{width-1} w[c,j] * x[b,t-j,c] ),   x[b,t<0,c] = 0.
+ * x, y : [B, L, D] of io_dtype (y may not alias x).  w : [D, width] fp32.  bias : [D] fp32 or NULL.
+ * act : 0 = identity, 1 = SiLU.  Supported: 1 <= width <= 16, D a multiple of 8.
+ */
+chela_status_t chela_shortconv_fwd(const void *x, const float *w, const float *bias, void *y,
+                                   int B, int L, int D, int width, int act,
+                                   chela_dtype_t io_dtype, cudaStream_t stream);
+
+/*
+ * Long convolution (Eq. 6, Sec. 2.2), optionally preceded by the short convolution + SiLU so
+ * that the whole of Eq. 7 is one call:
+ *   a = (w_short ? silu(shortconv(x; w_short)) : x) ;  z[b,t,c] = sum_{s=0}^{t} k_long[c,s] * a[b,t-s,c].
+ * The product is evaluated with fp32 FFTs of size >= 2L (zero padded), so it is the causal
+ * linear convolution, not the circular one.
+ * x : [B, L, D] in_dtype.  k_long : [D, L] fp32.  w_short : [D, short_width] fp32 or NULL.
+ * z : [B, L, D] out_dtype.  Supported: L <= 16384, D a multiple of 8.
+ */
+size_t chela_longconv_workspace_bytes(int B, int L, int D, chela_dtype_t in_dtype,
+                                      chela_dtype_t out_dtype);
+chela_status_t chela_longconv_fwd(const void *x, const float *k_long, const float *w_short,
+                                  int short_width, void *z, int B, int L, int D,
+                                  chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                                  void *workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/*
+ * Chunked causal linear attention forward (Eq. 2 with the causal mask; tiling of Sec. 4.1):
+ *   r_t = scale * sum_{s<=t} <q_t, k_s> v_s ;   o_t = Norm(r_t)
+ * evaluated chunk by chunk: inside a chunk the masked product (Q_i K_i^T . M) V_i, across chunks
+ * Q_i S_{i-1} with the running state S_i = S_{i-1} + K_i^T V_i kept on chip in fp32.
+ * q, k : [B, L, H, d_k] in_dtype.  v : [B, L, H, d_v] in_dtype.  o : [B, L, H, d_v] out_dtype.
+ * L need not be a multiple of chunk.  The result does not depend on chunk beyond rounding.
+ * Supported: d_k = d_v in {64, 128}, chunk in {64, 128}.
+ * Long sequences with few (batch, head) pairs are split along L; the per-split states live in
+ * `workspace` (fp32).
+ */
+size_t chela_linattn_workspace_bytes(int B, int H, int L, int d_k, int d_v, int chunk);
+chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, void *o,
+                                 int B, int H, int L, int d_k, int d_v, int chunk,
+                                 chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                                 chela_norm_t norm, float norm_eps, float scale,
+                                 void *workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/*
+ * Token mixer forward without the gates (Eq. 7, Eqs. 10-12, Eq. 8 without G_a):
+ *   A = silu(shortconv(X));  Z = longconv(A)
+ *   Q = Z W_q + b_q,  K = Z W_k + b_k            (qk_diag = 0: dense D x D weights)
+ *   Q = w_q . Z + b_q,  K = w_k . Z + b_k         (qk_diag = 1: w_q, w_k are length-D scalers, Eqs. 10-11)
+ *   V = act(X W_v + b_v), act = SiLU if v_silu else identity (Eq. 12)
+ *   O = per-head Norm(causal linear attention), head h = columns [h*D/H, (h+1)*D/H), scale 1.
+ * x, o : [B, L, D] (in_dtype / out_dtype).  Dense weights : [D_in, D_out] row-major, in_dtype.
+ * qk_diag scalers : [D], in_dtype.  Biases : [D] fp32 or NULL.  w_short : [D, short_width] fp32.
+ * k_long : [D, L] fp32.  Supported: D/H in {64, 128}, chunk in {64, 128}, L <= 16384.
+ */
+size_t chela_mixer_workspace_bytes(int B, int L, int D, int H, int chunk, chela_dtype_t in_dtype);
+chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_width,
+                               const float *k_long, const void *w_q, const void *w_k,
+                               const void *w_v, const float *b_q, const float *b_k,
+                               const float *b_v, int qk_diag, int v_silu, void *o, int B, int L,
+                               int D, int H, int chunk, chela_dtype_t in_dtype,
+                               chela_dtype_t out_dtype, chela_norm_t norm, float norm_eps,
+                               void *workspace, size_t workspace_bytes, cudaStream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CHELA_H_ */

@@ -1,0 +1,166 @@
+"""Thin Python binding of libchela's C ABI (argument marshalling only).
+
+Each function mirrors the C entry point of the same name: it reads shapes and device pointers
+from torch tensors, allocates the output and the workspace with torch, and passes torch's
+current CUDA stream.  Every step of the computation runs in the library's kernels.  There is no
+CPU fallback: if ``libchela.so`` has not been built (``python -m paper_2406_08128_b200.build``)
+loading fails with an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libchela.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+F32, BF16 = 0, 1
+NORM_NONE, NORM_RMS = 0, 1
+
+_DTYPES = {torch.float32: F32, torch.bfloat16: BF16}
+_lib = None
+
+_c_int, _c_float, _c_size_t, _vp = ctypes.c_int, ctypes.c_float, ctypes.c_size_t, ctypes.c_void_p
+
+_SIGNATURES = {
+    "chela_status_string": (ctypes.c_char_p, [_c_int]),
+    "chela_version": (_c_int, []),
+    "chela_linattn_kernel_kind": (_c_int, [_c_int] * 6 + [_c_int, _c_int]),
+    "chela_shortconv_fwd": (_c_int, [_vp, _vp, _vp, _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _vp]),
+    "chela_longconv_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int, _c_int, _c_int]),
+    "chela_longconv_fwd": (_c_int, [_vp, _vp, _vp, _c_int, _vp, _c_int, _c_int, _c_int, _c_int, _c_int,
+                                    _vp, _c_size_t, _vp]),
+    "chela_linattn_workspace_bytes": (_c_size_t, [_c_int] * 6),
+    "chela_linattn_fwd": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
+                                   _c_float, _vp, _c_size_t, _vp]),
+    "chela_mixer_workspace_bytes": (_c_size_t, [_c_int] * 5 + [_c_int]),
+    "chela_mixer_fwd": (_c_int, [_vp, _vp, _c_int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _c_int, _c_int, _vp,
+                                 _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_float,
+                                 _vp, _c_size_t, _vp]),
+}
+
+
+class ChelaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+
+
+def exported_symbols():
+    """Names the C header declares (the loader resolves every one of them)."""
+    return sorted(_SIGNATURES)
+
+
+def lib():
+    """Load libchela.so (once).  Raises if the library has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libchela.so is missing: build it with `python -m paper_2406_08128_b200.build` "
+                               "(there is no CPU fallback)")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().chela_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib().chela_version())
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise ChelaError(int(status), where)
+
+
+def _ptr(t):
+    return None if t is None else _vp(t.data_ptr())
+
+
+def _stream():
+    return _vp(torch.cuda.current_stream().cuda_stream)
+
+
+def _dt(t) -> int:
+    return _DTYPES[t.dtype]
+
+
+def _tdtype(code: int):
+    return torch.float32 if code == F32 else torch.bfloat16
+
+
+def _workspace(nbytes: int, device):
+    return torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=device)
+
+
+def linattn_kernel_kind(B, H, L, d_k, d_v, chunk, in_dtype=BF16, out_dtype=F32) -> int:
+    return int(lib().chela_linattn_kernel_kind(B, H, L, d_k, d_v, chunk, in_dtype, out_dtype))
+
+
+def shortconv_fwd(x, w, bias=None, act=True, out=None):
+    """x [B,L,D] (bf16/f32), w [D,width] f32 -> y like x."""
+    B, L, D = x.shape
+    y = torch.empty_like(x) if out is None else out
+    _check(lib().chela_shortconv_fwd(_ptr(x), _ptr(w), _ptr(bias), _ptr(y), B, L, D, w.shape[1], int(bool(act)),
+                                     _dt(x), _stream()), "chela_shortconv_fwd")
+    return y
+
+
+def longconv_workspace_bytes(B, L, D, in_dtype=BF16, out_dtype=F32) -> int:
+    return int(lib().chela_longconv_workspace_bytes(B, L, D, in_dtype, out_dtype))
+
+
+def longconv_fwd(x, k_long, w_short=None, out_dtype=F32, out=None, workspace=None):
+    """x [B,L,D], k_long [D,L] f32, optional short taps [D,width] f32 -> z [B,L,D] of out_dtype."""
+    B, L, D = x.shape
+    z = torch.empty((B, L, D), dtype=_tdtype(out_dtype), device=x.device) if out is None else out
+    if workspace is None:
+        workspace = _workspace(longconv_workspace_bytes(B, L, D, _dt(x), out_dtype), x.device)
+    width = 0 if w_short is None else w_short.shape[1]
+    _check(lib().chela_longconv_fwd(_ptr(x), _ptr(k_long), _ptr(w_short), width, _ptr(z), B, L, D, _dt(x),
+                                    _dt(z), _ptr(workspace), workspace.numel(), _stream()), "chela_longconv_fwd")
+    return z
+
+
+def linattn_workspace_bytes(B, H, L, d_k, d_v, chunk) -> int:
+    return int(lib().chela_linattn_workspace_bytes(B, H, L, d_k, d_v, chunk))
+
+
+def linattn_fwd(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale=1.0, out=None, workspace=None):
+    """q,k [B,L,H,d_k], v [B,L,H,d_v] -> o [B,L,H,d_v] of out_dtype."""
+    B, L, H, d_k = q.shape
+    d_v = v.shape[3]
+    o = torch.empty((B, L, H, d_v), dtype=_tdtype(out_dtype), device=q.device) if out is None else out
+    if workspace is None:
+        workspace = _workspace(linattn_workspace_bytes(B, H, L, d_k, d_v, chunk), q.device)
+    _check(lib().chela_linattn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, L, d_k, d_v, chunk, _dt(q), _dt(o),
+                                   int(norm), float(eps), float(scale), _ptr(workspace), workspace.numel(),
+                                   _stream()), "chela_linattn_fwd")
+    return o
+
+
+def mixer_workspace_bytes(B, L, D, H, chunk, in_dtype=BF16) -> int:
+    return int(lib().chela_mixer_workspace_bytes(B, L, D, H, chunk, in_dtype))
+
+
+def mixer_fwd(x, w_short, k_long, w_q, w_k, w_v, H, chunk=64, b_q=None, b_k=None, b_v=None, qk_diag=False,
+              v_silu=True, out_dtype=F32, norm=NORM_RMS, eps=1e-6, out=None, workspace=None):
+    """x [B,L,D] -> o [B,L,D]; weights as in the C header."""
+    B, L, D = x.shape
+    o = torch.empty((B, L, D), dtype=_tdtype(out_dtype), device=x.device) if out is None else out
+    if workspace is None:
+        workspace = _workspace(mixer_workspace_bytes(B, L, D, H, chunk, _dt(x)), x.device)
+    _check(lib().chela_mixer_fwd(_ptr(x), _ptr(w_short), w_short.shape[1], _ptr(k_long), _ptr(w_q), _ptr(w_k),
+                                 _ptr(w_v), _ptr(b_q), _ptr(b_k), _ptr(b_v), int(bool(qk_diag)),
+                                 int(bool(v_silu)), _ptr(o), B, L, D, H, chunk, _dt(x), _dt(o), int(norm),
+                                 float(eps), _ptr(workspace), workspace.numel(), _stream()), "chela_mixer_fwd")
+    return o

@@ -1,0 +1,169 @@
+// C ABI entry points: argument validation, workspace carving and dispatch.  No kernel code here.
+#include "common.cuh"
+
+using namespace chela;
+
+namespace {
+
+bool dtype_ok(chela_dtype_t t) { return t == CHELA_F32 || t == CHELA_BF16; }
+
+struct MixerPlan {
+    size_t off_conv, off_z, off_q, off_k, off_v, off_attn, total;
+    size_t conv_bytes, attn_bytes;
+};
+MixerPlan mixer_plan(int B, int L, int D, int H, int chunk)
+{
+    MixerPlan p;
+    const size_t act = align_up((size_t)B * L * D * sizeof(float), 256);
+    p.conv_bytes = longconv_workspace_bytes(B, L, D);
+    p.attn_bytes = chela_linattn_workspace_bytes(B, H, L, D / H, D / H, chunk);
+    p.off_conv = 0;
+    p.off_z = align_up(p.conv_bytes, 256);
+    p.off_q = p.off_z + act;
+    p.off_k = p.off_q + act;
+    p.off_v = p.off_k + act;
+    p.off_attn = p.off_v + act;
+    p.total = p.off_attn + align_up(p.attn_bytes, 256);
+    return p;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *chela_status_string(chela_status_t status)
+{
+    switch (status) {
+        case CHELA_OK: return "ok";
+        case CHELA_ERR_INVALID_ARG: return "invalid argument";
+        case CHELA_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case CHELA_ERR_WORKSPACE: return "workspace missing or too small";
+        case CHELA_ERR_CUDA: return "CUDA call failed";
+        case CHELA_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int chela_version(void) { return 100; }
+
+int chela_linattn_kernel_kind(int B, int H, int L, int d_k, int d_v, int chunk, chela_dtype_t in_dtype,
+                              chela_dtype_t out_dtype)
+{
+    if (B < 1 || H < 1 || L < 1 || !dtype_ok(in_dtype) || !dtype_ok(out_dtype)) return 0;
+    if (d_k != d_v || (d_k != 64 && d_k != 128) || (chunk != 64 && chunk != 128)) return 0;
+    if (linattn_sm100_supported(B, H, L, d_k, chunk, in_dtype, out_dtype)) return 2;
+    return 1;
+}
+
+chela_status_t chela_shortconv_fwd(const void *x, const float *w, const float *bias, void *y, int B, int L,
+                                   int D, int width, int act, chela_dtype_t io_dtype, cudaStream_t stream)
+{
+    if (!x || !w || !y || x == y || B < 1 || L < 1 || D < 1 || !dtype_ok(io_dtype) || (act != 0 && act != 1))
+        return CHELA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y)) return CHELA_ERR_INVALID_ARG;
+    if (width < 1 || width > 16 || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
+    return launch_shortconv(x, w, bias, y, B, L, D, width, act, io_dtype, stream);
+}
+
+size_t chela_longconv_workspace_bytes(int B, int L, int D, chela_dtype_t, chela_dtype_t)
+{
+    if (B < 1 || L < 1 || D < 1) return 0;
+    return longconv_workspace_bytes(B, L, D);
+}
+
+chela_status_t chela_longconv_fwd(const void *x, const float *k_long, const float *w_short, int short_width,
+                                  void *z, int B, int L, int D, chela_dtype_t in_dtype,
+                                  chela_dtype_t out_dtype, void *workspace, size_t workspace_bytes,
+                                  cudaStream_t stream)
+{
+    if (!x || !k_long || !z || B < 1 || L < 1 || D < 1 || !dtype_ok(in_dtype) || !dtype_ok(out_dtype))
+        return CHELA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(z) || !aligned16(workspace)) return CHELA_ERR_INVALID_ARG;
+    if (L > 16384 || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
+    if (w_short && (short_width < 1 || short_width > 16)) return CHELA_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < longconv_workspace_bytes(B, L, D)) return CHELA_ERR_WORKSPACE;
+    return launch_longconv(x, k_long, w_short, short_width, z, B, L, D, in_dtype, out_dtype, workspace, stream);
+}
+
+size_t chela_linattn_workspace_bytes(int B, int H, int L, int d_k, int d_v, int chunk)
+{
+    if (B < 1 || H < 1 || L < 1 || d_k != d_v || (d_k != 64 && d_k != 128) || (chunk != 64 && chunk != 128))
+        return 0;
+    return linattn_sm100_workspace_bytes(B, H, L, d_k, chunk);
+}
+
+chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
+                                 int d_k, int d_v, int chunk, chela_dtype_t in_dtype,
+                                 chela_dtype_t out_dtype, chela_norm_t norm, float norm_eps, float scale,
+                                 void *workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    if (!q || !k || !v || !o || B < 1 || H < 1 || L < 1 || d_k < 1 || d_v < 1 || chunk < 1 ||
+        !dtype_ok(in_dtype) || !dtype_ok(out_dtype) || (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) ||
+        !(norm_eps >= 0.f))
+        return CHELA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(workspace))
+        return CHELA_ERR_INVALID_ARG;
+    const int kind = chela_linattn_kernel_kind(B, H, L, d_k, d_v, chunk, in_dtype, out_dtype);
+    if (kind == 0) return CHELA_ERR_UNSUPPORTED;
+    if (kind == 2) {
+        const size_t need = linattn_sm100_workspace_bytes(B, H, L, d_k, chunk);
+        if (need && (!workspace || workspace_bytes < need)) return CHELA_ERR_WORKSPACE;
+        return launch_linattn_sm100(q, k, v, o, B, H, L, d_k, chunk, in_dtype, out_dtype, (int)norm, norm_eps,
+                                    scale, workspace, stream);
+    }
+    return launch_linattn_simt(q, k, v, o, B, H, L, d_k, chunk, in_dtype, out_dtype, (int)norm, norm_eps, scale,
+                               stream);
+}
+
+size_t chela_mixer_workspace_bytes(int B, int L, int D, int H, int chunk, chela_dtype_t)
+{
+    if (B < 1 || L < 1 || D < 1 || H < 1 || D % H != 0) return 0;
+    return mixer_plan(B, L, D, H, chunk).total;
+}
+
+chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_width, const float *k_long,
+                               const void *w_q, const void *w_k, const void *w_v, const float *b_q,
+                               const float *b_k, const float *b_v, int qk_diag, int v_silu, void *o, int B,
+                               int L, int D, int H, int chunk, chela_dtype_t in_dtype,
+                               chela_dtype_t out_dtype, chela_norm_t norm, float norm_eps, void *workspace,
+                               size_t workspace_bytes, cudaStream_t stream)
+{
+    if (!x || !w_short || !k_long || !w_q || !w_k || !w_v || !o || B < 1 || L < 1 || D < 1 || H < 1 ||
+        !dtype_ok(in_dtype) || !dtype_ok(out_dtype) || (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) ||
+        !(norm_eps >= 0.f))
+        return CHELA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(o) || !aligned16(w_q) || !aligned16(w_k) || !aligned16(w_v) ||
+        !aligned16(workspace))
+        return CHELA_ERR_INVALID_ARG;
+    if (D % H != 0) return CHELA_ERR_INVALID_ARG;
+    const int d = D / H;
+    if ((d != 64 && d != 128) || (chunk != 64 && chunk != 128) || L > 16384 || short_width < 1 || short_width > 16)
+        return CHELA_ERR_UNSUPPORTED;
+    const MixerPlan p = mixer_plan(B, L, D, H, chunk);
+    if (!workspace || workspace_bytes < p.total) return CHELA_ERR_WORKSPACE;
+    char *ws = (char *)workspace;
+    float *z = (float *)(ws + p.off_z), *qq = (float *)(ws + p.off_q), *kk = (float *)(ws + p.off_k),
+          *vv = (float *)(ws + p.off_v);
+    const size_t M = (size_t)B * L;
+
+    // Z = K_l(silu(K_s(X)))  (Eq. 7), kept in fp32
+    chela_status_t st = launch_longconv(x, k_long, w_short, short_width, z, B, L, D, in_dtype, CHELA_F32,
+                                        ws + p.off_conv, stream);
+    if (st != CHELA_OK) return st;
+    // Q, K from Z (Eqs. 10-11, or dense projections), V from X (Eq. 12)
+    if (qk_diag) {
+        st = launch_affine(z, w_q, b_q, qq, M, D, in_dtype, stream);
+        if (st == CHELA_OK) st = launch_affine(z, w_k, b_k, kk, M, D, in_dtype, stream);
+    } else {
+        st = launch_gemm_simt(z, w_q, b_q, qq, M, D, D, 0, CHELA_F32, in_dtype, CHELA_F32, stream);
+        if (st == CHELA_OK) st = launch_gemm_simt(z, w_k, b_k, kk, M, D, D, 0, CHELA_F32, in_dtype, CHELA_F32, stream);
+    }
+    if (st != CHELA_OK) return st;
+    st = launch_gemm_simt(x, w_v, b_v, vv, M, D, D, v_silu ? 1 : 0, in_dtype, in_dtype, CHELA_F32, stream);
+    if (st != CHELA_OK) return st;
+    // [B,L,D] with head h = columns [h*d,(h+1)*d) is [B,L,H,d]
+    return chela_linattn_fwd(qq, kk, vv, o, B, H, L, d, d, chunk, CHELA_F32, out_dtype, norm, norm_eps, 1.0f,
+                             ws + p.off_attn, p.attn_bytes, stream);
+}
+
+}  // extern "C"

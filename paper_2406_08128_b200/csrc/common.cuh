@@ -1,0 +1,77 @@
+// Internal helpers shared by the CUDA translation units of libchela (not part of the C ABI).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "chela.h"
+
+namespace chela {
+
+inline chela_status_t cuda_status(cudaError_t e) { return e == cudaSuccess ? CHELA_OK : CHELA_ERR_CUDA; }
+inline chela_status_t last_launch_status() { return cuda_status(cudaGetLastError()); }
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int next_pow2(int x) { int p = 1; while (p < x) p <<= 1; return p; }
+inline size_t dtype_size(chela_dtype_t t) { return t == CHELA_BF16 ? 2 : 4; }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+__device__ __forceinline__ float silu_f(float u) { return u / (1.0f + __expf(-u)); }
+
+// Load / store 4 consecutive elements as fp32.
+__device__ __forceinline__ float4 load4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16 *p)
+{
+    uint2 u = *reinterpret_cast<const uint2 *>(p);
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&u.x);
+    __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162 *>(&u.y);
+    float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+    return make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+__device__ __forceinline__ void store4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+__device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v)
+{
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t *>(&a);
+    u.y = *reinterpret_cast<uint32_t *>(&b);
+    *reinterpret_cast<uint2 *>(p) = u;
+}
+__device__ __forceinline__ float load1(const float *p) { return *p; }
+__device__ __forceinline__ float load1(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void store1(float *p, float v) { *p = v; }
+__device__ __forceinline__ void store1(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
+// ---- launchers implemented in the other translation units ------------------------------------
+
+chela_status_t launch_linattn_simt(const void *q, const void *k, const void *v, void *o, int B, int H,
+                                   int L, int d, int chunk, chela_dtype_t in_dtype,
+                                   chela_dtype_t out_dtype, int norm, float eps, float scale,
+                                   cudaStream_t stream);
+
+// tcgen05/TMEM/TMA kernel for bf16 inputs
+bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_t in_dtype,
+                             chela_dtype_t out_dtype);
+size_t linattn_sm100_workspace_bytes(int B, int H, int L, int d, int chunk);
+chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v, void *o, int B, int H,
+                                    int L, int d, int chunk, chela_dtype_t in_dtype,
+                                    chela_dtype_t out_dtype, int norm, float eps, float scale,
+                                    void *workspace, cudaStream_t stream);
+
+chela_status_t launch_shortconv(const void *x, const float *w, const float *bias, void *y, int B, int L,
+                                int D, int width, int act, chela_dtype_t io_dtype, cudaStream_t stream);
+
+size_t longconv_workspace_bytes(int B, int L, int D);
+chela_status_t launch_longconv(const void *x, const float *k_long, const float *w_short, int short_width,
+                               void *z, int B, int L, int D, chela_dtype_t in_dtype,
+                               chela_dtype_t out_dtype, void *workspace, cudaStream_t stream);
+
+// y[M,N] = act(a[M,K] w[K,N] + bias[N]); a: a_dtype, w: w_dtype, y: y_dtype.
+chela_status_t launch_gemm_simt(const void *a, const void *w, const float *bias, void *y, size_t M, int K,
+                                int N, int act, chela_dtype_t a_dtype, chela_dtype_t w_dtype,
+                                chela_dtype_t y_dtype, cudaStream_t stream);
+// y[m,c] = alpha[c] * z[m,c] + beta[c]
+chela_status_t launch_affine(const float *z, const void *alpha, const float *beta, float *y, size_t M, int D,
+                             chela_dtype_t alpha_dtype, cudaStream_t stream);
+
+}  // namespace chela

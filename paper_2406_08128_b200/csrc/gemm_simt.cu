@@ -1,0 +1,116 @@
+// fp32 SIMT GEMM for the Q/K/V formation of the mixer (Eqs. 10-12): y = act(a w + bias).
+// 128 x 128 x 16 tiles, 256 threads, 8 x 8 outputs per thread, fp32 FFMA accumulation.  It keeps
+// the long-convolution output Z and the resulting Q, K in fp32, which the normalised mixer
+// output needs (bf16 Q/K lose the result's leading digits to cancellation in Q K^T).
+#include "common.cuh"
+
+namespace chela {
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 16;
+
+template <typename TA, typename TW, typename TY>
+__global__ void __launch_bounds__(256)
+gemm_simt_kernel(const TA *__restrict__ a, const TW *__restrict__ w, const float *__restrict__ bias,
+                 TY *__restrict__ y, size_t M, int K, int N, int act)
+{
+    __shared__ float sA[BK][BM + 4];  // a tile transposed: [k][m]
+    __shared__ float sW[BK][BN + 4];  // [k][n]
+    const int tid = threadIdx.x;
+    const size_t m0 = (size_t)blockIdx.y * BM;
+    const int n0 = blockIdx.x * BN;
+    const int tm = (tid / 16) * 8, tn = (tid % 16) * 8;
+    float acc[8][8] = {};
+
+    for (int k0 = 0; k0 < K; k0 += BK) {
+        // a tile: 128 rows x 16 k; 2048 elements, 8 per thread
+        for (int idx = tid; idx < BM * BK; idx += 256) {
+            const int r = idx / BK, kk = idx % BK;
+            const size_t m = m0 + r;
+            sA[kk][r] = (m < M && k0 + kk < K) ? load1(a + m * K + k0 + kk) : 0.f;
+        }
+        for (int idx = tid; idx < BK * BN; idx += 256) {
+            const int kk = idx / BN, c = idx % BN;
+            sW[kk][c] = (k0 + kk < K && n0 + c < N) ? load1(w + (size_t)(k0 + kk) * N + n0 + c) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            const float4 a0 = load4(&sA[kk][tm]), a1 = load4(&sA[kk][tm + 4]);
+            const float4 w0 = load4(&sW[kk][tn]), w1 = load4(&sW[kk][tn + 4]);
+            const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(av[i], wv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const size_t m = m0 + tm + i;
+        if (m >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int n = n0 + tn + j;
+            if (n >= N) continue;
+            float r = acc[i][j] + (bias ? bias[n] : 0.f);
+            if (act) r = silu_f(r);
+            store1(y + m * N + n, r);
+        }
+    }
+}
+
+template <typename TA, typename TW, typename TY>
+chela_status_t launch_t(const void *a, const void *w, const float *bias, void *y, size_t M, int K, int N,
+                        int act, cudaStream_t stream)
+{
+    dim3 grid((N + BN - 1) / BN, (unsigned)((M + BM - 1) / BM));
+    gemm_simt_kernel<TA, TW, TY><<<grid, 256, 0, stream>>>((const TA *)a, (const TW *)w, bias, (TY *)y, M, K, N, act);
+    return last_launch_status();
+}
+
+template <typename TW>
+__global__ void affine_kernel(const float *__restrict__ z, const TW *__restrict__ alpha,
+                              const float *__restrict__ beta, float *__restrict__ y, size_t n, int D)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % D);
+        y[i] = fmaf(load1(alpha + c), z[i], beta ? beta[c] : 0.f);
+    }
+}
+
+}  // namespace
+
+chela_status_t launch_gemm_simt(const void *a, const void *w, const float *bias, void *y, size_t M, int K,
+                                int N, int act, chela_dtype_t a_dtype, chela_dtype_t w_dtype,
+                                chela_dtype_t y_dtype, cudaStream_t stream)
+{
+    typedef __nv_bfloat16 bf;
+    const int key = (a_dtype == CHELA_BF16) * 4 + (w_dtype == CHELA_BF16) * 2 + (y_dtype == CHELA_BF16);
+    switch (key) {
+        case 0: return launch_t<float, float, float>(a, w, bias, y, M, K, N, act, stream);
+        case 1: return launch_t<float, float, bf>(a, w, bias, y, M, K, N, act, stream);
+        case 2: return launch_t<float, bf, float>(a, w, bias, y, M, K, N, act, stream);
+        case 3: return launch_t<float, bf, bf>(a, w, bias, y, M, K, N, act, stream);
+        case 4: return launch_t<bf, float, float>(a, w, bias, y, M, K, N, act, stream);
+        case 5: return launch_t<bf, float, bf>(a, w, bias, y, M, K, N, act, stream);
+        case 6: return launch_t<bf, bf, float>(a, w, bias, y, M, K, N, act, stream);
+        default: return launch_t<bf, bf, bf>(a, w, bias, y, M, K, N, act, stream);
+    }
+}
+
+chela_status_t launch_affine(const float *z, const void *alpha, const float *beta, float *y, size_t M, int D,
+                             chela_dtype_t alpha_dtype, cudaStream_t stream)
+{
+    const size_t n = M * D;
+    const int blocks = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
+    if (alpha_dtype == CHELA_BF16)
+        affine_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>(z, (const __nv_bfloat16 *)alpha, beta, y, n, D);
+    else
+        affine_kernel<float><<<blocks, 256, 0, stream>>>(z, (const float *)alpha, beta, y, n, D);
+    return last_launch_status();
+}
+
+}  // namespace chela

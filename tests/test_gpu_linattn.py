@@ -1,0 +1,94 @@
+"""GPU parity: chela_linattn_fwd (through the C ABI) against the float64 oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2406_08128_b200 import chela, inputs
+from util import rel_err, to_device, to_numpy
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}   # max|err| / RMS(oracle output)
+
+
+def run(q, k, v, dtype, chunk, norm=True, scale=1.0, out_dtype=chela.F32):
+    import torch
+    o = chela.linattn_fwd(to_device(q, dtype), to_device(k, dtype), to_device(v, dtype), chunk=chunk,
+                          out_dtype=out_dtype, norm=chela.NORM_RMS if norm else chela.NORM_NONE, scale=scale)
+    torch.cuda.synchronize()
+    return to_numpy(o)
+
+
+def test_config1_fp32_quadratic_and_recurrent():
+    # B=1, H=1, L=1024, d=64, C=64, seed 0, N(0,1)/sqrt(64)
+    q, k, v = inputs.qkv(0, 1, 1024, 1, 64, 64, "f32")
+    for norm in (True, False):
+        got = run(q, k, v, "f32", 64, norm=norm)
+        assert rel_err(got, oracle.linattn_quadratic(q, k, v, norm=norm)) <= TOL["f32"]
+        assert rel_err(got, oracle.linattn_recurrent(q, k, v, norm=norm)) <= TOL["f32"]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d,chunk", [(64, 64), (64, 128), (128, 64), (128, 128)])
+@pytest.mark.parametrize("L", [1, 63, 64, 65, 200, 333])
+def test_small_shapes_ragged_tails(dtype, d, chunk, L):
+    B, H = 2, 3
+    q, k, v = inputs.qkv(10 + L, B, L, H, d, d, dtype)
+    for norm in (True, False):
+        got = run(q, k, v, dtype, chunk, norm=norm)
+        ref = oracle.linattn_recurrent(q, k, v, norm=norm)
+        assert rel_err(got, ref) <= TOL[dtype], (dtype, d, chunk, L, norm)
+
+
+def test_config2_bf16_full_size():
+    # B=8, H=8, L=4096, d=64, C=64
+    q, k, v = inputs.qkv(1, 8, 4096, 8, 64, 64, "bf16")
+    got = run(q, k, v, "bf16", 64)
+    ref = oracle.linattn_recurrent(q, k, v)
+    assert rel_err(got, ref) <= TOL["bf16"]
+    # a few (b,h) pairs also against the quadratic definition
+    for b, h in ((0, 0), (7, 7), (3, 5)):
+        sl = (slice(b, b + 1), slice(None), slice(h, h + 1))
+        quad = oracle.linattn_quadratic(q[sl], k[sl], v[sl])
+        assert rel_err(got[sl], quad) <= TOL["bf16"]
+
+
+def test_chunk_invariance_and_causality_on_gpu():
+    q, k, v = inputs.qkv(5, 2, 700, 4, 64, 64, "bf16")
+    a = run(q, k, v, "bf16", 64)
+    b = run(q, k, v, "bf16", 128)
+    assert rel_err(a, b) <= TOL["bf16"]
+    q2, k2, v2 = inputs.qkv(6, 2, 700, 4, 64, 64, "bf16")
+    t0 = 389
+    for x, y in ((q2, q), (k2, k), (v2, v)):
+        x[:, :t0] = y[:, :t0]
+    c = run(q2, k2, v2, "bf16", 64)
+    assert np.array_equal(a[:, :t0], c[:, :t0])
+    assert not np.allclose(a[:, t0:], c[:, t0:])
+
+
+def test_scale_and_bf16_output():
+    q, k, v = inputs.qkv(7, 1, 300, 2, 64, 64, "bf16")
+    got = run(q, k, v, "bf16", 64, norm=False, scale=0.125)
+    assert rel_err(got, oracle.linattn_recurrent(q, k, v, scale=0.125, norm=False)) <= TOL["bf16"]
+    got = run(q, k, v, "bf16", 64, out_dtype=chela.BF16)
+    # bf16 storage of a unit-RMS row costs up to 2^-8 relative per element
+    assert rel_err(got, oracle.linattn_recurrent(q, k, v)) <= 3e-2
+
+
+@pytest.mark.parametrize("B,L", inputs.sweep_shapes())
+def test_sweep_shapes_sampled(B, L):
+    """Full sweep sizes (B*L = 262144, H=16, d=64, C=64): the oracle checks sampled (b,h) pairs."""
+    import torch
+    H, d = 16, 64
+    q, k, v = inputs.qkv(100 + int(np.log2(L)), B, L, H, d, d, "bf16")
+    o = chela.linattn_fwd(to_device(q, "bf16"), to_device(k, "bf16"), to_device(v, "bf16"), chunk=64)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(L)
+    pairs = {(0, 0), (B - 1, H - 1)} | {(int(rng.integers(B)), int(rng.integers(H))) for _ in range(4)}
+    for b, h in pairs:
+        sl = (slice(b, b + 1), slice(None), slice(h, h + 1))
+        ref = oracle.linattn_recurrent(q[sl], k[sl], v[sl])
+        got = to_numpy(o[b:b + 1, :, h:h + 1])
+        assert rel_err(got, ref) <= TOL["bf16"], (B, L, b, h)
+    assert bool(torch.isfinite(o).all())
