@@ -25,7 +25,10 @@ def test_shortconv(dtype, tol, B, L, D, width, act):
     bias = rng.standard_normal(D, dtype=np.float32) if L % 2 else None
     got = to_numpy(chela.shortconv_fwd(to_device(x, dtype), dev_f32(w), None if bias is None else dev_f32(bias), act=act))
     ref = oracle.shortconv(x, w, bias=bias, act=act)
-    assert rel_err(got, ref) <= tol  # bf16: output storage rounding only
+    if dtype == "bf16":  # output storage rounding only: half an ulp of the largest element
+        assert np.abs(got - ref).max() <= 2.0 ** -8 * np.abs(ref).max()
+    else:
+        assert rel_err(got, ref) <= tol
 
 
 @pytest.mark.parametrize("B,L,D", [(1, 1, 8), (2, 3, 8), (2, 5, 16), (1, 16, 8), (2, 17, 24), (1, 64, 8),
@@ -49,4 +52,4 @@ def test_longconv_f32_input_and_bf16_output():
     m = inputs.mixer(7, B, L, D, dtype="f32")
     z = to_numpy(chela.longconv_fwd(to_device(m["x"], "f32"), dev_f32(m["k_long"]), out_dtype=chela.BF16))
     ref = oracle.longconv_fft(m["x"], m["k_long"])
-    assert rel_err(z, ref) <= 3e-2  # bf16 storage of the output
+    assert np.abs(z - ref).max() <= 2.0 ** -8 * np.abs(ref).max()  # bf16 storage of the output

@@ -72,8 +72,9 @@ def test_scale_and_bf16_output():
     got = run(q, k, v, "bf16", 64, norm=False, scale=0.125)
     assert rel_err(got, oracle.linattn_recurrent(q, k, v, scale=0.125, norm=False)) <= TOL["bf16"]
     got = run(q, k, v, "bf16", 64, out_dtype=chela.BF16)
-    # bf16 storage of a unit-RMS row costs up to 2^-8 relative per element
-    assert rel_err(got, oracle.linattn_recurrent(q, k, v)) <= 3e-2
+    # bf16 storage costs up to half an ulp (2^-8 relative) of the largest element on top of the bound
+    ref = oracle.linattn_recurrent(q, k, v)
+    assert np.abs(got - ref).max() <= 2e-2 * np.sqrt(np.mean(ref ** 2)) + 2.0 ** -8 * np.abs(ref).max()
 
 
 @pytest.mark.parametrize("B,L", inputs.sweep_shapes())
