@@ -101,6 +101,16 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
                                  void *workspace, size_t workspace_bytes, cudaStream_t stream);
 
 /*
+ * Asynchronous status of the last chela_linattn_fwd / chela_mixer_fwd launch that used `workspace`.
+ * Device-side waits in the tensor-core kernel are bounded; a wait that gives up makes its CTA stop
+ * cleanly and records CHELA_ERR_TIMEOUT in the first word of the workspace.  This call synchronises
+ * `stream`, copies that word to the host and returns it (CHELA_OK if nothing was recorded, or if the
+ * launch used a kernel without device-side waits).  `workspace` must be the pointer given to the
+ * launch (for the mixer: its own workspace pointer).
+ */
+chela_status_t chela_async_status(const void *workspace, cudaStream_t stream);
+
+/*
  * Token mixer forward without the gates (Eq. 7, Eqs. 10-12, Eq. 8 without G_a):
  *   A = silu(shortconv(X));  Z = longconv(A)
  *   Q = Z W_q + b_q,  K = Z W_k + b_k            (qk_diag = 0: dense D x D weights)

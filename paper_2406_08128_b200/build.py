@@ -45,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if p.wait() != 0:
             raise RuntimeError("nvcc failed on %s" % src)
     tmp = LIB + ".tmp.%d" % os.getpid()
-    subprocess.check_call([nvcc, "-shared", "-o", tmp, *objs, "-lcuda", "-lcudart"])
+    subprocess.check_call([nvcc, "-shared", "-o", tmp, *objs, "-lcudart"])
     os.replace(tmp, LIB)
     return LIB
 

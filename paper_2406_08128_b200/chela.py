@@ -36,6 +36,7 @@ _SIGNATURES = {
     "chela_linattn_workspace_bytes": (_c_size_t, [_c_int] * 6),
     "chela_linattn_fwd": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                    _c_float, _vp, _c_size_t, _vp]),
+    "chela_async_status": (_c_int, [_vp, _vp]),
     "chela_mixer_workspace_bytes": (_c_size_t, [_c_int] * 5 + [_c_int]),
     "chela_mixer_fwd": (_c_int, [_vp, _vp, _c_int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _c_int, _c_int, _vp,
                                  _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_float,
@@ -146,6 +147,11 @@ def linattn_fwd(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale
                                    int(norm), float(eps), float(scale), _ptr(workspace), workspace.numel(),
                                    _stream()), "chela_linattn_fwd")
     return o
+
+
+def async_status(workspace) -> int:
+    """Synchronise the current stream and return the asynchronous status recorded in ``workspace``."""
+    return int(lib().chela_async_status(_ptr(workspace), _stream()))
 
 
 def mixer_workspace_bytes(B, L, D, H, chunk, in_dtype=BF16) -> int:

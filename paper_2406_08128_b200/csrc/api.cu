@@ -17,13 +17,13 @@ MixerPlan mixer_plan(int B, int L, int D, int H, int chunk)
     const size_t act = align_up((size_t)B * L * D * sizeof(float), 256);
     p.conv_bytes = longconv_workspace_bytes(B, L, D);
     p.attn_bytes = chela_linattn_workspace_bytes(B, H, L, D / H, D / H, chunk);
-    p.off_conv = 0;
-    p.off_z = align_up(p.conv_bytes, 256);
+    p.off_attn = 0;  // first, so that the asynchronous status word heads the mixer workspace too
+    p.off_conv = align_up(p.attn_bytes, 256);
+    p.off_z = p.off_conv + align_up(p.conv_bytes, 256);
     p.off_q = p.off_z + act;
     p.off_k = p.off_q + act;
     p.off_v = p.off_k + act;
-    p.off_attn = p.off_v + act;
-    p.total = p.off_attn + align_up(p.attn_bytes, 256);
+    p.total = p.off_v + act;
     return p;
 }
 
@@ -113,6 +113,16 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
     }
     return launch_linattn_simt(q, k, v, o, B, H, L, d_k, chunk, in_dtype, out_dtype, (int)norm, norm_eps, scale,
                                stream);
+}
+
+chela_status_t chela_async_status(const void *workspace, cudaStream_t stream)
+{
+    if (!workspace) return CHELA_ERR_INVALID_ARG;
+    int word = 0;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return CHELA_ERR_CUDA;
+    return word == (int)CHELA_ERR_TIMEOUT ? CHELA_ERR_TIMEOUT : CHELA_OK;
 }
 
 size_t chela_mixer_workspace_bytes(int B, int L, int D, int H, int chunk, chela_dtype_t)

@@ -1,11 +1,471 @@
-// placeholder until the tensor-core kernel lands
+// Chunked causal linear attention for bf16 inputs on sm_100a: tcgen05 tensor-core tiles with TMEM
+// accumulators, operands staged by TMA (Sec. 4.1 tiling of Eq. 2 with the causal mask).
+//
+// One CTA (128 threads) walks one (batch, head) sequence chunk by chunk.  Per chunk of C tokens:
+//   TMA      : Q_i, K_i, V_i tiles ([C rows] x 128 B, 128-byte swizzle) into a 2-stage ring
+//   MMA 1    : P = Q_i K_i^T                      -> TMEM   (both operands K-major)
+//   threads  : P -> registers, causal mask, bf16  -> shared (K-major tile for the next MMA)
+//   MMA 2    : O = Q_i S_hi + Q_i S_lo + P V_i    -> TMEM   (S, V as MN-major B operands)
+//   MMA 3    : S += K_i^T V_i                     -> TMEM   (fp32 running state, never leaves the SM)
+//   threads  : O -> registers, scale, row normaliser, store; S -> bf16 hi/lo split -> shared
+// The state is fed back to the tensor core as S_hi + S_lo (two bf16 terms, ~16 mantissa bits) so the
+// inter-chunk term keeps fp32-like accuracy; P is rounded to bf16 once.
+// P and O share TMEM columns (P is consumed before O is produced).
+//
+// Every wait is bounded: on a timeout the CTA records CHELA_ERR_TIMEOUT in the status word, drains its
+// outstanding TMA loads (bounded), frees its TMEM and returns.
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace chela {
-bool linattn_sm100_supported(int, int, int, int, int, chela_dtype_t, chela_dtype_t) { return false; }
-size_t linattn_sm100_workspace_bytes(int, int, int, int, int) { return 0; }
-chela_status_t launch_linattn_sm100(const void *, const void *, const void *, void *, int, int, int, int, int,
-                                    chela_dtype_t, chela_dtype_t, int, float, float, void *, cudaStream_t)
+namespace {
+
+constexpr int kD = 64;            // head dimension handled by this kernel (d_k = d_v)
+constexpr int kStages = 2;
+constexpr int kThreads = 128;
+constexpr long long kWaitCycles = 2000000000LL;  // ~1 s at B200 clocks
+
+// ------------------------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
-    return CHELA_ERR_UNSUPPORTED;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within kWaitCycles.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > kWaitCycles) return false;
+    return true;
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem], bf16 operands, fp32 accumulate; issued by a single thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier receives one arrival once all MMAs issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp receives lane (base lane + t).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32])
+{
+    uint32_t *u = reinterpret_cast<uint32_t *>(r);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]),
+          "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]),
+          "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]),
+          "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------- descriptors
+
+// Shared-memory matrix descriptor for a [rows] x 128-byte tile with 128-byte swizzle (tile base
+// 1024-byte aligned).  Bits: [0,14) address >> 4, [16,30) leading byte offset >> 4, [32,46) stride
+// byte offset >> 4 (distance between 8-row groups = 1024 B), [46,48) version = 1, [61,64) layout = 2.
+// The same physical tile serves as a K-major operand (row = M/N index, 128 B along K) or as an
+// MN-major operand (row = K index, 128 B along M/N); the instruction descriptor says which.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulator (bits [4,6) = 1), bf16 A and B (bits [7,10),
+// [10,13) = 1), A/B major (bit 15 / bit 16: 0 = K-major, 1 = MN-major), N >> 3 at [17,23), M >> 4 at [24,29).
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, int b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------- kernel
+
+template <int C>
+struct Smem {
+    static constexpr int kTile = C * 128;                 // one Q/K/V tile, bytes
+    static constexpr int kP = C * C * 2;                  // masked scores, bf16
+    static constexpr int kS = kD * 128;                   // one half (hi or lo) of the state, bf16
+    static constexpr int offQ = 0;
+    static constexpr int offK = offQ + kStages * kTile;
+    static constexpr int offV = offK + kStages * kTile;
+    static constexpr int offP = offV + kStages * kTile;
+    static constexpr int offShi = offP + kP;
+    static constexpr int offSlo = offShi + kS;
+    static constexpr int offBar = offSlo + kS;            // full[kStages], mma
+    static constexpr int offTmem = offBar + 8 * (kStages + 1);
+    static constexpr int bytes = offTmem + 16;
+    static constexpr int tmemCols = (C == 64) ? 128 : 256;
+    static constexpr int colO = 0;                        // O (and P before it): columns [0, C)
+    static constexpr int colS = (C == 64) ? 64 : 128;     // running state: 64 columns
+};
+
+// byte offset of element (row, 16-byte chunk) inside a 128-byte-swizzled [rows] x 128 B tile
+__device__ __forceinline__ uint32_t sw128(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b)
+{
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+
+template <int C, typename TOut>
+__global__ void __launch_bounds__(kThreads)
+linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                     const __grid_constant__ CUtensorMap tm_v, TOut *__restrict__ o, int H, int L, float scale,
+                     int norm, float eps, int *__restrict__ status)
+{
+    using SM = Smem<C>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.x / H, h = blockIdx.x % H;
+    const int nchunks = (L + C - 1) / C;
+
+    const uint32_t bar_full0 = sbase + SM::offBar;
+    const uint32_t bar_mma = sbase + SM::offBar + 8 * kStages;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(bar_full0 + 8 * s, 1);
+        mbar_init(bar_mma, 1);
+        fence_barrier_init();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    if (warp == 0) {
+        tmem_alloc(sbase + SM::offTmem, SM::tmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    auto issue_load = [&](int stage, int chunk) {
+        const uint32_t bar = bar_full0 + 8 * stage;
+        mbar_expect_tx(bar, 3 * SM::kTile);
+        const int t0 = chunk * C;
+        tma_load_4d(sbase + SM::offQ + stage * SM::kTile, &tm_q, bar, 0, h, t0, b);
+        tma_load_4d(sbase + SM::offK + stage * SM::kTile, &tm_k, bar, 0, h, t0, b);
+        tma_load_4d(sbase + SM::offV + stage * SM::kTile, &tm_v, bar, 0, h, t0, b);
+    };
+
+    int loads_issued = 0;
+    if (tid == 0)
+        for (; loads_issued < kStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued, loads_issued);
+
+    // Row of the C x * accumulator tiles (P, O) and of the 64 x 64 state this thread owns.
+    // M = 128 tiles: row = TMEM lane = thread.  M = 64 tiles: row r sits in lane 32*(r/16) + r%16,
+    // so lanes 16..31 of each warp hold nothing.
+    const bool s_active = lane < 16;
+    const int s_row = warp * 16 + lane;
+    const bool o_active = (C == 128) ? true : s_active;
+    const int o_row = (C == 128) ? tid : s_row;
+    const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
+
+    constexpr uint32_t idescP = make_idesc(C, C, 0, 0);
+    constexpr uint32_t idescO = make_idesc(C, kD, 0, 1);
+    constexpr uint32_t idescS = make_idesc(kD, kD, 1, 1);
+
+    uint32_t mma_parity = 0;
+    bool failed = false;
+    int i = 0;
+    for (; i < nchunks; ++i) {
+        const int stage = i % kStages;
+        const uint32_t sQ = sbase + SM::offQ + stage * SM::kTile, sK = sbase + SM::offK + stage * SM::kTile,
+                       sV = sbase + SM::offV + stage * SM::kTile;
+        // ---- MMA 1: P = Q K^T ------------------------------------------------------------------
+        if (tid == 0) {
+            if (mbar_wait(bar_full0 + 8 * stage, (i / kStages) & 1)) {
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < kD / 16; ++k)
+                    umma_bf16(tmem + SM::colO, smem_desc_sw128(sQ + k * 32, 16), smem_desc_sw128(sK + k * 32, 16),
+                              idescP, k > 0);
+                umma_commit(bar_mma);
+            }
+        }
+        bool ok = mbar_wait(bar_mma, mma_parity);
+        mma_parity ^= 1;
+        if (__syncthreads_or(!ok)) { failed = true; break; }
+        tc_fence_after();
+
+        // ---- P: TMEM -> mask -> bf16 -> shared (K-major, [C/64 column halves][C rows][128 B]) --------
+        {
+            uint8_t *sP = smem + SM::offP;
+#pragma unroll
+            for (int cb = 0; cb < C / 32; ++cb) {
+                // rows of this warp are < 32*(warp+1) (C = 128) or < 16*(warp+1) (C = 64):
+                // column blocks entirely above the diagonal are written as zeros without a TMEM read
+                const int warp_max_row = (C == 128) ? warp * 32 + 31 : warp * 16 + 15;
+                float p[32];
+                if (cb * 32 <= warp_max_row) {
+                    tmem_ld32(tmem_warp + SM::colO + cb * 32, p);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) p[j] = 0.f;
+                }
+                if (o_active) {
+                    uint8_t *half = sP + (cb / 2) * (C * 128);
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int col = cb * 32 + c8 * 8 + e * 2;
+                            const float lo = (col <= o_row) ? p[c8 * 8 + e * 2] : 0.f;
+                            const float hi = (col + 1 <= o_row) ? p[c8 * 8 + e * 2 + 1] : 0.f;
+                            w[e] = pack_bf16(lo, hi);
+                        }
+                        *reinterpret_cast<uint4 *>(half + sw128(o_row, (cb % 2) * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+
+        // ---- MMA 2: O = Q S_hi + Q S_lo + P V ;  MMA 3: S += K^T V ---------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+            uint32_t acc = 0;
+            if (i > 0) {
+#pragma unroll
+                for (int part = 0; part < 2; ++part) {
+                    const uint32_t sS = sbase + (part == 0 ? SM::offShi : SM::offSlo);
+#pragma unroll
+                    for (int k = 0; k < kD / 16; ++k) {
+                        umma_bf16(tmem + SM::colO, smem_desc_sw128(sQ + k * 32, 16), smem_desc_sw128(sS + k * 2048, 16),
+                                  idescO, acc);
+                        acc = 1;
+                    }
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < C / 16; ++k) {
+                const uint32_t sP = sbase + SM::offP + (k / 4) * (C * 128) + (k % 4) * 32;
+                umma_bf16(tmem + SM::colO, smem_desc_sw128(sP, 16), smem_desc_sw128(sV + k * 2048, 16), idescO, acc);
+                acc = 1;
+            }
+#pragma unroll
+            for (int k = 0; k < C / 16; ++k)
+                umma_bf16(tmem + SM::colS, smem_desc_sw128(sK + k * 2048, 16), smem_desc_sw128(sV + k * 2048, 16), idescS,
+                          (i > 0 || k > 0) ? 1u : 0u);
+            umma_commit(bar_mma);
+        }
+        ok = mbar_wait(bar_mma, mma_parity);
+        mma_parity ^= 1;
+        if (__syncthreads_or(!ok)) { failed = true; break; }
+        tc_fence_after();
+
+        // the stage is free again: prefetch the chunk that will use it next
+        if (tid == 0 && i + kStages < nchunks) {
+            issue_load(stage, i + kStages);
+            ++loads_issued;
+        }
+
+        // ---- O: TMEM -> scale, normaliser -> global ---------------------------------------------------
+        {
+            float acc[kD];
+            tmem_ld32(tmem_warp + SM::colO, *reinterpret_cast<float(*)[32]>(&acc[0]));
+            tmem_ld32(tmem_warp + SM::colO + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
+            tmem_ld_wait();
+            const int t = i * C + o_row;
+            if (o_active && t < L) {
+                float ss = 0.f;
+#pragma unroll
+                for (int j = 0; j < kD; ++j) {
+                    acc[j] *= scale;
+                    ss = fmaf(acc[j], acc[j], ss);
+                }
+                const float inv = norm ? rsqrtf(ss * (1.0f / kD) + eps) : 1.0f;
+                TOut *dst = o + (((size_t)b * L + t) * H + h) * kD;
+#pragma unroll
+                for (int j = 0; j < kD; j += 4)
+                    store4(dst + j, make_float4(acc[j] * inv, acc[j + 1] * inv, acc[j + 2] * inv, acc[j + 3] * inv));
+            }
+        }
+        // ---- S: TMEM -> bf16 hi + lo -> shared (MN-major B operand of the next chunk) -------------
+        if (i + 1 < nchunks) {
+            float sv[kD];
+            tmem_ld32(tmem_warp + SM::colS, *reinterpret_cast<float(*)[32]>(&sv[0]));
+            tmem_ld32(tmem_warp + SM::colS + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+            tmem_ld_wait();
+            if (s_active) {
+                uint8_t *sHi = smem + SM::offShi, *sLo = smem + SM::offSlo;
+#pragma unroll
+                for (int c8 = 0; c8 < 8; ++c8) {
+                    uint32_t wh[4], wl[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float x0 = sv[c8 * 8 + e * 2], x1 = sv[c8 * 8 + e * 2 + 1];
+                        const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                        const float2 hf = __bfloat1622float2(hh);
+                        wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                        wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                    }
+                    const uint32_t off = sw128(s_row, c8);
+                    *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                    *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+    }
+
+    if (failed) {
+        if (tid == 0) {
+            atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+            // drain loads that were issued but never consumed (bounded), so no copy lands after exit
+            for (int c = i; c < loads_issued; ++c) mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, SM::tmemCols);
+}
+
+// ------------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// [B, L, H, 64] bf16 viewed as a rank-4 tensor (d, H, L, B); box = 64 x 1 x C x 1, 128-byte swizzle.
+// Rows past L are out of bounds for the copy engine and arrive as zeros.
+bool make_qkv_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int C)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)H * kD * 2, (cuuint64_t)L * H * kD * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)kD, 1, (cuuint32_t)C, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int C, typename TOut>
+chela_status_t launch_t(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, void *o, int B, int H,
+                        int L, int norm, float eps, float scale, int *status, cudaStream_t stream)
+{
+    auto kern = linattn_sm100_kernel<C, TOut>;
+    const int smem = Smem<C>::bytes + 1024;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return CHELA_ERR_CUDA;
+    kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, (TOut *)o, H, L, scale, norm, eps, status);
+    return last_launch_status();
+}
+
+}  // namespace
+
+bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_t in_dtype, chela_dtype_t)
+{
+    (void)B; (void)H; (void)L;
+    return in_dtype == CHELA_BF16 && d == kD && (chunk == 64 || chunk == 128);
+}
+
+// 256 bytes: word 0 is the asynchronous status of the last launch that used this workspace.
+size_t linattn_sm100_workspace_bytes(int, int, int, int d, int) { return d == kD ? 256 : 0; }
+
+chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int d,
+                                    int chunk, chela_dtype_t, chela_dtype_t out_dtype, int norm, float eps,
+                                    float scale, void *workspace, cudaStream_t stream)
+{
+    (void)d;
+    CUtensorMap mq, mk, mv;
+    if (!make_qkv_map(&mq, q, B, H, L, chunk) || !make_qkv_map(&mk, k, B, H, L, chunk) ||
+        !make_qkv_map(&mv, v, B, H, L, chunk))
+        return CHELA_ERR_CUDA;
+    int *status = (int *)workspace;
+    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+    if (chunk == 64) {
+        if (out_dtype == CHELA_F32) return launch_t<64, float>(mq, mk, mv, o, B, H, L, norm, eps, scale, status, stream);
+        return launch_t<64, __nv_bfloat16>(mq, mk, mv, o, B, H, L, norm, eps, scale, status, stream);
+    }
+    if (out_dtype == CHELA_F32) return launch_t<128, float>(mq, mk, mv, o, B, H, L, norm, eps, scale, status, stream);
+    return launch_t<128, __nv_bfloat16>(mq, mk, mv, o, B, H, L, norm, eps, scale, status, stream);
+}
+
 }  // namespace chela
