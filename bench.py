@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the CHELA hot path on B200: chunked causal linear attention forward.
+
+One "step" = one chela_linattn_fwd call (through the C ABI) over the sequence-length-sweep workload at
+L = 16384: B*L = 262144 tokens, H = 16, d_k = d_v = 64, chunk 64, bf16 inputs, fp32 accumulate and output.
+Prints ONE JSON line (rank 0) with tokens/s, the roofline fraction of the dominant kernel against the
+measured HBM peak, the end-to-end figure with host buffers, the clock record and the timed CPU oracle.
+Extra keys: "sweep" (every L of the sweep, same launch configuration), "config2" and "mixer".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    torchrun --nproc-per-node N bench.py --gpus N ...      (independent replicas, no collective on the path)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+TOTAL_TOKENS = 262144
+H, D, CHUNK = 16, 64, 64
+L_MAIN = 16384
+SWEEP_L = (1024, 2048, 4096, 8192, 16384, 32768, 65536)
+# algorithmic bytes per token-head: read Q, K, V (bf16) once, write O (fp32) once
+BYTES_PER_TOKEN_HEAD = 3 * D * 2 + D * 4
+METRIC = "linattn_fwd_tokens_per_s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this workload,
+# from the ncu capture summarised under profiles/ (None until a capture exists)
+NCU_TRAFFIC_BYTES = None
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": 1590.0}, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock and throttle reasons through NVML while the benchmark runs."""
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        super().__init__(daemon=True)
+        self.index, self.period, self.samples, self._stop_evt = index, period_s, [], threading.Event()
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        while not self._stop_evt.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)
+                reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                self.samples.append((time.perf_counter(), mhz, reasons))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+
+    def summary(self, t0: float, t1: float):
+        if self.nv is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml_unavailable"], "samples": 0}
+        nv = self.nv
+        window = [s for s in self.samples if t0 <= s[0] <= t1]
+        names = {"sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+                 "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80)}
+        seen = sorted({n for _, _, r in window for n, bit in names.items() if r & bit})
+        return {"sm_mhz": statistics.median([m for _, m, _ in window]) if window else None,
+                "sm_max_mhz": self.max_mhz, "reasons": seen, "samples": len(window)}
+
+
+def time_oracle_sample(n_batches: int, L: int, seed: int = 1234):
+    """Times the float64 oracle (recurrent form, as it stands) on n_batches x L tokens of the workload."""
+    import numpy as np
+    import oracle
+    from paper_2406_08128_b200 import inputs
+    q, k, v = inputs.qkv(seed, n_batches, L, H, D, D, "bf16")
+    q, k, v = (a.astype(np.float64) for a in (q, k, v))
+    t0 = time.perf_counter()
+    oracle.linattn_recurrent(q, k, v)
+    dt = time.perf_counter() - t0
+    return n_batches * L / dt, dt, oracle.num_threads()
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, timed on the host cores, on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    nb = 1
+    times = []
+    for i in range(args.warmup + args.steps):
+        tps, dt, cores = time_oracle_sample(nb, L_MAIN, seed=1234 + i)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = nb * L_MAIN / (ms * 1e-3)
+    sample = "recurrent-form oracle on %d of %d sequences-batches (B=%d, L=%d, H=%d, d=%d) per step" % (
+        nb, TOTAL_TOKENS // L_MAIN, nb, L_MAIN, H, D)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config():
+    return {"workload": "linattn_fwd sweep point L=16384: B=16, H=16, d_k=d_v=64, chunk=64, bf16 in, fp32 out",
+            "B": TOTAL_TOKENS // L_MAIN, "L": L_MAIN, "H": H, "d_k": D, "d_v": D, "chunk": CHUNK,
+            "l2": "inputs+outputs 2.7 GB per step, far larger than L2: no flush needed"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="chela", choices=["chela", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the sweep / config-2 / mixer / CPU-oracle extras")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2406_08128_b200 import build as _build, chela
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    chela.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    B = TOTAL_TOKENS // L_MAIN
+    gen = torch.Generator(device=dev).manual_seed(100 + 14 + rank)
+    flat = [(torch.randn(TOTAL_TOKENS * H * D, device=dev, generator=gen) * 0.125).to(torch.bfloat16) for _ in range(3)]
+    out_flat = torch.empty(TOTAL_TOKENS * H * D, device=dev, dtype=torch.float32)
+    ws = torch.zeros(max(chela.linattn_workspace_bytes(4, H, 65536, D, D, CHUNK),
+                         chela.linattn_workspace_bytes(256, H, 1024, D, D, CHUNK), 256), dtype=torch.uint8, device=dev)
+
+    def views(L):
+        b = TOTAL_TOKENS // L
+        return [t.view(b, L, H, D) for t in flat], out_flat.view(b, L, H, D)
+
+    def step(L):
+        (q, k, v), o = views(L)
+        chela.linattn_fwd(q, k, v, chunk=CHUNK, out_dtype=chela.F32, out=o, workspace=ws)
+
+    kind = chela.linattn_kernel_kind(B, H, L_MAIN, D, D, CHUNK)
+    sampler = ClockSampler(local)
+    sampler.start()
+
+    # ---- timed region: exactly K steps, CUDA events on the launching stream ---------------------------
+    for _ in range(args.warmup):
+        step(L_MAIN)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.perf_counter()
+    ev0.record()
+    for _ in range(args.steps):
+        step(L_MAIN)
+    ev1.record()
+    barrier()
+    t_wall1 = time.perf_counter()
+    ms_total = ev0.elapsed_time(ev1)
+    if chela.async_status(ws) != chela.OK:
+        raise RuntimeError("device-side wait timed out during the timed region")
+    # keep the GPU under the same load a little longer if the timed region was too short to sample clocks
+    clocks = sampler.summary(t_wall0, t_wall1)
+    if clocks["samples"] < 5:
+        t_b0 = time.perf_counter()
+        while time.perf_counter() - t_b0 < 0.5:
+            for _ in range(20):
+                step(L_MAIN)
+            torch.cuda.synchronize()
+        clocks = sampler.summary(t_wall0, time.perf_counter())
+        clocks["note"] = "timed region too short for NVML polling: window extended over an identical untimed burst"
+    t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    value = world * TOTAL_TOKENS / (ms_step * 1e-3)
+
+    # ---- end to end: host buffers in, host buffer out, through the same C-ABI call ---------------------
+    host_in = [torch.empty(x.shape, dtype=x.dtype, pin_memory=True).copy_(x) for x in flat]
+    host_out = torch.empty(out_flat.shape, dtype=out_flat.dtype, pin_memory=True)
+    e2e_steps = max(2, min(args.steps, 5))
+
+    def e2e_step():
+        for d_, h_ in zip(flat, host_in):
+            d_.copy_(h_, non_blocking=True)
+        step(L_MAIN)
+        host_out.copy_(out_flat, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record()
+    barrier()
+    t = torch.tensor([ev0.elapsed_time(ev1)], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item()) / e2e_steps
+    e2e = {"value": world * TOTAL_TOKENS / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+           "steps": e2e_steps, "h2d_bytes_per_step": int(sum(x.numel() * x.element_size() for x in flat)),
+           "d2h_bytes_per_step": int(out_flat.numel() * out_flat.element_size())}
+    del host_in, host_out
+
+    peaks, peak_kind = measured_peaks()
+    alg_bytes = BYTES_PER_TOKEN_HEAD * TOTAL_TOKENS * H
+    achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES, "peak_source": peak_kind,
+                "kernel": "linattn_sm100_kernel<64,float>" if kind == 2 else "linattn_simt_kernel",
+                "algorithmic_bytes_per_launch": alg_bytes, "launch_ms": ms_step}
+
+    line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "kernel_kind": kind, "roofline": roofline}
+
+    def timed(fn, iters, warm=3):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b_.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b_) / iters
+
+    if rank == 0 and not args.no_extras:
+        # ---- every L of the sweep, same kernel and launch path ---------------------------------------
+        sweep = []
+        for L in SWEEP_L:
+            ms = timed(lambda: step(L), 20)
+            sweep.append({"L": L, "B": TOTAL_TOKENS // L, "ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
+                          "hbm_frac": alg_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]})
+        line["sweep"] = sweep
+        # ---- config 2: B=8, H=8, L=4096 (134 MB in + 67 MB out; four rotating buffer sets exceed L2) ----
+        sets = []
+        for s in range(4):
+            n = 8 * 4096 * 8 * 64
+            sets.append(([flat[j][s * n:(s + 1) * n].view(8, 4096, 8, 64) for j in range(3)],
+                         out_flat[s * n:(s + 1) * n].view(8, 4096, 8, 64)))
+        state = {"i": 0}
+
+        def c2():
+            (q, k, v), o = sets[state["i"] % 4]
+            state["i"] += 1
+            chela.linattn_fwd(q, k, v, chunk=64, out_dtype=chela.F32, out=o, workspace=ws)
+
+        ms = timed(c2, 40)
+        c2_bytes = BYTES_PER_TOKEN_HEAD * 8 * 4096 * 8
+        line["config2"] = {"ms": ms, "tokens_per_s": 8 * 4096 / (ms * 1e-3),
+                           "hbm_frac": c2_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        if chela.async_status(ws) != chela.OK:
+            raise RuntimeError("device-side wait timed out in the extras")
+        del sets
+        # ---- CPU oracle on the host cores, bounded sample -----------------------------------------------
+        import oracle
+        oracle.build()
+        time_oracle_sample(1, 2048)  # warm the thread pool
+        tps, dt, cores = time_oracle_sample(2, L_MAIN)
+        line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle", "seconds": dt,
+                                "sample": "recurrent-form float64 oracle on 2 of the 16 sequences-batches "
+                                          "(B=2, L=16384, H=16, d=64) of the same workload"}
+    sampler.stop()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
