@@ -22,7 +22,6 @@ namespace chela {
 namespace {
 
 constexpr int kD = 64;            // head dimension handled by this kernel (d_k = d_v)
-constexpr int kStages = 2;
 constexpr int kThreads = 128;
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s at B200 clocks
 
@@ -86,16 +85,6 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem] * B[smem], bf16 operands, fp32 accumulate; issued by a single thread.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
 // The mbarrier receives one arrival once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
@@ -122,15 +111,16 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 // ------------------------------------------------------------------------------- descriptors
 
 // Shared-memory matrix descriptor for a [rows] x 128-byte tile with 128-byte swizzle (tile base
-// 1024-byte aligned).  Bits: [0,14) address >> 4, [16,30) leading byte offset >> 4, [32,46) stride
-// byte offset >> 4 (distance between 8-row groups = 1024 B), [46,48) version = 1, [61,64) layout = 2.
+// 1024-byte aligned).  Bits: [0,14) address >> 4, [16,30) leading byte offset >> 4 (unused by these
+// single-atom-wide tiles, set to 1), [32,46) stride byte offset >> 4 (distance between 8-row groups =
+// 1024 B), [46,48) version = 1, [61,64) layout = 2 (128-byte swizzle).
 // The same physical tile serves as a K-major operand (row = M/N index, 128 B along K) or as an
 // MN-major operand (row = K index, 128 B along M/N); the instruction descriptor says which.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes)
-{
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           (1ull << 46) | (2ull << 61);
-}
+// Only the low word depends on the address, so the issuing thread keeps the high word constant and
+// advances the low word: +2 per 32 bytes along a K-major row, +128 per 16 rows of an MN-major tile.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (1u << 16); }
+
 // Instruction descriptor, kind::f16: fp32 accumulator (bits [4,6) = 1), bf16 A and B (bits [7,10),
 // [10,13) = 1), A/B major (bit 15 / bit 16: 0 = K-major, 1 = MN-major), N >> 3 at [17,23), M >> 4 at [24,29).
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, int b_mn_major)
@@ -139,25 +129,54 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, 
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// D[tmem] (+)= A[smem] * B[smem], bf16 operands, fp32 accumulate; issued by a single thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+        : "memory");
+}
+
+// TMA store of a shared-memory box to global memory (bulk async-group completion).
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // ------------------------------------------------------------------------------- kernel
 
-template <int C>
+template <int C, typename TOut>
 struct Smem {
+    static constexpr int kStages = (C == 64) ? 3 : 2;
     static constexpr int kTile = C * 128;                 // one Q/K/V tile, bytes
     static constexpr int kP = C * C * 2;                  // masked scores, bf16
     static constexpr int kS = kD * 128;                   // one half (hi or lo) of the state, bf16
+    static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as [C rows] x 128 B boxes
+    static constexpr int kO = kOBoxes * C * 128;
     static constexpr int offQ = 0;
     static constexpr int offK = offQ + kStages * kTile;
     static constexpr int offV = offK + kStages * kTile;
     static constexpr int offP = offV + kStages * kTile;
     static constexpr int offShi = offP + kP;
     static constexpr int offSlo = offShi + kS;
-    static constexpr int offBar = offSlo + kS;            // full[kStages], mma
-    static constexpr int offTmem = offBar + 8 * (kStages + 1);
+    static constexpr int offO = offSlo + kS;
+    static constexpr int offBar = offO + kO;              // full[kStages], barP, barO
+    static constexpr int offTmem = offBar + 8 * (kStages + 2);
     static constexpr int bytes = offTmem + 16;
-    static constexpr int tmemCols = (C == 64) ? 128 : 256;
-    static constexpr int colO = 0;                        // O (and P before it): columns [0, C)
-    static constexpr int colS = (C == 64) ? 64 : 128;     // running state: 64 columns
+    static constexpr int tmemCols = 256;
+    static constexpr int colO = 0;                        // output accumulator: 64 columns
+    static constexpr int colS = 64;                       // running state: 64 columns
+    static constexpr int colP = 128;                      // scores: C columns
 };
 
 // byte offset of element (row, 16-byte chunk) inside a 128-byte-swizzled [rows] x 128 B tile
@@ -169,31 +188,44 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
     return *reinterpret_cast<uint32_t *>(&h);
 }
 
+#ifdef CHELA_TIMING
+#define TMARK(n) do { long long tn = clock64(); tacc[n] += tn - tprev; tprev = tn; } while (0)
+#else
+#define TMARK(n)
+#endif
+
 template <int C, typename TOut>
 __global__ void __launch_bounds__(kThreads)
 linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                     const __grid_constant__ CUtensorMap tm_v, TOut *__restrict__ o, int H, int L, float scale,
-                     int norm, float eps, int *__restrict__ status)
+                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
+                     float scale, int norm, float eps, int *__restrict__ status)
 {
-    using SM = Smem<C>;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    using SM = Smem<C, TOut>;
+    constexpr int kStages = SM::kStages;
+    extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {  // swizzled tiles need a 1024-byte aligned base: report instead of corrupting
+        if (threadIdx.x == 0) atomicExch(status, (int)CHELA_ERR_CUDA);
+        return;
+    }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int b = blockIdx.x / H, h = blockIdx.x % H;
     const int nchunks = (L + C - 1) / C;
 
     const uint32_t bar_full0 = sbase + SM::offBar;
-    const uint32_t bar_mma = sbase + SM::offBar + 8 * kStages;
+    const uint32_t bar_p = sbase + SM::offBar + 8 * kStages;
+    const uint32_t bar_o = bar_p + 8;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) mbar_init(bar_full0 + 8 * s, 1);
-        mbar_init(bar_mma, 1);
+        mbar_init(bar_p, 1);
+        mbar_init(bar_o, 1);
         fence_barrier_init();
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_o);
     }
     if (warp == 0) {
         tmem_alloc(sbase + SM::offTmem, SM::tmemCols);
@@ -204,7 +236,8 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    auto issue_load = [&](int stage, int chunk) {
+    auto issue_load = [&](int chunk) {
+        const int stage = chunk % kStages;
         const uint32_t bar = bar_full0 + 8 * stage;
         mbar_expect_tx(bar, 3 * SM::kTile);
         const int t0 = chunk * C;
@@ -212,10 +245,26 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         tma_load_4d(sbase + SM::offK + stage * SM::kTile, &tm_k, bar, 0, h, t0, b);
         tma_load_4d(sbase + SM::offV + stage * SM::kTile, &tm_v, bar, 0, h, t0, b);
     };
+    constexpr uint32_t idescP = make_idesc(C, C, 0, 0);
+    constexpr uint32_t idescO = make_idesc(C, kD, 0, 1);
+    constexpr uint32_t idescS = make_idesc(kD, kD, 1, 1);
+    // MMA 1 of a chunk: P = Q K^T (both K-major); false if the chunk's tiles never arrived
+    auto issue_scores = [&](int chunk) -> bool {
+        const int stage = chunk % kStages;
+        if (!mbar_wait(bar_full0 + 8 * stage, (chunk / kStages) & 1)) return false;
+        tc_fence_after();
+        const uint32_t q_lo = desc_lo(sbase + SM::offQ + stage * SM::kTile), k_lo = desc_lo(sbase + SM::offK + stage * SM::kTile);
+#pragma unroll
+        for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + SM::colP, q_lo + 2 * k, k_lo + 2 * k, idescP, k > 0);
+        umma_commit(bar_p);
+        return true;
+    };
 
     int loads_issued = 0;
-    if (tid == 0)
-        for (; loads_issued < kStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued, loads_issued);
+    if (tid == 0) {
+        for (; loads_issued < kStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued);
+        issue_scores(0);
+    }
 
     // Row of the C x * accumulator tiles (P, O) and of the 64 x 64 state this thread owns.
     // M = 128 tiles: row = TMEM lane = thread.  M = 64 tiles: row r sits in lane 32*(r/16) + r%16,
@@ -225,60 +274,43 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const bool o_active = (C == 128) ? true : s_active;
     const int o_row = (C == 128) ? tid : s_row;
     const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
+    const int warp_max_row = (C == 128) ? warp * 32 + 31 : warp * 16 + 15;
 
-    constexpr uint32_t idescP = make_idesc(C, C, 0, 0);
-    constexpr uint32_t idescO = make_idesc(C, kD, 0, 1);
-    constexpr uint32_t idescS = make_idesc(kD, kD, 1, 1);
-
-    uint32_t mma_parity = 0;
+    uint32_t par_p = 0, par_o = 0;
     bool failed = false;
     int i = 0;
+#ifdef CHELA_TIMING
+    long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, tprev = clock64();
+#endif
     for (; i < nchunks; ++i) {
         const int stage = i % kStages;
-        const uint32_t sQ = sbase + SM::offQ + stage * SM::kTile, sK = sbase + SM::offK + stage * SM::kTile,
-                       sV = sbase + SM::offV + stage * SM::kTile;
-        // ---- MMA 1: P = Q K^T ------------------------------------------------------------------
-        if (tid == 0) {
-            if (mbar_wait(bar_full0 + 8 * stage, (i / kStages) & 1)) {
-                tc_fence_after();
-#pragma unroll
-                for (int k = 0; k < kD / 16; ++k)
-                    umma_bf16(tmem + SM::colO, smem_desc_sw128(sQ + k * 32, 16), smem_desc_sw128(sK + k * 32, 16),
-                              idescP, k > 0);
-                umma_commit(bar_mma);
-            }
-        }
-        bool ok = mbar_wait(bar_mma, mma_parity);
-        mma_parity ^= 1;
+        // ---- P_i: TMEM -> causal mask -> bf16 -> shared (K-major, [C/64 column halves][C rows][128 B]) ----
+        bool ok = mbar_wait(bar_p, par_p);
+        par_p ^= 1;
         if (__syncthreads_or(!ok)) { failed = true; break; }
         tc_fence_after();
-
-        // ---- P: TMEM -> mask -> bf16 -> shared (K-major, [C/64 column halves][C rows][128 B]) --------
+        TMARK(0);
         {
             uint8_t *sP = smem + SM::offP;
+            // column blocks entirely above the diagonal for every row of this warp are zeros, no TMEM read
+            float p[C / 32][32];
 #pragma unroll
-            for (int cb = 0; cb < C / 32; ++cb) {
-                // rows of this warp are < 32*(warp+1) (C = 128) or < 16*(warp+1) (C = 64):
-                // column blocks entirely above the diagonal are written as zeros without a TMEM read
-                const int warp_max_row = (C == 128) ? warp * 32 + 31 : warp * 16 + 15;
-                float p[32];
-                if (cb * 32 <= warp_max_row) {
-                    tmem_ld32(tmem_warp + SM::colO + cb * 32, p);
-                    tmem_ld_wait();
-                } else {
+            for (int cb = 0; cb < C / 32; ++cb)
+                if (cb * 32 <= warp_max_row) tmem_ld32(tmem_warp + SM::colP + cb * 32, p[cb]);
+            tmem_ld_wait();
+            if (o_active) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) p[j] = 0.f;
-                }
-                if (o_active) {
+                for (int cb = 0; cb < C / 32; ++cb) {
                     uint8_t *half = sP + (cb / 2) * (C * 128);
+                    const bool live = cb * 32 <= warp_max_row;
 #pragma unroll
                     for (int c8 = 0; c8 < 4; ++c8) {
                         uint32_t w[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int col = cb * 32 + c8 * 8 + e * 2;
-                            const float lo = (col <= o_row) ? p[c8 * 8 + e * 2] : 0.f;
-                            const float hi = (col + 1 <= o_row) ? p[c8 * 8 + e * 2 + 1] : 0.f;
+                            const float lo = (live && col <= o_row) ? p[cb][c8 * 8 + e * 2] : 0.f;
+                            const float hi = (live && col + 1 <= o_row) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
                             w[e] = pack_bf16(lo, hi);
                         }
                         *reinterpret_cast<uint4 *>(half + sw128(o_row, (cb % 2) * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -289,54 +321,61 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
+        TMARK(1);
 
-        // ---- MMA 2: O = Q S_hi + Q S_lo + P V ;  MMA 3: S += K^T V ---------------------------------
+        // ---- MMA 2: O = Q S_hi + Q S_lo + P V ;  MMA 3: S += K^T V ;  then MMA 1 of the next chunk ----
         if (tid == 0) {
             tc_fence_after();
+            const uint32_t q_lo = desc_lo(sbase + SM::offQ + stage * SM::kTile), k_lo = desc_lo(sbase + SM::offK + stage * SM::kTile),
+                           v_lo = desc_lo(sbase + SM::offV + stage * SM::kTile), p_lo = desc_lo(sbase + SM::offP),
+                           shi_lo = desc_lo(sbase + SM::offShi), slo_lo = desc_lo(sbase + SM::offSlo);
             uint32_t acc = 0;
             if (i > 0) {
 #pragma unroll
-                for (int part = 0; part < 2; ++part) {
-                    const uint32_t sS = sbase + (part == 0 ? SM::offShi : SM::offSlo);
-#pragma unroll
-                    for (int k = 0; k < kD / 16; ++k) {
-                        umma_bf16(tmem + SM::colO, smem_desc_sw128(sQ + k * 32, 16), smem_desc_sw128(sS + k * 2048, 16),
-                                  idescO, acc);
-                        acc = 1;
-                    }
+                for (int k = 0; k < kD / 16; ++k) {
+                    umma_bf16(tmem + SM::colO, q_lo + 2 * k, shi_lo + 128 * k, idescO, acc);
+                    acc = 1;
                 }
+#pragma unroll
+                for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + SM::colO, q_lo + 2 * k, slo_lo + 128 * k, idescO, 1);
             }
 #pragma unroll
             for (int k = 0; k < C / 16; ++k) {
-                const uint32_t sP = sbase + SM::offP + (k / 4) * (C * 128) + (k % 4) * 32;
-                umma_bf16(tmem + SM::colO, smem_desc_sw128(sP, 16), smem_desc_sw128(sV + k * 2048, 16), idescO, acc);
+                umma_bf16(tmem + SM::colO, p_lo + (k / 4) * (C * 128 / 16) + 2 * (k % 4), v_lo + 128 * k, idescO, acc);
                 acc = 1;
             }
 #pragma unroll
             for (int k = 0; k < C / 16; ++k)
-                umma_bf16(tmem + SM::colS, smem_desc_sw128(sK + k * 2048, 16), smem_desc_sw128(sV + k * 2048, 16), idescS,
-                          (i > 0 || k > 0) ? 1u : 0u);
-            umma_commit(bar_mma);
+                umma_bf16(tmem + SM::colS, k_lo + 128 * k, v_lo + 128 * k, idescS, (i > 0 || k > 0) ? 1u : 0u);
+            umma_commit(bar_o);
+            if (i + 1 < nchunks) issue_scores(i + 1);
         }
-        ok = mbar_wait(bar_mma, mma_parity);
-        mma_parity ^= 1;
+        TMARK(2);
+        ok = mbar_wait(bar_o, par_o);
+        par_o ^= 1;
+        if (tid == 0) bulk_wait_read0();   // the previous chunk's output box has left shared memory
         if (__syncthreads_or(!ok)) { failed = true; break; }
         tc_fence_after();
+        TMARK(3);
 
         // the stage is free again: prefetch the chunk that will use it next
         if (tid == 0 && i + kStages < nchunks) {
-            issue_load(stage, i + kStages);
+            issue_load(i + kStages);
             ++loads_issued;
         }
 
-        // ---- O: TMEM -> scale, normaliser -> global ---------------------------------------------------
+        // ---- O_i: TMEM -> scale, normaliser -> shared staging ;  S_i: TMEM -> bf16 hi + lo -> shared ----
         {
-            float acc[kD];
+            float acc[kD], sv[kD];
             tmem_ld32(tmem_warp + SM::colO, *reinterpret_cast<float(*)[32]>(&acc[0]));
             tmem_ld32(tmem_warp + SM::colO + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
+            const bool need_s = i + 1 < nchunks;
+            if (need_s) {
+                tmem_ld32(tmem_warp + SM::colS, *reinterpret_cast<float(*)[32]>(&sv[0]));
+                tmem_ld32(tmem_warp + SM::colS + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+            }
             tmem_ld_wait();
-            const int t = i * C + o_row;
-            if (o_active && t < L) {
+            if (o_active) {
                 float ss = 0.f;
 #pragma unroll
                 for (int j = 0; j < kD; ++j) {
@@ -344,19 +383,22 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     ss = fmaf(acc[j], acc[j], ss);
                 }
                 const float inv = norm ? rsqrtf(ss * (1.0f / kD) + eps) : 1.0f;
-                TOut *dst = o + (((size_t)b * L + t) * H + h) * kD;
+                uint8_t *sO = smem + SM::offO;
+                if (sizeof(TOut) == 4) {
 #pragma unroll
-                for (int j = 0; j < kD; j += 4)
-                    store4(dst + j, make_float4(acc[j] * inv, acc[j + 1] * inv, acc[j + 2] * inv, acc[j + 3] * inv));
+                    for (int j = 0; j < kD; j += 4)
+                        *reinterpret_cast<float4 *>(sO + (j / 32) * (C * 128) + sw128(o_row, (j % 32) / 4)) =
+                            make_float4(acc[j] * inv, acc[j + 1] * inv, acc[j + 2] * inv, acc[j + 3] * inv);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kD; j += 8)
+                        *reinterpret_cast<uint4 *>(sO + sw128(o_row, j / 8)) =
+                            make_uint4(pack_bf16(acc[j] * inv, acc[j + 1] * inv), pack_bf16(acc[j + 2] * inv, acc[j + 3] * inv),
+                                       pack_bf16(acc[j + 4] * inv, acc[j + 5] * inv), pack_bf16(acc[j + 6] * inv, acc[j + 7] * inv));
+                }
             }
-        }
-        // ---- S: TMEM -> bf16 hi + lo -> shared (MN-major B operand of the next chunk) -------------
-        if (i + 1 < nchunks) {
-            float sv[kD];
-            tmem_ld32(tmem_warp + SM::colS, *reinterpret_cast<float(*)[32]>(&sv[0]));
-            tmem_ld32(tmem_warp + SM::colS + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
-            tmem_ld_wait();
-            if (s_active) {
+            TMARK(4);
+            if (need_s && s_active) {
                 uint8_t *sHi = smem + SM::offShi, *sLo = smem + SM::offSlo;
 #pragma unroll
                 for (int c8 = 0; c8 < 8; ++c8) {
@@ -378,10 +420,23 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
-    }
-
-    if (failed) {
+        // rows past L are clipped by the copy engine
         if (tid == 0) {
+#pragma unroll
+            for (int bx = 0; bx < SM::kOBoxes; ++bx)
+                tma_store_4d(&tm_o, sbase + SM::offO + bx * (C * 128), bx * (128 / (int)sizeof(TOut)), h, i * C, b);
+            bulk_commit();
+        }
+        TMARK(5);
+    }
+#ifdef CHELA_TIMING
+    if (tid == 0 && blockIdx.x == 0)
+        for (int n = 0; n < 8; ++n) reinterpret_cast<long long *>(status)[4 + n] = tacc[n];
+#endif
+
+    if (tid == 0) {
+        bulk_wait0();
+        if (failed) {
             atomicExch(status, (int)CHELA_ERR_TIMEOUT);
             // drain loads that were issued but never consumed (bounded), so no copy lands after exit
             for (int c = i; c < loads_issued; ++c) mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1);
@@ -411,30 +466,36 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// [B, L, H, 64] bf16 viewed as a rank-4 tensor (d, H, L, B); box = 64 x 1 x C x 1, 128-byte swizzle.
-// Rows past L are out of bounds for the copy engine and arrive as zeros.
-bool make_qkv_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int C)
+// [B, L, H, 64] viewed as a rank-4 tensor (d, H, L, B); box = (128 bytes of d) x 1 x C x 1, 128-byte
+// swizzle.  Loads: rows past L are out of bounds for the copy engine and arrive as zeros.  Stores: rows
+// past L are clipped.
+bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int C, bool f32)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
+    const cuuint64_t es = f32 ? 4 : 2;
     const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)H * kD * 2, (cuuint64_t)L * H * kD * 2};
-    const cuuint32_t box[4] = {(cuuint32_t)kD, 1, (cuuint32_t)C, 1};
+    const cuuint64_t strides[3] = {(cuuint64_t)kD * es, (cuuint64_t)H * kD * es, (cuuint64_t)L * H * kD * es};
+    const cuuint32_t box[4] = {(cuuint32_t)(128 / es), 1, (cuuint32_t)C, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr),
+              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int C, typename TOut>
-chela_status_t launch_t(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, void *o, int B, int H,
-                        int L, int norm, float eps, float scale, int *status, cudaStream_t stream)
+chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
+                        float scale, int *status, cudaStream_t stream)
 {
+    CUtensorMap mq, mk, mv, mo;
+    if (!make_map(&mq, q, B, H, L, C, false) || !make_map(&mk, k, B, H, L, C, false) ||
+        !make_map(&mv, v, B, H, L, C, false) || !make_map(&mo, o, B, H, L, C, sizeof(TOut) == 4))
+        return CHELA_ERR_CUDA;
     auto kern = linattn_sm100_kernel<C, TOut>;
-    const int smem = Smem<C>::bytes + 1024;
+    const int smem = Smem<C, TOut>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return CHELA_ERR_CUDA;
-    kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, (TOut *)o, H, L, scale, norm, eps, status);
+    kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status);
     return last_launch_status();
 }
 
@@ -454,18 +515,14 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
                                     float scale, void *workspace, cudaStream_t stream)
 {
     (void)d;
-    CUtensorMap mq, mk, mv;
-    if (!make_qkv_map(&mq, q, B, H, L, chunk) || !make_qkv_map(&mk, k, B, H, L, chunk) ||
-        !make_qkv_map(&mv, v, B, H, L, chunk))
-        return CHELA_ERR_CUDA;
     int *status = (int *)workspace;
     if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
     if (chunk == 64) {
-        if (out_dtype == CHELA_F32) return launch_t<64, float>(mq, mk, mv, o, B, H, L, norm, eps, scale, status, stream);
-        return launch_t<64, __nv_bfloat16>(mq, mk, mv, o, B, H, L, norm, eps, scale, status, stream);
+        if (out_dtype == CHELA_F32) return launch_t<64, float>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+        return launch_t<64, __nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
     }
-    if (out_dtype == CHELA_F32) return launch_t<128, float>(mq, mk, mv, o, B, H, L, norm, eps, scale, status, stream);
-    return launch_t<128, __nv_bfloat16>(mq, mk, mv, o, B, H, L, norm, eps, scale, status, stream);
+    if (out_dtype == CHELA_F32) return launch_t<128, float>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+    return launch_t<128, __nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
 }
 
 }  // namespace chela
