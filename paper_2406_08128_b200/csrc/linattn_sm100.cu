@@ -1,16 +1,20 @@
 // Chunked causal linear attention for bf16 inputs on sm_100a: tcgen05 tensor-core tiles with TMEM
 // accumulators, operands staged by TMA (Sec. 4.1 tiling of Eq. 2 with the causal mask).
 //
-// One CTA (128 threads) walks one (batch, head) sequence chunk by chunk.  Per chunk of C tokens:
-//   TMA      : Q_i, K_i, V_i tiles ([C rows] x 128 B, 128-byte swizzle) into a 2-stage ring
-//   MMA 1    : P = Q_i K_i^T                      -> TMEM   (both operands K-major)
-//   threads  : P -> registers, causal mask, bf16  -> shared (K-major tile for the next MMA)
-//   MMA 2    : O = Q_i S_hi + Q_i S_lo + P V_i    -> TMEM   (S, V as MN-major B operands)
-//   MMA 3    : S += K_i^T V_i                     -> TMEM   (fp32 running state, never leaves the SM)
-//   threads  : O -> registers, scale, row normaliser, store; S -> bf16 hi/lo split -> shared
+// One CTA (128 threads) walks one (batch, head) sequence in tiles of 64 tokens.  The tensor core
+// charges a tcgen05.mma by the instruction (about 46 cycles for any N <= 93 and any M <= 128), so the
+// five 64 x 64 x 64 products of a tile are packed into M = 128 instructions:
+//   TMA     : Q_i, K_i, V_i ([64 rows] x 128 B, 128-byte swizzle, adjacent in one stage of a 3-stage ring)
+//   G1      : [Q_i ; K_i] Q_i^T                       -> TMEM tile PT; rows 64..127 are P^T = K_i Q_i^T
+//   warps 2,3: P^T -> registers, causal mask (t >= s), bf16 -> shared tile (rows = s)
+//   G2      : rows 0..63 of tile OS = Q_i S_hi + Q_i S_lo (A = [Q_i ; K_i], lanes 64..127 write-disabled)
+//   G3      : OS += [P^T tile | K_i tile]^T V_i          rows 0..63 += P V_i (output), rows 64..127 += K_i^T V_i
+//             (one MN-major A operand of two 64-wide atoms: the score tile and, through the descriptor's
+//              leading-dimension offset, the K tile of the current stage)
+//   warps 0,1: output rows -> scale, row normaliser -> swizzled staging -> TMA store
+//   warps 2,3: state rows (fp32, never leave the SM) -> bf16 hi + lo -> shared (B operand of the next G2)
 // The state is fed back to the tensor core as S_hi + S_lo (two bf16 terms, ~16 mantissa bits) so the
 // inter-chunk term keeps fp32-like accuracy; P is rounded to bf16 once.
-// P and O share TMEM columns (P is consumed before O is produced).
 //
 // Every wait is bounded: on a timeout the CTA records CHELA_ERR_TIMEOUT in the status word, drains its
 // outstanding TMA loads (bounded), frees its TMEM and returns.
@@ -110,16 +114,20 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 // ------------------------------------------------------------------------------- descriptors
 
-// Shared-memory matrix descriptor for a [rows] x 128-byte tile with 128-byte swizzle (tile base
-// 1024-byte aligned).  Bits: [0,14) address >> 4, [16,30) leading byte offset >> 4 (unused by these
-// single-atom-wide tiles, set to 1), [32,46) stride byte offset >> 4 (distance between 8-row groups =
-// 1024 B), [46,48) version = 1, [61,64) layout = 2 (128-byte swizzle).
-// The same physical tile serves as a K-major operand (row = M/N index, 128 B along K) or as an
-// MN-major operand (row = K index, 128 B along M/N); the instruction descriptor says which.
-// Only the low word depends on the address, so the issuing thread keeps the high word constant and
+// Shared-memory matrix descriptor for [rows] x 128-byte tiles with 128-byte swizzle (tile bases
+// 1024-byte aligned).  Bits: [0,14) address >> 4, [16,30) leading byte offset >> 4, [32,46) stride byte
+// offset >> 4 (distance between 8-row groups = 1024 B), [46,48) version = 1, [61,64) layout = 2
+// (128-byte swizzle).  The same physical tile serves as a K-major operand (row = M/N index, 128 B along
+// K) or as an MN-major operand (row = K index, 128 B along M/N); the instruction descriptor says which.
+// For an MN-major operand wider than 64 elements the leading byte offset is the distance from one
+// 64-element atom to the next; K-major operands here never use it.
+// Only the low word depends on addresses, so the issuing thread keeps the high word constant and
 // advances the low word: +2 per 32 bytes along a K-major row, +128 per 16 rows of an MN-major tile.
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint32_t desc_lo(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes = 16)
+{
+    return ((addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
 
 // Instruction descriptor, kind::f16: fp32 accumulator (bits [4,6) = 1), bf16 A and B (bits [7,10),
 // [10,13) = 1), A/B major (bit 15 / bit 16: 0 = K-major, 1 = MN-major), N >> 3 at [17,23), M >> 4 at [24,29).
@@ -130,15 +138,18 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, 
 }
 
 // D[tmem] (+)= A[smem] * B[smem], bf16 operands, fp32 accumulate; issued by a single thread.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate)
+// upper_off != 0 write-disables TMEM lanes 64..127 (rows 64..127 of an M = 128 result).
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate,
+                                          uint32_t upper_off = 0)
 {
+    const uint32_t m = upper_off ? 0xFFFFFFFFu : 0u;
     asm volatile(
         "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "mov.b64 da, {%1, %5};\n\t"
         "mov.b64 db, {%2, %5};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, {%6, %6, %7, %7}, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi), "r"(0u), "r"(m)
         : "memory");
 }
 
@@ -155,29 +166,25 @@ __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_
 
 // ------------------------------------------------------------------------------- kernel
 
-template <int C, typename TOut>
+constexpr int kC = 64;       // tokens per tile
+constexpr int kStages = 3;
+constexpr int kTile = kC * 128;   // one 64-row x 128-byte tile
+
+template <typename TOut>
 struct Smem {
-    static constexpr int kStages = (C == 64) ? 3 : 2;
-    static constexpr int kTile = C * 128;                 // one Q/K/V tile, bytes
-    static constexpr int kP = C * C * 2;                  // masked scores, bf16
-    static constexpr int kS = kD * 128;                   // one half (hi or lo) of the state, bf16
-    static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as [C rows] x 128 B boxes
-    static constexpr int kO = kOBoxes * C * 128;
-    static constexpr int offQ = 0;
-    static constexpr int offK = offQ + kStages * kTile;
-    static constexpr int offV = offK + kStages * kTile;
-    static constexpr int offP = offV + kStages * kTile;
-    static constexpr int offShi = offP + kP;
-    static constexpr int offSlo = offShi + kS;
-    static constexpr int offO = offSlo + kS;
-    static constexpr int offBar = offO + kO;              // full[kStages], barP, barO
+    static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as 64-row x 128 B boxes
+    static constexpr int offPT = 0;                       // masked scores, transposed: rows = s, 64 t per row
+    static constexpr int offShi = offPT + kTile;          // state, bf16 high part: rows = d_k
+    static constexpr int offSlo = offShi + kTile;         // state, bf16 low part
+    static constexpr int offO = offSlo + kTile;           // output staging
+    static constexpr int offStage = offO + kOBoxes * kTile;   // per stage: Q, K, V tiles, adjacent
+    static constexpr int offBar = offStage + kStages * 3 * kTile;   // full[kStages], barP, barO
     static constexpr int offTmem = offBar + 8 * (kStages + 2);
     static constexpr int bytes = offTmem + 16;
-    static constexpr int tmemCols = 256;
-    static constexpr int colO = 0;                        // output accumulator: 64 columns
-    static constexpr int colS = 64;                       // running state: 64 columns
-    static constexpr int colP = 128;                      // scores: C columns
 };
+constexpr int kTmemCols = 128;
+constexpr int kColOS = 0;    // rows 0..63: output tile, rows 64..127: running state; 64 columns
+constexpr int kColPT = 64;   // rows 64..127: transposed scores; 64 columns
 
 // byte offset of element (row, 16-byte chunk) inside a 128-byte-swizzled [rows] x 128 B tile
 __device__ __forceinline__ uint32_t sw128(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
@@ -194,23 +201,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 #define TMARK(n)
 #endif
 
-template <int C, typename TOut>
+template <typename TOut>
 __global__ void __launch_bounds__(kThreads)
 linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
                      float scale, int norm, float eps, int *__restrict__ status)
 {
-    using SM = Smem<C, TOut>;
-    constexpr int kStages = SM::kStages;
+    using SM = Smem<TOut>;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     if (sbase & 1023u) {  // swizzled tiles need a 1024-byte aligned base: report instead of corrupting
         if (threadIdx.x == 0) atomicExch(status, (int)CHELA_ERR_CUDA);
         return;
     }
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, warp = tid >> 5;
     const int b = blockIdx.x / H, h = blockIdx.x % H;
-    const int nchunks = (L + C - 1) / C;
+    const int nchunks = (L + kC - 1) / kC;
 
     const uint32_t bar_full0 = sbase + SM::offBar;
     const uint32_t bar_p = sbase + SM::offBar + 8 * kStages;
@@ -228,7 +234,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         tma_prefetch_desc(&tm_o);
     }
     if (warp == 0) {
-        tmem_alloc(sbase + SM::offTmem, SM::tmemCols);
+        tmem_alloc(sbase + SM::offTmem, kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -236,28 +242,35 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
+    auto stage_base = [&](int chunk) { return sbase + SM::offStage + (chunk % kStages) * 3 * kTile; };
     auto issue_load = [&](int chunk) {
-        const int stage = chunk % kStages;
-        const uint32_t bar = bar_full0 + 8 * stage;
-        mbar_expect_tx(bar, 3 * SM::kTile);
-        const int t0 = chunk * C;
-        tma_load_4d(sbase + SM::offQ + stage * SM::kTile, &tm_q, bar, 0, h, t0, b);
-        tma_load_4d(sbase + SM::offK + stage * SM::kTile, &tm_k, bar, 0, h, t0, b);
-        tma_load_4d(sbase + SM::offV + stage * SM::kTile, &tm_v, bar, 0, h, t0, b);
+        const uint32_t bar = bar_full0 + 8 * (chunk % kStages), dst = stage_base(chunk);
+        mbar_expect_tx(bar, 3 * kTile);
+        tma_load_4d(dst, &tm_q, bar, 0, h, chunk * kC, b);
+        tma_load_4d(dst + kTile, &tm_k, bar, 0, h, chunk * kC, b);
+        tma_load_4d(dst + 2 * kTile, &tm_v, bar, 0, h, chunk * kC, b);
     };
-    constexpr uint32_t idescP = make_idesc(C, C, 0, 0);
-    constexpr uint32_t idescO = make_idesc(C, kD, 0, 1);
-    constexpr uint32_t idescS = make_idesc(kD, kD, 1, 1);
-    // MMA 1 of a chunk: P = Q K^T (both K-major); false if the chunk's tiles never arrived
+    constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [Q;K] (K-major) x Q^T (K-major)
+    constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;K] (K-major) x S (MN-major)
+    constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
+    // G1 of a chunk; false if the chunk's tiles never arrived
     auto issue_scores = [&](int chunk) -> bool {
-        const int stage = chunk % kStages;
-        if (!mbar_wait(bar_full0 + 8 * stage, (chunk / kStages) & 1)) return false;
+        if (!mbar_wait(bar_full0 + 8 * (chunk % kStages), (chunk / kStages) & 1)) return false;
         tc_fence_after();
-        const uint32_t q_lo = desc_lo(sbase + SM::offQ + stage * SM::kTile), k_lo = desc_lo(sbase + SM::offK + stage * SM::kTile);
+        const uint32_t qk_lo = desc_lo(stage_base(chunk));
 #pragma unroll
-        for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + SM::colP, q_lo + 2 * k, k_lo + 2 * k, idescP, k > 0);
+        for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk_lo + 2 * k, qk_lo + 2 * k, idescG1, k > 0);
         umma_commit(bar_p);
         return true;
+    };
+    // G2 of a chunk: rows 0..63 of OS = Q S_hi + Q S_lo (the stage's tiles have arrived: G1 ran before)
+    auto issue_inter = [&](int chunk) {
+        const uint32_t qk_lo = desc_lo(stage_base(chunk)), shi_lo = desc_lo(sbase + SM::offShi),
+                       slo_lo = desc_lo(sbase + SM::offSlo);
+#pragma unroll
+        for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, shi_lo + 128 * k, idescG2, k > 0, 1);
+#pragma unroll
+        for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, slo_lo + 128 * k, idescG2, 1, 1);
     };
 
     int loads_issued = 0;
@@ -266,15 +279,11 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         issue_scores(0);
     }
 
-    // Row of the C x * accumulator tiles (P, O) and of the 64 x 64 state this thread owns.
-    // M = 128 tiles: row = TMEM lane = thread.  M = 64 tiles: row r sits in lane 32*(r/16) + r%16,
-    // so lanes 16..31 of each warp hold nothing.
-    const bool s_active = lane < 16;
-    const int s_row = warp * 16 + lane;
-    const bool o_active = (C == 128) ? true : s_active;
-    const int o_row = (C == 128) ? tid : s_row;
+    // TMEM lane = accumulator row = thread.  Warps 0,1 own output rows t = tid; warps 2,3 own row
+    // r = tid - 64 of the transposed scores (s) and of the state (d_k).
+    const bool upper = warp >= 2;
+    const int r = tid & 63;
     const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
-    const int warp_max_row = (C == 128) ? warp * 32 + 31 : warp * 16 + 15;
 
     uint32_t par_p = 0, par_o = 0;
     bool failed = false;
@@ -283,38 +292,33 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, tprev = clock64();
 #endif
     for (; i < nchunks; ++i) {
-        const int stage = i % kStages;
-        // ---- P_i: TMEM -> causal mask -> bf16 -> shared (K-major, [C/64 column halves][C rows][128 B]) ----
+        // ---- P^T_i: TMEM -> causal mask -> bf16 -> shared (rows = s, 64 t per row) ---------------------
         bool ok = mbar_wait(bar_p, par_p);
         par_p ^= 1;
         if (__syncthreads_or(!ok)) { failed = true; break; }
         tc_fence_after();
         TMARK(0);
-        {
-            uint8_t *sP = smem + SM::offP;
-            // column blocks entirely above the diagonal for every row of this warp are zeros, no TMEM read
-            float p[C / 32][32];
-#pragma unroll
-            for (int cb = 0; cb < C / 32; ++cb)
-                if (cb * 32 <= warp_max_row) tmem_ld32(tmem_warp + SM::colP + cb * 32, p[cb]);
+        if (upper) {
+            // row s keeps t >= s; for warp 3 (s >= 32) the block t < 32 is all zeros: no TMEM read
+            float p[2][32];
+            if (warp == 2) tmem_ld32(tmem_warp + kColPT, p[0]);
+            tmem_ld32(tmem_warp + kColPT + 32, p[1]);
             tmem_ld_wait();
-            if (o_active) {
+            uint8_t *sP = smem + SM::offPT;
 #pragma unroll
-                for (int cb = 0; cb < C / 32; ++cb) {
-                    uint8_t *half = sP + (cb / 2) * (C * 128);
-                    const bool live = cb * 32 <= warp_max_row;
+            for (int cb = 0; cb < 2; ++cb) {
+                const bool live = cb == 1 || warp == 2;
 #pragma unroll
-                    for (int c8 = 0; c8 < 4; ++c8) {
-                        uint32_t w[4];
+                for (int c8 = 0; c8 < 4; ++c8) {
+                    uint32_t w[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int col = cb * 32 + c8 * 8 + e * 2;
-                            const float lo = (live && col <= o_row) ? p[cb][c8 * 8 + e * 2] : 0.f;
-                            const float hi = (live && col + 1 <= o_row) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
-                            w[e] = pack_bf16(lo, hi);
-                        }
-                        *reinterpret_cast<uint4 *>(half + sw128(o_row, (cb % 2) * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    for (int e = 0; e < 4; ++e) {
+                        const int t = cb * 32 + c8 * 8 + e * 2;
+                        const float lo = (live && t >= r) ? p[cb][c8 * 8 + e * 2] : 0.f;
+                        const float hi = (live && t + 1 >= r) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
+                        w[e] = pack_bf16(lo, hi);
                     }
+                    *reinterpret_cast<uint4 *>(sP + sw128(r, cb * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
         }
@@ -323,30 +327,15 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         __syncthreads();
         TMARK(1);
 
-        // ---- MMA 2: O = Q S_hi + Q S_lo + P V ;  MMA 3: S += K^T V ;  then MMA 1 of the next chunk ----
+        // ---- G2 (inter-chunk term), G3 (intra-chunk term and state update), then G1 of the next chunk ----
         if (tid == 0) {
             tc_fence_after();
-            const uint32_t q_lo = desc_lo(sbase + SM::offQ + stage * SM::kTile), k_lo = desc_lo(sbase + SM::offK + stage * SM::kTile),
-                           v_lo = desc_lo(sbase + SM::offV + stage * SM::kTile), p_lo = desc_lo(sbase + SM::offP),
-                           shi_lo = desc_lo(sbase + SM::offShi), slo_lo = desc_lo(sbase + SM::offSlo);
-            uint32_t acc = 0;
-            if (i > 0) {
+            if (i > 0) issue_inter(i);
+            const uint32_t st = stage_base(i);
+            // A: atom 0 = score tile, atom 1 = K tile of this stage (leading byte offset = their distance)
+            const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st + 2 * kTile);
 #pragma unroll
-                for (int k = 0; k < kD / 16; ++k) {
-                    umma_bf16(tmem + SM::colO, q_lo + 2 * k, shi_lo + 128 * k, idescO, acc);
-                    acc = 1;
-                }
-#pragma unroll
-                for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + SM::colO, q_lo + 2 * k, slo_lo + 128 * k, idescO, 1);
-            }
-#pragma unroll
-            for (int k = 0; k < C / 16; ++k) {
-                umma_bf16(tmem + SM::colO, p_lo + (k / 4) * (C * 128 / 16) + 2 * (k % 4), v_lo + 128 * k, idescO, acc);
-                acc = 1;
-            }
-#pragma unroll
-            for (int k = 0; k < C / 16; ++k)
-                umma_bf16(tmem + SM::colS, k_lo + 128 * k, v_lo + 128 * k, idescS, (i > 0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS, a_lo + 128 * k, v_lo + 128 * k, idescG3, (i > 0 || k > 0) ? 1u : 0u);
             umma_commit(bar_o);
             if (i + 1 < nchunks) issue_scores(i + 1);
         }
@@ -364,18 +353,16 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             ++loads_issued;
         }
 
-        // ---- O_i: TMEM -> scale, normaliser -> shared staging ;  S_i: TMEM -> bf16 hi + lo -> shared ----
         {
-            float acc[kD], sv[kD];
-            tmem_ld32(tmem_warp + SM::colO, *reinterpret_cast<float(*)[32]>(&acc[0]));
-            tmem_ld32(tmem_warp + SM::colO + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
-            const bool need_s = i + 1 < nchunks;
-            if (need_s) {
-                tmem_ld32(tmem_warp + SM::colS, *reinterpret_cast<float(*)[32]>(&sv[0]));
-                tmem_ld32(tmem_warp + SM::colS + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+            float acc[kD];
+            const bool need = !upper || i + 1 < nchunks;
+            if (need) {
+                tmem_ld32(tmem_warp + kColOS, *reinterpret_cast<float(*)[32]>(&acc[0]));
+                tmem_ld32(tmem_warp + kColOS + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
+                tmem_ld_wait();
             }
-            tmem_ld_wait();
-            if (o_active) {
+            if (!upper) {
+                // ---- output row t: scale, normaliser -> swizzled staging boxes ----------------------------
                 float ss = 0.f;
 #pragma unroll
                 for (int j = 0; j < kD; ++j) {
@@ -387,31 +374,30 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (sizeof(TOut) == 4) {
 #pragma unroll
                     for (int j = 0; j < kD; j += 4)
-                        *reinterpret_cast<float4 *>(sO + (j / 32) * (C * 128) + sw128(o_row, (j % 32) / 4)) =
+                        *reinterpret_cast<float4 *>(sO + (j / 32) * kTile + sw128(r, (j % 32) / 4)) =
                             make_float4(acc[j] * inv, acc[j + 1] * inv, acc[j + 2] * inv, acc[j + 3] * inv);
                 } else {
 #pragma unroll
                     for (int j = 0; j < kD; j += 8)
-                        *reinterpret_cast<uint4 *>(sO + sw128(o_row, j / 8)) =
+                        *reinterpret_cast<uint4 *>(sO + sw128(r, j / 8)) =
                             make_uint4(pack_bf16(acc[j] * inv, acc[j + 1] * inv), pack_bf16(acc[j + 2] * inv, acc[j + 3] * inv),
                                        pack_bf16(acc[j + 4] * inv, acc[j + 5] * inv), pack_bf16(acc[j + 6] * inv, acc[j + 7] * inv));
                 }
-            }
-            TMARK(4);
-            if (need_s && s_active) {
+            } else if (need) {
+                // ---- state row d_k: bf16 hi + lo -> shared (MN-major B operand of the next chunk's G2) ------
                 uint8_t *sHi = smem + SM::offShi, *sLo = smem + SM::offSlo;
 #pragma unroll
                 for (int c8 = 0; c8 < 8; ++c8) {
                     uint32_t wh[4], wl[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const float x0 = sv[c8 * 8 + e * 2], x1 = sv[c8 * 8 + e * 2 + 1];
+                        const float x0 = acc[c8 * 8 + e * 2], x1 = acc[c8 * 8 + e * 2 + 1];
                         const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
                         const float2 hf = __bfloat1622float2(hh);
                         wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
                         wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
                     }
-                    const uint32_t off = sw128(s_row, c8);
+                    const uint32_t off = sw128(r, c8);
                     *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
                     *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
                 }
@@ -424,10 +410,10 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         if (tid == 0) {
 #pragma unroll
             for (int bx = 0; bx < SM::kOBoxes; ++bx)
-                tma_store_4d(&tm_o, sbase + SM::offO + bx * (C * 128), bx * (128 / (int)sizeof(TOut)), h, i * C, b);
+                tma_store_4d(&tm_o, sbase + SM::offO + bx * kTile, bx * (128 / (int)sizeof(TOut)), h, i * kC, b);
             bulk_commit();
         }
-        TMARK(5);
+        TMARK(4);
     }
 #ifdef CHELA_TIMING
     if (tid == 0 && blockIdx.x == 0)
@@ -444,7 +430,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, SM::tmemCols);
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------- host side
@@ -483,16 +469,16 @@ bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int C, boo
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int C, typename TOut>
+template <typename TOut>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
                         float scale, int *status, cudaStream_t stream)
 {
     CUtensorMap mq, mk, mv, mo;
-    if (!make_map(&mq, q, B, H, L, C, false) || !make_map(&mk, k, B, H, L, C, false) ||
-        !make_map(&mv, v, B, H, L, C, false) || !make_map(&mo, o, B, H, L, C, sizeof(TOut) == 4))
+    if (!make_map(&mq, q, B, H, L, kC, false) || !make_map(&mk, k, B, H, L, kC, false) ||
+        !make_map(&mv, v, B, H, L, kC, false) || !make_map(&mo, o, B, H, L, kC, sizeof(TOut) == 4))
         return CHELA_ERR_CUDA;
-    auto kern = linattn_sm100_kernel<C, TOut>;
-    const int smem = Smem<C, TOut>::bytes;
+    auto kern = linattn_sm100_kernel<TOut>;
+    const int smem = Smem<TOut>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return CHELA_ERR_CUDA;
     kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status);
@@ -517,12 +503,10 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
     (void)d;
     int *status = (int *)workspace;
     if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
-    if (chunk == 64) {
-        if (out_dtype == CHELA_F32) return launch_t<64, float>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
-        return launch_t<64, __nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
-    }
-    if (out_dtype == CHELA_F32) return launch_t<128, float>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
-    return launch_t<128, __nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+    // The result does not depend on the chunk size: both supported values run on 64-token tiles.
+    (void)chunk;
+    if (out_dtype == CHELA_F32) return launch_t<float>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+    return launch_t<__nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
 }
 
 }  // namespace chela
