@@ -1,7 +1,9 @@
 // Chunked causal linear attention for bf16 inputs on sm_100a: tcgen05 tensor-core tiles with TMEM
 // accumulators, operands staged by TMA (Sec. 4.1 tiling of Eq. 2 with the causal mask).
 //
-// One CTA (128 threads) walks one (batch, head) sequence in tiles of 64 tokens.  The tensor core
+// One CTA walks one (batch, head) sequence in tiles of 64 tokens: four compute warps plus one issuer
+// warp whose lane 0 drives TMA and the tensor core (its own warp, so that its instruction stream is
+// not interleaved with spinning lanes); roles meet only through mbarriers, every wait bounded.  The tensor core
 // charges a tcgen05.mma by the instruction (about 46 cycles for any N <= 93 and any M <= 128), so the
 // five 64 x 64 x 64 products of a tile are packed into M = 128 instructions:
 //   TMA     : Q_i, K_i, V_i ([64 rows] x 128 B, 128-byte swizzle, adjacent in one stage of a 3-stage ring)
@@ -26,7 +28,7 @@ namespace chela {
 namespace {
 
 constexpr int kD = 64;            // head dimension handled by this kernel (d_k = d_v)
-constexpr int kThreads = 128;
+constexpr int kThreads = 160;            // 4 compute warps + 1 issuer warp
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s at B200 clocks
 
 // ------------------------------------------------------------------------------- PTX wrappers
@@ -53,14 +55,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kWaitCycles.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Bounded wait: false if the phase did not complete within kWaitCycles, or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity))
-        if (clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > kWaitCycles || (abort_flag && *abort_flag)) return false;
     return true;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -172,15 +178,16 @@ constexpr int kTile = kC * 128;   // one 64-row x 128-byte tile
 
 template <typename TOut>
 struct Smem {
-    static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as 64-row x 128 B boxes
+    static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as 128-byte wide boxes
     static constexpr int offPT = 0;                       // masked scores, transposed: rows = s, 64 t per row
     static constexpr int offShi = offPT + kTile;          // state, bf16 high part: rows = d_k
     static constexpr int offSlo = offShi + kTile;         // state, bf16 low part
     static constexpr int offO = offSlo + kTile;           // output staging
     static constexpr int offStage = offO + kOBoxes * kTile;   // per stage: Q, K, V tiles, adjacent
-    static constexpr int offBar = offStage + kStages * 3 * kTile;   // full[kStages], barP, barO
-    static constexpr int offTmem = offBar + 8 * (kStages + 2);
-    static constexpr int bytes = offTmem + 16;
+    static constexpr int offBar = offStage + kStages * 3 * kTile;   // full[kStages], p, o, pt, s
+    static constexpr int offTmem = offBar + 8 * (kStages + 4);
+    static constexpr int offAbort = offTmem + 8;
+    static constexpr int bytes = offAbort + 8;
 };
 constexpr int kTmemCols = 128;
 constexpr int kColOS = 0;    // rows 0..63: output tile, rows 64..127: running state; 64 columns
@@ -197,8 +204,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 
 #ifdef CHELA_TIMING
 #define TMARK(n) do { long long tn = clock64(); tacc[n] += tn - tprev; tprev = tn; } while (0)
+#define TDECL long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, tprev = clock64()
+#define TDUMP(slot) do { for (int n_ = 0; n_ < 8; ++n_) reinterpret_cast<long long *>(status)[4 + 8 * (slot) + n_] = tacc[n_]; } while (0)
 #else
 #define TMARK(n)
+#define TDECL
+#define TDUMP(slot)
 #endif
 
 template <typename TOut>
@@ -214,19 +225,25 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         if (threadIdx.x == 0) atomicExch(status, (int)CHELA_ERR_CUDA);
         return;
     }
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int b = blockIdx.x / H, h = blockIdx.x % H;
     const int nchunks = (L + kC - 1) / kC;
 
     const uint32_t bar_full0 = sbase + SM::offBar;
-    const uint32_t bar_p = sbase + SM::offBar + 8 * kStages;
-    const uint32_t bar_o = bar_p + 8;
+    const uint32_t bar_p = bar_full0 + 8 * kStages;   // G1 of a chunk has completed (tensor core -> warps 2,3)
+    const uint32_t bar_o = bar_p + 8;                 // G2 + G3 of a chunk have completed (-> all roles)
+    const uint32_t bar_pt = bar_o + 8;                // score tile of a chunk is in shared memory (warps 2,3 -> issuer)
+    const uint32_t bar_s = bar_pt + 8;                // output/state rows read, state tiles written (4 warps -> issuer)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) mbar_init(bar_full0 + 8 * s, 1);
         mbar_init(bar_p, 1);
         mbar_init(bar_o, 1);
+        mbar_init(bar_pt, 2);
+        mbar_init(bar_s, 4);
+        *abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
@@ -242,127 +259,148 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    auto stage_base = [&](int chunk) { return sbase + SM::offStage + (chunk % kStages) * 3 * kTile; };
-    auto issue_load = [&](int chunk) {
-        const uint32_t bar = bar_full0 + 8 * (chunk % kStages), dst = stage_base(chunk);
-        mbar_expect_tx(bar, 3 * kTile);
-        tma_load_4d(dst, &tm_q, bar, 0, h, chunk * kC, b);
-        tma_load_4d(dst + kTile, &tm_k, bar, 0, h, chunk * kC, b);
-        tma_load_4d(dst + 2 * kTile, &tm_v, bar, 0, h, chunk * kC, b);
-    };
-    constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [Q;K] (K-major) x Q^T (K-major)
-    constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;K] (K-major) x S (MN-major)
-    constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
-    // G1 of a chunk; false if the chunk's tiles never arrived
-    auto issue_scores = [&](int chunk) -> bool {
-        if (!mbar_wait(bar_full0 + 8 * (chunk % kStages), (chunk / kStages) & 1)) return false;
-        tc_fence_after();
-        const uint32_t qk_lo = desc_lo(stage_base(chunk));
+    if (warp == 4) {
+        // =========================================== issuer: TMA loads and every tcgen05.mma ==========
+        if (lane == 0) {
+            TDECL;
+            auto stage_base = [&](int chunk) { return sbase + SM::offStage + (chunk % kStages) * 3 * kTile; };
+            auto issue_load = [&](int chunk) {
+                const uint32_t bar = bar_full0 + 8 * (chunk % kStages), dst = stage_base(chunk);
+                mbar_expect_tx(bar, 3 * kTile);
+                tma_load_4d(dst, &tm_q, bar, 0, h, chunk * kC, b);
+                tma_load_4d(dst + kTile, &tm_k, bar, 0, h, chunk * kC, b);
+                tma_load_4d(dst + 2 * kTile, &tm_v, bar, 0, h, chunk * kC, b);
+            };
+            constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [Q;K] (K-major) x Q^T (K-major)
+            constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;K] (K-major) x S (MN-major)
+            constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
+            // G1 of a chunk; false if the chunk's tiles never arrived
+            auto issue_scores = [&](int chunk) -> bool {
+                if (!mbar_wait(bar_full0 + 8 * (chunk % kStages), (chunk / kStages) & 1, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t qk_lo = desc_lo(stage_base(chunk));
 #pragma unroll
-        for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk_lo + 2 * k, qk_lo + 2 * k, idescG1, k > 0);
-        umma_commit(bar_p);
-        return true;
-    };
-    // G2 of a chunk: rows 0..63 of OS = Q S_hi + Q S_lo (the stage's tiles have arrived: G1 ran before)
-    auto issue_inter = [&](int chunk) {
-        const uint32_t qk_lo = desc_lo(stage_base(chunk)), shi_lo = desc_lo(sbase + SM::offShi),
-                       slo_lo = desc_lo(sbase + SM::offSlo);
+                for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk_lo + 2 * k, qk_lo + 2 * k, idescG1, k > 0);
+                umma_commit(bar_p);
+                return true;
+            };
+            const uint32_t shi_lo = desc_lo(sbase + SM::offShi), slo_lo = desc_lo(sbase + SM::offSlo);
+            int loads_issued = 0, consumed = 0;
+            for (; loads_issued < kStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued);
+            bool ok = issue_scores(0);
+            for (int i = 0; ok && i < nchunks; ++i) {
+                const uint32_t st = stage_base(i);
+                if (i > 0) {
+                    // G2: rows 0..63 of OS = Q S_hi + Q S_lo; needs the state tiles of chunk i-1 and its
+                    // output rows out of TMEM
+                    ok = mbar_wait(bar_s, (i - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    TMARK(0);
+                    const uint32_t qk_lo = desc_lo(st);
 #pragma unroll
-        for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, shi_lo + 128 * k, idescG2, k > 0, 1);
+                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, shi_lo + 128 * k, idescG2, k > 0, 1);
 #pragma unroll
-        for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, slo_lo + 128 * k, idescG2, 1, 1);
-    };
-
-    int loads_issued = 0;
-    if (tid == 0) {
-        for (; loads_issued < kStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued);
-        issue_scores(0);
-    }
-
-    // TMEM lane = accumulator row = thread.  Warps 0,1 own output rows t = tid; warps 2,3 own row
-    // r = tid - 64 of the transposed scores (s) and of the state (d_k).
-    const bool upper = warp >= 2;
-    const int r = tid & 63;
-    const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
-
-    uint32_t par_p = 0, par_o = 0;
-    bool failed = false;
-    int i = 0;
-#ifdef CHELA_TIMING
-    long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, tprev = clock64();
-#endif
-    for (; i < nchunks; ++i) {
-        // ---- P^T_i: TMEM -> causal mask -> bf16 -> shared (rows = s, 64 t per row) ---------------------
-        bool ok = mbar_wait(bar_p, par_p);
-        par_p ^= 1;
-        if (__syncthreads_or(!ok)) { failed = true; break; }
-        tc_fence_after();
-        TMARK(0);
-        if (upper) {
-            // row s keeps t >= s; for warp 3 (s >= 32) the block t < 32 is all zeros: no TMEM read
-            float p[2][32];
-            if (warp == 2) tmem_ld32(tmem_warp + kColPT, p[0]);
-            tmem_ld32(tmem_warp + kColPT + 32, p[1]);
-            tmem_ld_wait();
-            uint8_t *sP = smem + SM::offPT;
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                const bool live = cb == 1 || warp == 2;
-#pragma unroll
-                for (int c8 = 0; c8 < 4; ++c8) {
-                    uint32_t w[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int t = cb * 32 + c8 * 8 + e * 2;
-                        const float lo = (live && t >= r) ? p[cb][c8 * 8 + e * 2] : 0.f;
-                        const float hi = (live && t + 1 >= r) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
-                        w[e] = pack_bf16(lo, hi);
-                    }
-                    *reinterpret_cast<uint4 *>(sP + sw128(r, cb * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, slo_lo + 128 * k, idescG2, 1, 1);
+                    TMARK(1);
                 }
-            }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        TMARK(1);
-
-        // ---- G2 (inter-chunk term), G3 (intra-chunk term and state update), then G1 of the next chunk ----
-        if (tid == 0) {
-            tc_fence_after();
-            if (i > 0) issue_inter(i);
-            const uint32_t st = stage_base(i);
-            // A: atom 0 = score tile, atom 1 = K tile of this stage (leading byte offset = their distance)
-            const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st + 2 * kTile);
+                // G3: OS += [P^T | K]^T V; atom 0 = score tile, atom 1 = K tile of this stage
+                ok = mbar_wait(bar_pt, i & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                TMARK(2);
+                const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st + 2 * kTile);
 #pragma unroll
-            for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS, a_lo + 128 * k, v_lo + 128 * k, idescG3, (i > 0 || k > 0) ? 1u : 0u);
-            umma_commit(bar_o);
-            if (i + 1 < nchunks) issue_scores(i + 1);
+                for (int k = 0; k < kC / 16; ++k)
+                    umma_bf16(tmem + kColOS, a_lo + 128 * k, v_lo + 128 * k, idescG3, (i > 0 || k > 0) ? 1u : 0u);
+                umma_commit(bar_o);
+                if (i + 1 < nchunks) {
+                    ok = issue_scores(i + 1);
+                    if (!ok) break;
+                }
+                TMARK(3);
+                // the stage is free once G3 has completed: prefetch the chunk that will use it next
+                ok = mbar_wait(bar_o, i & 1, abort_flag);
+                if (!ok) break;
+                consumed = i + 1;
+                if (i + kStages < nchunks) {
+                    issue_load(i + kStages);
+                    ++loads_issued;
+                }
+                TMARK(4);
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+                // drain loads that were issued but never consumed (bounded), so no copy lands after exit
+                for (int c = consumed; c < loads_issued; ++c)
+                    mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1, nullptr);
+            }
+#ifdef CHELA_TIMING
+            if (blockIdx.x == 0) TDUMP(0);
+#endif
         }
-        TMARK(2);
-        ok = mbar_wait(bar_o, par_o);
-        par_o ^= 1;
-        if (tid == 0) bulk_wait_read0();   // the previous chunk's output box has left shared memory
-        if (__syncthreads_or(!ok)) { failed = true; break; }
-        tc_fence_after();
-        TMARK(3);
-
-        // the stage is free again: prefetch the chunk that will use it next
-        if (tid == 0 && i + kStages < nchunks) {
-            issue_load(i + kStages);
-            ++loads_issued;
-        }
-
-        {
+    } else {
+        // =========================================== compute warps ====================================
+        // TMEM lane = accumulator row = thread.  Warps 0,1 own output rows t = tid; warps 2,3 own row
+        // r = tid - 64 of the transposed scores (s) and of the state (d_k).
+        const bool upper = warp >= 2;
+        const int r = tid & 63;
+        const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
+        bool ok = true;
+        TDECL;
+        for (int i = 0; i < nchunks; ++i) {
+            if (upper) {
+                // ---- P^T_i: TMEM -> causal mask -> bf16 -> shared (rows = s, 64 t per row) -------------
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_p, i & 1, abort_flag));
+                if (!ok) break;
+                tc_fence_after();
+                TMARK(0);
+                // row s keeps t >= s; for warp 3 (s >= 32) the block t < 32 is all zeros: no TMEM read
+                float p[2][32];
+                if (warp == 2) tmem_ld32(tmem_warp + kColPT, p[0]);
+                tmem_ld32(tmem_warp + kColPT + 32, p[1]);
+                tmem_ld_wait();
+                uint8_t *sP = smem + SM::offPT;
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    const bool live = cb == 1 || warp == 2;
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int t = cb * 32 + c8 * 8 + e * 2;
+                            const float lo = (live && t >= r) ? p[cb][c8 * 8 + e * 2] : 0.f;
+                            const float hi = (live && t + 1 >= r) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
+                            w[e] = pack_bf16(lo, hi);
+                        }
+                        *reinterpret_cast<uint4 *>(sP + sw128(r, cb * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_pt);
+                TMARK(1);
+            }
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            TMARK(2);
             float acc[kD];
-            const bool need = !upper || i + 1 < nchunks;
-            if (need) {
+            if (!upper) {
+                // ---- output row t: scale, normaliser -> swizzled staging -> TMA store (per warp: 32 rows) ----
                 tmem_ld32(tmem_warp + kColOS, *reinterpret_cast<float(*)[32]>(&acc[0]));
                 tmem_ld32(tmem_warp + kColOS + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
                 tmem_ld_wait();
-            }
-            if (!upper) {
-                // ---- output row t: scale, normaliser -> swizzled staging boxes ----------------------------
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar_s);     // the output rows are out of TMEM: G2 of the next chunk may overwrite them
+                    bulk_wait_read0();      // this warp's previous output boxes have left shared memory
+                }
+                __syncwarp();
                 float ss = 0.f;
 #pragma unroll
                 for (int j = 0; j < kD; ++j) {
@@ -383,50 +421,55 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             make_uint4(pack_bf16(acc[j] * inv, acc[j + 1] * inv), pack_bf16(acc[j + 2] * inv, acc[j + 3] * inv),
                                        pack_bf16(acc[j + 4] * inv, acc[j + 5] * inv), pack_bf16(acc[j + 6] * inv, acc[j + 7] * inv));
                 }
-            } else if (need) {
-                // ---- state row d_k: bf16 hi + lo -> shared (MN-major B operand of the next chunk's G2) ------
-                uint8_t *sHi = smem + SM::offShi, *sLo = smem + SM::offSlo;
+                fence_proxy_async();
+                __syncwarp();
+                // rows past L are clipped by the copy engine
+                if (lane == 0) {
 #pragma unroll
-                for (int c8 = 0; c8 < 8; ++c8) {
-                    uint32_t wh[4], wl[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float x0 = acc[c8 * 8 + e * 2], x1 = acc[c8 * 8 + e * 2 + 1];
-                        const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
-                        const float2 hf = __bfloat1622float2(hh);
-                        wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
-                        wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
-                    }
-                    const uint32_t off = sw128(r, c8);
-                    *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
-                    *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                    for (int bx = 0; bx < SM::kOBoxes; ++bx)
+                        tma_store_4d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
+                                     i * kC + warp * 32, b);
+                    bulk_commit();
                 }
+                TMARK(3);
+            } else {
+                // ---- state row d_k: bf16 hi + lo -> shared (MN-major B operand of the next chunk's G2) ------
+                if (i + 1 < nchunks) {
+                    tmem_ld32(tmem_warp + kColOS, *reinterpret_cast<float(*)[32]>(&acc[0]));
+                    tmem_ld32(tmem_warp + kColOS + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
+                    tmem_ld_wait();
+                    uint8_t *sHi = smem + SM::offShi, *sLo = smem + SM::offSlo;
+#pragma unroll
+                    for (int c8 = 0; c8 < 8; ++c8) {
+                        uint32_t wh[4], wl[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float x0 = acc[c8 * 8 + e * 2], x1 = acc[c8 * 8 + e * 2 + 1];
+                            const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                            const float2 hf = __bfloat1622float2(hh);
+                            wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                            wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                        }
+                        const uint32_t off = sw128(r, c8);
+                        *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                        *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                    }
+                    fence_proxy_async();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_s);
+                }
+                TMARK(3);
             }
         }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        // rows past L are clipped by the copy engine
-        if (tid == 0) {
-#pragma unroll
-            for (int bx = 0; bx < SM::kOBoxes; ++bx)
-                tma_store_4d(&tm_o, sbase + SM::offO + bx * kTile, bx * (128 / (int)sizeof(TOut)), h, i * kC, b);
-            bulk_commit();
-        }
-        TMARK(4);
-    }
-#ifdef CHELA_TIMING
-    if (tid == 0 && blockIdx.x == 0)
-        for (int n = 0; n < 8; ++n) reinterpret_cast<long long *>(status)[4 + n] = tacc[n];
-#endif
-
-    if (tid == 0) {
-        bulk_wait0();
-        if (failed) {
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
             atomicExch(status, (int)CHELA_ERR_TIMEOUT);
-            // drain loads that were issued but never consumed (bounded), so no copy lands after exit
-            for (int c = i; c < loads_issued; ++c) mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1);
         }
+        if (!upper && lane == 0) bulk_wait0();   // output boxes fully written before the CTA retires
+#ifdef CHELA_TIMING
+        if (blockIdx.x == 0 && (tid == 0 || tid == 64)) TDUMP(tid == 0 ? 1 : 2);
+#endif
     }
     tc_fence_before();
     __syncthreads();
@@ -475,7 +518,7 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
 {
     CUtensorMap mq, mk, mv, mo;
     if (!make_map(&mq, q, B, H, L, kC, false) || !make_map(&mk, k, B, H, L, kC, false) ||
-        !make_map(&mv, v, B, H, L, kC, false) || !make_map(&mo, o, B, H, L, kC, sizeof(TOut) == 4))
+        !make_map(&mv, v, B, H, L, kC, false) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4))
         return CHELA_ERR_CUDA;
     auto kern = linattn_sm100_kernel<TOut>;
     const int smem = Smem<TOut>::bytes;
@@ -494,7 +537,7 @@ bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_
 }
 
 // 256 bytes: word 0 is the asynchronous status of the last launch that used this workspace.
-size_t linattn_sm100_workspace_bytes(int, int, int, int d, int) { return d == kD ? 256 : 0; }
+size_t linattn_sm100_workspace_bytes(int, int, int, int d, int) { return d == kD ? 512 : 0; }
 
 chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int d,
                                     int chunk, chela_dtype_t, chela_dtype_t out_dtype, int norm, float eps,
