@@ -116,6 +116,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32])
         : "r"(taddr)
         : "memory");
 }
+// Store counterpart: thread t of the warp writes 32 consecutive fp32 columns of lane (base lane + t).
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&r)[32])
+{
+    const uint32_t *u = reinterpret_cast<const uint32_t *>(r);
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7]),
+          "r"(u[8]), "r"(u[9]), "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15]),
+          "r"(u[16]), "r"(u[17]), "r"(u[18]), "r"(u[19]), "r"(u[20]), "r"(u[21]), "r"(u[22]), "r"(u[23]),
+          "r"(u[24]), "r"(u[25]), "r"(u[26]), "r"(u[27]), "r"(u[28]), "r"(u[29]), "r"(u[30]), "r"(u[31]),
+          "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------- descriptors
@@ -216,8 +232,11 @@ template <typename TOut>
 __global__ void __launch_bounds__(kThreads)
 linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
-                     float scale, int norm, float eps, int *__restrict__ status)
+                     float scale, int norm, float eps, int *__restrict__ status, const float *__restrict__ s_part,
+                     int G, int cpg)
 {
+    // Grid: one CTA per (batch*head, group).  Group g covers chunks [g*cpg, (g+1)*cpg) of its sequence and
+    // starts from the state sum_{g' < g} s_part[bh][g'] (per-group K^T V sums written by the state kernel).
     using SM = Smem<TOut>;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -226,8 +245,11 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         return;
     }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int b = blockIdx.x / H, h = blockIdx.x % H;
-    const int nchunks = (L + kC - 1) / kC;
+    const int bh = blockIdx.x / G, g = blockIdx.x % G;
+    const int b = bh / H, h = bh % H;
+    const int c0 = g * cpg;                                        // first chunk of this group
+    const int nchunks = min(cpg, (L + kC - 1) / kC - c0);          // chunks of this group
+    const bool has_init = g > 0;
 
     const uint32_t bar_full0 = sbase + SM::offBar;
     const uint32_t bar_p = bar_full0 + 8 * kStages;   // G1 of a chunk has completed (tensor core -> warps 2,3)
@@ -267,9 +289,9 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             auto issue_load = [&](int chunk) {
                 const uint32_t bar = bar_full0 + 8 * (chunk % kStages), dst = stage_base(chunk);
                 mbar_expect_tx(bar, 3 * kTile);
-                tma_load_4d(dst, &tm_q, bar, 0, h, chunk * kC, b);
-                tma_load_4d(dst + kTile, &tm_k, bar, 0, h, chunk * kC, b);
-                tma_load_4d(dst + 2 * kTile, &tm_v, bar, 0, h, chunk * kC, b);
+                tma_load_4d(dst, &tm_q, bar, 0, h, (c0 + chunk) * kC, b);
+                tma_load_4d(dst + kTile, &tm_k, bar, 0, h, (c0 + chunk) * kC, b);
+                tma_load_4d(dst + 2 * kTile, &tm_v, bar, 0, h, (c0 + chunk) * kC, b);
             };
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [Q;K] (K-major) x Q^T (K-major)
             constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;K] (K-major) x S (MN-major)
@@ -288,12 +310,14 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             int loads_issued = 0, consumed = 0;
             for (; loads_issued < kStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued);
             bool ok = issue_scores(0);
+            uint32_t par_s = 0;
             for (int i = 0; ok && i < nchunks; ++i) {
                 const uint32_t st = stage_base(i);
-                if (i > 0) {
-                    // G2: rows 0..63 of OS = Q S_hi + Q S_lo; needs the state tiles of chunk i-1 and its
-                    // output rows out of TMEM
-                    ok = mbar_wait(bar_s, (i - 1) & 1, abort_flag);
+                if (i > 0 || has_init) {
+                    // G2: rows 0..63 of OS = Q S_hi + Q S_lo; needs the state tiles of the previous chunk (or
+                    // of the group's initial state) and the previous output rows out of TMEM
+                    ok = mbar_wait(bar_s, par_s, abort_flag);
+                    par_s ^= 1;
                     if (!ok) break;
                     tc_fence_after();
                     TMARK(0);
@@ -312,7 +336,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st + 2 * kTile);
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k)
-                    umma_bf16(tmem + kColOS, a_lo + 128 * k, v_lo + 128 * k, idescG3, (i > 0 || k > 0) ? 1u : 0u);
+                    umma_bf16(tmem + kColOS, a_lo + 128 * k, v_lo + 128 * k, idescG3, (i > 0 || has_init || k > 0) ? 1u : 0u);
                 umma_commit(bar_o);
                 if (i + 1 < nchunks) {
                     ok = issue_scores(i + 1);
@@ -349,6 +373,50 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
         bool ok = true;
         TDECL;
+        // state row r -> bf16 hi + lo -> shared (MN-major B operand of G2)
+        auto write_state_tiles = [&](const float(&sv)[kD]) {
+            uint8_t *sHi = smem + SM::offShi, *sLo = smem + SM::offSlo;
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) {
+                uint32_t wh[4], wl[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float x0 = sv[c8 * 8 + e * 2], x1 = sv[c8 * 8 + e * 2 + 1];
+                    const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                    const float2 hf = __bfloat1622float2(hh);
+                    wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                    wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                }
+                const uint32_t off = sw128(r, c8);
+                *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+            }
+        };
+        if (has_init) {
+            // initial state of the group: sum of the preceding groups' K^T V, into TMEM rows 64..127 and
+            // into the G2 operand tiles
+            if (upper) {
+                float sv[kD];
+#pragma unroll
+                for (int j = 0; j < kD; ++j) sv[j] = 0.f;
+                for (int gp = 0; gp < g; ++gp) {
+                    const float4 *src = reinterpret_cast<const float4 *>(s_part + (((size_t)bh * (G - 1) + gp) * kD + r) * kD);
+#pragma unroll
+                    for (int j = 0; j < kD / 4; ++j) {
+                        const float4 x = src[j];
+                        sv[4 * j] += x.x; sv[4 * j + 1] += x.y; sv[4 * j + 2] += x.z; sv[4 * j + 3] += x.w;
+                    }
+                }
+                tmem_st32(tmem_warp + kColOS, *reinterpret_cast<const float(*)[32]>(&sv[0]));
+                tmem_st32(tmem_warp + kColOS + 32, *reinterpret_cast<const float(*)[32]>(&sv[32]));
+                tmem_st_wait();
+                write_state_tiles(sv);
+                fence_proxy_async();
+                tc_fence_before();
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_s);
+        }
         for (int i = 0; i < nchunks; ++i) {
             if (upper) {
                 // ---- P^T_i: TMEM -> causal mask -> bf16 -> shared (rows = s, 64 t per row) -------------
@@ -428,7 +496,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
                     for (int bx = 0; bx < SM::kOBoxes; ++bx)
                         tma_store_4d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
-                                     i * kC + warp * 32, b);
+                                     (c0 + i) * kC + warp * 32, b);
                     bulk_commit();
                 }
                 TMARK(3);
@@ -438,22 +506,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     tmem_ld32(tmem_warp + kColOS, *reinterpret_cast<float(*)[32]>(&acc[0]));
                     tmem_ld32(tmem_warp + kColOS + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
                     tmem_ld_wait();
-                    uint8_t *sHi = smem + SM::offShi, *sLo = smem + SM::offSlo;
-#pragma unroll
-                    for (int c8 = 0; c8 < 8; ++c8) {
-                        uint32_t wh[4], wl[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float x0 = acc[c8 * 8 + e * 2], x1 = acc[c8 * 8 + e * 2 + 1];
-                            const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
-                            const float2 hf = __bfloat1622float2(hh);
-                            wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
-                            wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
-                        }
-                        const uint32_t off = sw128(r, c8);
-                        *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
-                        *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-                    }
+                    write_state_tiles(acc);
                     fence_proxy_async();
                     tc_fence_before();
                     __syncwarp();
@@ -474,6 +527,121 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// ------------------------------------------------------------------------------- state kernel
+
+// Per-group state sums for sequences that are split along L: CTA (batch*head, g), g < G-1, writes
+// s_part[bh][g] = sum over the group's chunks of K_i^T V_i (fp32, [d_k][d_v]).  Only K and V are read.
+// One tcgen05.mma group per chunk: A = [K_i | V_i] (MN-major, two atoms), B = V_i; rows 0..63 of the
+// accumulator are K^T V, rows 64..127 (V^T V) are ignored.
+constexpr int kStStages = 4;
+struct SmemState {
+    static constexpr int offStage = 0;                              // per stage: K, V tiles, adjacent
+    static constexpr int offBar = kStStages * 2 * kTile;            // full[kStStages], empty[kStStages], done
+    static constexpr int offTmem = offBar + 8 * (2 * kStStages + 1);
+    static constexpr int offAbort = offTmem + 8;
+    static constexpr int bytes = offAbort + 8;
+};
+
+__global__ void __launch_bounds__(kThreads)
+linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                     float *__restrict__ s_part, int H, int G, int cpg, int *__restrict__ status)
+{
+    using SM = SmemState;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {
+        if (threadIdx.x == 0) atomicExch(status, (int)CHELA_ERR_CUDA);
+        return;
+    }
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.x / (G - 1), g = blockIdx.x % (G - 1);
+    const int b = bh / H, h = bh % H;
+    const int c0 = g * cpg, nchunks = cpg;    // every group but the last is full
+
+    const uint32_t bar_full0 = sbase + SM::offBar, bar_empty0 = bar_full0 + 8 * kStStages,
+                   bar_done = bar_empty0 + 8 * kStStages;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
+    if (tid == 0) {
+        for (int s = 0; s < kStStages; ++s) {
+            mbar_init(bar_full0 + 8 * s, 1);
+            mbar_init(bar_empty0 + 8 * s, 1);
+        }
+        mbar_init(bar_done, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    if (warp == 0) {
+        tmem_alloc(sbase + SM::offTmem, 64);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            auto issue_load = [&](int chunk) {
+                const uint32_t bar = bar_full0 + 8 * (chunk % kStStages), dst = sbase + SM::offStage + (chunk % kStStages) * 2 * kTile;
+                mbar_expect_tx(bar, 2 * kTile);
+                tma_load_4d(dst, &tm_k, bar, 0, h, (c0 + chunk) * kC, b);
+                tma_load_4d(dst + kTile, &tm_v, bar, 0, h, (c0 + chunk) * kC, b);
+            };
+            constexpr uint32_t idesc = make_idesc(128, kD, 1, 1);
+            int loads_issued = 0, consumed = 0;
+            for (; loads_issued < kStStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued);
+            bool ok = true;
+            for (int i = 0; i < nchunks; ++i) {
+                const int stage = i % kStStages;
+                ok = mbar_wait(bar_full0 + 8 * stage, (i / kStStages) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t st = sbase + SM::offStage + stage * 2 * kTile;
+                const uint32_t a_lo = desc_lo(st, kTile), v_lo = desc_lo(st + kTile);
+#pragma unroll
+                for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem, a_lo + 128 * k, v_lo + 128 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                umma_commit(bar_empty0 + 8 * stage);
+                consumed = i + 1;
+                if (i + kStStages < nchunks) {
+                    ok = mbar_wait(bar_empty0 + 8 * stage, (i / kStStages) & 1, abort_flag);
+                    if (!ok) break;
+                    issue_load(i + kStStages);
+                    ++loads_issued;
+                }
+            }
+            if (ok) umma_commit(bar_done);
+            else {
+                *abort_flag = 1;
+                atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+                for (int c = consumed; c < loads_issued; ++c)
+                    mbar_wait(bar_full0 + 8 * (c % kStStages), (c / kStStages) & 1, nullptr);
+            }
+        }
+    } else if (warp < 2) {
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_done, 0, abort_flag));
+        if (ok) {
+            tc_fence_after();
+            float sv[kD];
+            const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
+            tmem_ld32(tmem_warp, *reinterpret_cast<float(*)[32]>(&sv[0]));
+            tmem_ld32(tmem_warp + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+            tmem_ld_wait();
+            float4 *dst = reinterpret_cast<float4 *>(s_part + (((size_t)bh * (G - 1) + g) * kD + tid) * kD);
+#pragma unroll
+            for (int j = 0; j < kD / 4; ++j) dst[j] = make_float4(sv[4 * j], sv[4 * j + 1], sv[4 * j + 2], sv[4 * j + 3]);
+        } else if (lane == 0) {
+            *abort_flag = 1;
+            atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 64);
 }
 
 // ------------------------------------------------------------------------------- host side
@@ -512,19 +680,58 @@ bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int C, boo
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// How a call is split along L.  The grid holds B*H*G CTAs, at most two per SM so that all of them are
+// resident at once; a group never has fewer than 8 chunks.
+struct SplitPlan {
+    int G, cpg;
+    size_t part_bytes;
+};
+SplitPlan split_plan(int B, int H, int L)
+{
+    int sms = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        sms <= 0)
+        sms = 148;
+    const long long bh = (long long)B * H;
+    const int nchunks = (L + kC - 1) / kC;
+    int G = 1;
+    if (bh < 2LL * sms) {
+        G = (int)((2LL * sms) / bh);
+        if (G > nchunks / 8) G = nchunks / 8;
+        if (G < 1) G = 1;
+    }
+    SplitPlan p;
+    p.cpg = (nchunks + G - 1) / G;
+    p.G = (nchunks + p.cpg - 1) / p.cpg;
+    p.part_bytes = (size_t)bh * (p.G - 1) * kD * kD * sizeof(float);
+    return p;
+}
+constexpr size_t kWsHeader = 512;   // word 0: asynchronous status; the rest: diagnostics
+
 template <typename TOut>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
-                        float scale, int *status, cudaStream_t stream)
+                        float scale, void *workspace, cudaStream_t stream)
 {
     CUtensorMap mq, mk, mv, mo;
     if (!make_map(&mq, q, B, H, L, kC, false) || !make_map(&mk, k, B, H, L, kC, false) ||
         !make_map(&mv, v, B, H, L, kC, false) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4))
         return CHELA_ERR_CUDA;
+    const SplitPlan plan = split_plan(B, H, L);
+    int *status = (int *)workspace;
+    float *s_part = (float *)((char *)workspace + kWsHeader);
+    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+    if (plan.G > 1) {
+        if (cudaFuncSetAttribute(linattn_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemState::bytes) != cudaSuccess)
+            return CHELA_ERR_CUDA;
+        linattn_state_kernel<<<B * H * (plan.G - 1), kThreads, SmemState::bytes, stream>>>(mk, mv, s_part, H, plan.G, plan.cpg, status);
+        if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
+    }
     auto kern = linattn_sm100_kernel<TOut>;
     const int smem = Smem<TOut>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return CHELA_ERR_CUDA;
-    kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status);
+    kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg);
     return last_launch_status();
 }
 
@@ -536,20 +743,22 @@ bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_
     return in_dtype == CHELA_BF16 && d == kD && (chunk == 64 || chunk == 128);
 }
 
-// 256 bytes: word 0 is the asynchronous status of the last launch that used this workspace.
-size_t linattn_sm100_workspace_bytes(int, int, int, int d, int) { return d == kD ? 512 : 0; }
+// Header (word 0 = asynchronous status of the last launch that used this workspace) followed by the
+// per-group state sums [B*H][G-1][64][64] fp32 of a call that is split along L.
+size_t linattn_sm100_workspace_bytes(int B, int H, int L, int d, int)
+{
+    return d == kD ? kWsHeader + split_plan(B, H, L).part_bytes : 0;
+}
 
 chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int d,
                                     int chunk, chela_dtype_t, chela_dtype_t out_dtype, int norm, float eps,
                                     float scale, void *workspace, cudaStream_t stream)
 {
     (void)d;
-    int *status = (int *)workspace;
-    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
     // The result does not depend on the chunk size: both supported values run on 64-token tiles.
     (void)chunk;
-    if (out_dtype == CHELA_F32) return launch_t<float>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
-    return launch_t<__nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+    if (out_dtype == CHELA_F32) return launch_t<float>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
+    return launch_t<__nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
 }
 
 }  // namespace chela

@@ -93,3 +93,35 @@ def test_sweep_shapes_sampled(B, L):
         got = to_numpy(o[b:b + 1, :, h:h + 1])
         assert rel_err(got, ref) <= TOL["bf16"], (B, L, b, h)
     assert bool(torch.isfinite(o).all())
+
+
+@pytest.mark.parametrize("B,L,H", [(1, 8192, 2), (1, 5000, 3), (1, 1100, 1), (2, 4096, 1)])
+def test_sequences_split_along_length(B, L, H):
+    """Few (batch, head) pairs: the tensor-core path splits each sequence into groups of chunks whose
+    initial states come from a separate K^T V pass; the result must still match the oracle."""
+    import torch
+    q, k, v = inputs.qkv(40 + L, B, L, H, 64, 64, "bf16")
+    assert chela.linattn_workspace_bytes(B, H, L, 64, 64, 64) > 512 + 64 * 64 * 4 - 1
+    for norm in (True, False):
+        got = run(q, k, v, "bf16", 64, norm=norm)
+        assert rel_err(got, oracle.linattn_recurrent(q, k, v, norm=norm)) <= TOL["bf16"]
+
+
+def test_async_status_is_ok_and_tensor_core_path_is_used():
+    import torch
+    assert chela.linattn_kernel_kind(2, 2, 256, 64, 64, 64, chela.BF16, chela.F32) == 2
+    assert chela.linattn_kernel_kind(2, 2, 256, 64, 64, 64, chela.F32, chela.F32) == 1
+    q, k, v = inputs.qkv(3, 2, 256, 2, 64, 64, "bf16")
+    ws = torch.zeros(chela.linattn_workspace_bytes(2, 2, 256, 64, 64, 64), dtype=torch.uint8, device="cuda")
+    chela.linattn_fwd(to_device(q, "bf16"), to_device(k, "bf16"), to_device(v, "bf16"), workspace=ws)
+    assert chela.async_status(ws) == chela.OK
+
+
+def test_workspace_too_small_is_rejected():
+    import torch
+    q, k, v = (to_device(a, "bf16") for a in inputs.qkv(3, 1, 4096, 1, 64, 64, "bf16"))
+    need = chela.linattn_workspace_bytes(1, 1, 4096, 64, 64, 64)
+    ws = torch.zeros(need - 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(chela.ChelaError) as e:
+        chela.linattn_fwd(q, k, v, workspace=ws)
+    assert e.value.status == chela.ERR_WORKSPACE
