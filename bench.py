@@ -31,9 +31,10 @@ SWEEP_L = (1024, 2048, 4096, 8192, 16384, 32768, 65536)
 # algorithmic bytes per token-head: read Q, K, V (bf16) once, write O (fp32) once
 BYTES_PER_TOKEN_HEAD = 3 * D * 2 + D * 4
 METRIC = "linattn_fwd_tokens_per_s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this workload,
-# from the ncu capture summarised under profiles/ (None until a capture exists)
-NCU_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
+# summarised in profiles/linattn_sm100_L2048_B16_ncu_full.md: 294.8 MB for 32768 tokens (B=16, L=2048, same
+# grid), scaled by tokens to the timed workload (traffic is proportional to tokens: every tile is read once)
+NCU_TRAFFIC_BYTES_PER_TOKEN = 294.8e6 / 32768
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -92,17 +93,27 @@ class ClockSampler(threading.Thread):
                 "sm_max_mhz": self.max_mhz, "reasons": seen, "samples": len(window)}
 
 
-def time_oracle_sample(n_batches: int, L: int, seed: int = 1234):
-    """Times the float64 oracle (recurrent form, as it stands) on n_batches x L tokens of the workload."""
+def oracle_inputs(n_batches: int, L: int, seed: int = 1234):
     import numpy as np
-    import oracle
     from paper_2406_08128_b200 import inputs
-    q, k, v = inputs.qkv(seed, n_batches, L, H, D, D, "bf16")
-    q, k, v = (a.astype(np.float64) for a in (q, k, v))
-    t0 = time.perf_counter()
-    oracle.linattn_recurrent(q, k, v)
-    dt = time.perf_counter() - t0
-    return n_batches * L / dt, dt, oracle.num_threads()
+    return tuple(a.astype(np.float64) for a in inputs.qkv(seed, n_batches, L, H, D, D, "bf16"))
+
+
+def time_oracle_sample(qkv64, budget_s: float = 0.0):
+    """Times the float64 oracle (recurrent form, as it stands) on the given inputs, repeating the pass until
+    ``budget_s`` seconds of CPU work have been spent.  Returns (tokens/s, seconds, passes, threads)."""
+    import oracle
+    q, k, v = qkv64
+    tokens = q.shape[0] * q.shape[1]
+    passes, total = 0, 0.0
+    while True:
+        t0 = time.perf_counter()
+        oracle.linattn_recurrent(q, k, v)
+        total += time.perf_counter() - t0
+        passes += 1
+        if total >= budget_s or passes >= 200:
+            break
+    return passes * tokens / total, total, passes, oracle.num_threads()
 
 
 def run_reference(args):
@@ -112,15 +123,16 @@ def run_reference(args):
         return
     import oracle
     oracle.build()
-    nb = 1
+    nb = max(1, min(4, TOTAL_TOKENS // L_MAIN))
+    data = oracle_inputs(nb, L_MAIN)
     times = []
     for i in range(args.warmup + args.steps):
-        tps, dt, cores = time_oracle_sample(nb, L_MAIN, seed=1234 + i)
+        tps, dt, _, cores = time_oracle_sample(data)
         if i >= args.warmup:
             times.append(dt)
     ms = 1e3 * sum(times) / len(times)
     value = nb * L_MAIN / (ms * 1e-3)
-    sample = "recurrent-form oracle on %d of %d sequences-batches (B=%d, L=%d, H=%d, d=%d) per step" % (
+    sample = "recurrent-form float64 oracle on %d of the %d batch rows of the step (B=%d, L=%d, H=%d, d=%d) per step" % (
         nb, TOTAL_TOKENS // L_MAIN, nb, L_MAIN, H, D)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
@@ -132,10 +144,27 @@ def run_reference(args):
     }))
 
 
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Elapsed time of the slowest rank (one MAX all-reduce of a scalar; the only collective of the job)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(ms_step: float, world: int, tokens_per_rank: int) -> float:
+    """Whole-job throughput of `world` independent replicas that each process tokens_per_rank per step."""
+    return world * tokens_per_rank / (ms_step * 1e-3)
+
+
 def workload_config():
-    return {"workload": "linattn_fwd sweep point L=16384: B=16, H=16, d_k=d_v=64, chunk=64, bf16 in, fp32 out",
+    return {"workload": "linattn_fwd sweep point L=%d: B=%d, H=16, d_k=d_v=64, chunk=64, bf16 in, fp32 out" % (
+                L_MAIN, TOTAL_TOKENS // L_MAIN),
             "B": TOTAL_TOKENS // L_MAIN, "L": L_MAIN, "H": H, "d_k": D, "d_v": D, "chunk": CHUNK,
-            "l2": "inputs+outputs 2.7 GB per step, far larger than L2: no flush needed"}
+            "l2": "inputs+outputs %.2f GB per step, larger than L2: no flush needed" % (BYTES_PER_TOKEN_HEAD * TOTAL_TOKENS * H / 1e9)}
 
 
 def main():
@@ -145,7 +174,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="chela", choices=["chela", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the sweep / config-2 / mixer / CPU-oracle extras")
+    ap.add_argument("--tokens", type=int, default=TOTAL_TOKENS, help="B*L of the timed step (profiling captures use a smaller case)")
+    ap.add_argument("--L", type=int, default=L_MAIN, help="sequence length of the timed step")
     args = ap.parse_args()
+    if (args.tokens, args.L) != (TOTAL_TOKENS, L_MAIN):
+        globals().update(TOTAL_TOKENS=args.tokens, L_MAIN=args.L)
+        args.no_extras = True
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         return run_reference(args)
@@ -176,8 +210,9 @@ def main():
     gen = torch.Generator(device=dev).manual_seed(100 + 14 + rank)
     flat = [(torch.randn(TOTAL_TOKENS * H * D, device=dev, generator=gen) * 0.125).to(torch.bfloat16) for _ in range(3)]
     out_flat = torch.empty(TOTAL_TOKENS * H * D, device=dev, dtype=torch.float32)
-    ws = torch.zeros(max(chela.linattn_workspace_bytes(4, H, 65536, D, D, CHUNK),
-                         chela.linattn_workspace_bytes(256, H, 1024, D, D, CHUNK), 256), dtype=torch.uint8, device=dev)
+    ws_bytes = max([chela.linattn_workspace_bytes(max(TOTAL_TOKENS // L, 1), H, L, D, D, CHUNK) for L in SWEEP_L + (L_MAIN,)]
+                   + [chela.linattn_workspace_bytes(8, 8, 4096, D, D, CHUNK)])
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
 
     def views(L):
         b = TOTAL_TOKENS // L
@@ -216,11 +251,8 @@ def main():
             torch.cuda.synchronize()
         clocks = sampler.summary(t_wall0, time.perf_counter())
         clocks["note"] = "timed region too short for NVML polling: window extended over an identical untimed burst"
-    t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
-    value = world * TOTAL_TOKENS / (ms_step * 1e-3)
+    ms_step = max_over_ranks(ms_total, world, dev) / args.steps
+    value = job_tokens_per_s(ms_step, world, TOTAL_TOKENS)
 
     # ---- end to end: host buffers in, host buffer out, through the same C-ABI call ---------------------
     host_in = [torch.empty(x.shape, dtype=x.dtype, pin_memory=True).copy_(x) for x in flat]
@@ -240,11 +272,8 @@ def main():
         e2e_step()
     ev1.record()
     barrier()
-    t = torch.tensor([ev0.elapsed_time(ev1)], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item()) / e2e_steps
-    e2e = {"value": world * TOTAL_TOKENS / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / e2e_steps
+    e2e = {"value": job_tokens_per_s(e2e_ms, world, TOTAL_TOKENS), "unit": "tokens/s", "ms_per_step": e2e_ms,
            "steps": e2e_steps, "h2d_bytes_per_step": int(sum(x.numel() * x.element_size() for x in flat)),
            "d2h_bytes_per_step": int(out_flat.numel() * out_flat.element_size())}
     del host_in, host_out
@@ -253,7 +282,8 @@ def main():
     alg_bytes = BYTES_PER_TOKEN_HEAD * TOTAL_TOKENS * H
     achieved = alg_bytes / (ms_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES, "peak_source": peak_kind,
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES_PER_TOKEN * TOTAL_TOKENS,
+                "traffic_source": "ncu capture of a 32768-token case scaled by tokens", "peak_source": peak_kind,
                 "kernel": "linattn_sm100_kernel<64,float>" if kind == 2 else "linattn_simt_kernel",
                 "algorithmic_bytes_per_launch": alg_bytes, "launch_ms": ms_step}
 
@@ -305,11 +335,13 @@ def main():
         # ---- CPU oracle on the host cores, bounded sample -----------------------------------------------
         import oracle
         oracle.build()
-        time_oracle_sample(1, 2048)  # warm the thread pool
-        tps, dt, cores = time_oracle_sample(2, L_MAIN)
-        line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle", "seconds": dt,
-                                "sample": "recurrent-form float64 oracle on 2 of the 16 sequences-batches "
-                                          "(B=2, L=16384, H=16, d=64) of the same workload"}
+        nb = max(1, min(4, TOTAL_TOKENS // L_MAIN))
+        data = oracle_inputs(nb, L_MAIN)
+        time_oracle_sample(oracle_inputs(1, 2048))  # warm the thread pool
+        tps, secs, passes, cores = time_oracle_sample(data, budget_s=12.0)
+        line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle", "seconds": secs,
+                                "sample": "recurrent-form float64 oracle, %d passes over %d of the %d batch rows of the "
+                                          "step (B=%d, L=%d, H=16, d=64)" % (passes, nb, TOTAL_TOKENS // L_MAIN, nb, L_MAIN)}
     sampler.stop()
     if rank == 0:
         print(json.dumps(line))
