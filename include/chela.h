@@ -111,6 +111,37 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
 chela_status_t chela_async_status(const void *workspace, cudaStream_t stream);
 
 /*
+ * chela_linattn_fwd without a caller-provided workspace and without any allocation.  (The paper has no
+ * counterpart: this is a packaging variant of the entry point above, same kernels, same results.)
+ *
+ * For callers that cannot allocate device memory: a plug-in inside a server whose device memory was all
+ * handed to another framework's pool at start-up, a latency-critical loop in which cudaMalloc (it may
+ * synchronise the device) is forbidden once initialisation is over, a component that only ever receives
+ * finished input and output buffers.  Inputs and outputs are still the caller's; only the scratch (the
+ * asynchronous status word and, for sequences that are split along L, the per-group state sums) comes
+ * from an 8 MiB array built into the library image.  Every GPU that loads the library holds those 8 MiB
+ * until the process exits.
+ *
+ *   - Arguments as chela_linattn_fwd, minus workspace and workspace_bytes.
+ *   - A call whose chela_linattn_workspace_bytes() exceeds 8 MiB returns CHELA_ERR_WORKSPACE and launches
+ *     nothing (use chela_linattn_fwd with your own workspace); with at most two CTAs per SM of split
+ *     work the need stays below 5 MiB on a B200, so this is a guard, not an expected outcome.
+ *   - The first call on each device looks up the device address of the built-in array (with that device
+ *     current) and caches it; make that first call during set-up, before any stream capture.
+ *   - The call itself calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - All calls on one GPU share the one array, which keeps the previous call's contents.  Nothing in it
+ *     needs to start at zero except the status word, which each launch clears on `stream` itself.  Two
+ *     calls that overlap on the GPU (different streams without an ordering event) race on it: order them.
+ *   - The asynchronous status word lives inside the built-in array and is not exposed; callers that want
+ *     to poll it use chela_linattn_fwd + chela_async_status.
+ */
+chela_status_t chela_linattn_fwd_static_ws(const void *q, const void *k, const void *v, void *o,
+                                           int B, int H, int L, int d_k, int d_v, int chunk,
+                                           chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                                           chela_norm_t norm, float norm_eps, float scale,
+                                           cudaStream_t stream);
+
+/*
  * Token mixer forward without the gates (Eq. 7, Eqs. 10-12, Eq. 8 without G_a):
  *   A = silu(shortconv(X));  Z = longconv(A)
  *   Q = Z W_q + b_q,  K = Z W_k + b_k            (qk_diag = 0: dense D x D weights)

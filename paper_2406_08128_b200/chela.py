@@ -37,6 +37,8 @@ _SIGNATURES = {
     "chela_linattn_fwd": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                    _c_float, _vp, _c_size_t, _vp]),
     "chela_async_status": (_c_int, [_vp, _vp]),
+    "chela_linattn_fwd_static_ws": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
+                                             _c_float, _vp]),
     "chela_mixer_workspace_bytes": (_c_size_t, [_c_int] * 5 + [_c_int]),
     "chela_mixer_fwd": (_c_int, [_vp, _vp, _c_int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _c_int, _c_int, _vp,
                                  _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_float,
@@ -146,6 +148,21 @@ def linattn_fwd(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale
     _check(lib().chela_linattn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, L, d_k, d_v, chunk, _dt(q), _dt(o),
                                    int(norm), float(eps), float(scale), _ptr(workspace), workspace.numel(),
                                    _stream()), "chela_linattn_fwd")
+    return o
+
+
+def linattn_fwd_static_ws(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale=1.0, out=None):
+    """chela_linattn_fwd_static_ws: same result as linattn_fwd, scratch from the library's built-in array.
+
+    For hosts that cannot allocate device memory; here torch still allocates the output unless ``out`` is
+    given, the library call itself allocates nothing.
+    """
+    B, L, H, d_k = q.shape
+    d_v = v.shape[3]
+    o = torch.empty((B, L, H, d_v), dtype=_tdtype(out_dtype), device=q.device) if out is None else out
+    _check(lib().chela_linattn_fwd_static_ws(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, L, d_k, d_v, chunk, _dt(q),
+                                             _dt(o), int(norm), float(eps), float(scale), _stream()),
+           "chela_linattn_fwd_static_ws")
     return o
 
 
