@@ -42,7 +42,10 @@ typedef enum {
     CHELA_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (reported asynchronously) */
 } chela_status_t;
 
-typedef enum { CHELA_F32 = 0, CHELA_BF16 = 1 } chela_dtype_t;
+/* CHELA_BF16_PAIR: a tensor stored as two bf16 planes of the same shape, the high plane first and the low
+ * plane directly after it (numel elements later); its value is hi + lo (about 16 mantissa bits).
+ * Accepted only where an entry point says so. */
+typedef enum { CHELA_F32 = 0, CHELA_BF16 = 1, CHELA_BF16_PAIR = 2 } chela_dtype_t;
 
 /* CHELA_NORM_RMS: o = r * (mean_j r_j^2 + eps)^(-1/2) over the d_v entries of one head's output
  * row, no learnable gain -- the library's reading of "Norm" in Eq. 2.  CHELA_NORM_NONE: o = r. */
@@ -99,6 +102,21 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
                                  chela_dtype_t in_dtype, chela_dtype_t out_dtype,
                                  chela_norm_t norm, float norm_eps, float scale,
                                  void *workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/*
+ * Dense projection with optional SiLU, the building block of the Q/K/V formation (Eq. 12; Eqs. 10-11 in
+ * their dense form): y = act(a w + bias), fp32 accumulation.
+ * a : [M, K], a_dtype in {F32, BF16, BF16_PAIR}.  w : [K, N] row-major, w_dtype in {F32, BF16}.
+ * bias : [N] fp32 or NULL.  y : [M, N], y_dtype in {F32, BF16, BF16_PAIR}.  act : 0 identity, 1 SiLU.
+ * Tensor-core path (tcgen05): a BF16 or BF16_PAIR, w BF16, y BF16 or BF16_PAIR, K a multiple of 64, N a
+ * multiple of 128.  Other combinations without a pair run on an fp32 SIMT kernel; pairs outside the
+ * tensor-core path are CHELA_ERR_UNSUPPORTED.  The workspace holds the asynchronous status word
+ * (chela_async_status).
+ */
+size_t chela_dense_workspace_bytes(void);
+chela_status_t chela_dense_fwd(const void *a, const void *w, const float *bias, void *y, int M, int K, int N,
+                               int act, chela_dtype_t a_dtype, chela_dtype_t w_dtype, chela_dtype_t y_dtype,
+                               void *workspace, size_t workspace_bytes, cudaStream_t stream);
 
 /*
  * Asynchronous status of the last chela_linattn_fwd / chela_mixer_fwd launch that used `workspace`.

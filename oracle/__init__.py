@@ -142,3 +142,15 @@ def mixer(x, w_short, k_long, w_q, w_k, w_v, H, b_q=None, b_k=None, b_v=None,
                          _p(bq), _p(bk), _p(bv), int(bool(qk_diag)), int(bool(v_silu)), _p(o), _p(z),
                          B, L, D, H, int(bool(norm)), ctypes.c_double(eps), int(bool(use_fft)))
     return (o, z) if return_z else o
+
+
+def dense(x, w, bias=None, act=False):
+    """y = act(x w + bias) by the plain triple loop; act = SiLU (Eq. 12)."""
+    x, w = _f64(x), _f64(w)
+    M, K = x.shape
+    assert w.shape[0] == K
+    N = w.shape[1]
+    b = None if bias is None else _f64(bias)
+    y = np.empty((M, N))
+    _load().oracle_dense(_p(x), _p(w), _p(b), _p(y), ctypes.c_size_t(M), K, N, int(bool(act)))
+    return y

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libchela.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
-F32, BF16 = 0, 1
+F32, BF16, BF16_PAIR = 0, 1, 2
 NORM_NONE, NORM_RMS = 0, 1
 
 _DTYPES = {torch.float32: F32, torch.bfloat16: BF16}
@@ -36,6 +36,9 @@ _SIGNATURES = {
     "chela_linattn_workspace_bytes": (_c_size_t, [_c_int] * 6),
     "chela_linattn_fwd": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                    _c_float, _vp, _c_size_t, _vp]),
+    "chela_dense_workspace_bytes": (_c_size_t, []),
+    "chela_dense_fwd": (_c_int, [_vp, _vp, _vp, _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _vp,
+                                 _c_size_t, _vp]),
     "chela_async_status": (_c_int, [_vp, _vp]),
     "chela_linattn_fwd_static_ws": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                              _c_float, _vp]),
@@ -164,6 +167,22 @@ def linattn_fwd_static_ws(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1
                                              _dt(o), int(norm), float(eps), float(scale), _stream()),
            "chela_linattn_fwd_static_ws")
     return o
+
+
+def dense_fwd(a, w, bias=None, act=False, a_dtype=None, y_dtype=BF16, out=None, workspace=None):
+    """y = act(a w + bias).  a [M,K] (a bf16 pair is passed as a [2,M,K] bf16 tensor with a_dtype=BF16_PAIR),
+    w [K,N]; returns y [M,N] (or [2,M,N] bf16 for y_dtype=BF16_PAIR)."""
+    a_dtype = _dt(a) if a_dtype is None else a_dtype
+    M, K = a.shape[-2], a.shape[-1]
+    N = w.shape[1]
+    if out is None:
+        shape = (2, M, N) if y_dtype == BF16_PAIR else (M, N)
+        out = torch.empty(shape, dtype=torch.float32 if y_dtype == F32 else torch.bfloat16, device=a.device)
+    if workspace is None:
+        workspace = _workspace(int(lib().chela_dense_workspace_bytes()), a.device)
+    _check(lib().chela_dense_fwd(_ptr(a), _ptr(w), _ptr(bias), _ptr(out), M, K, N, int(bool(act)), a_dtype, _dt(w),
+                                 y_dtype, _ptr(workspace), workspace.numel(), _stream()), "chela_dense_fwd")
+    return out
 
 
 def async_status(workspace) -> int:

@@ -115,6 +115,25 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
                                stream);
 }
 
+size_t chela_dense_workspace_bytes(void) { return 256; }
+
+chela_status_t chela_dense_fwd(const void *a, const void *w, const float *bias, void *y, int M, int K, int N, int act,
+                               chela_dtype_t a_dtype, chela_dtype_t w_dtype, chela_dtype_t y_dtype, void *workspace,
+                               size_t workspace_bytes, cudaStream_t stream)
+{
+    auto any_dtype = [](chela_dtype_t t) { return t == CHELA_F32 || t == CHELA_BF16 || t == CHELA_BF16_PAIR; };
+    if (!a || !w || !y || M < 1 || K < 1 || N < 1 || (act != 0 && act != 1) || !any_dtype(a_dtype) || !dtype_ok(w_dtype) ||
+        !any_dtype(y_dtype))
+        return CHELA_ERR_INVALID_ARG;
+    if (!aligned16(a) || !aligned16(w) || !aligned16(y) || !aligned16(workspace)) return CHELA_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < chela_dense_workspace_bytes()) return CHELA_ERR_WORKSPACE;
+    if (cudaMemsetAsync(workspace, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+    if (gemm_sm100_supported((size_t)M, K, N, a_dtype, w_dtype, y_dtype))
+        return launch_gemm_sm100(a, w, bias, y, (size_t)M, K, N, act, a_dtype, y_dtype, (int *)workspace, stream);
+    if (a_dtype == CHELA_BF16_PAIR || y_dtype == CHELA_BF16_PAIR) return CHELA_ERR_UNSUPPORTED;
+    return launch_gemm_simt(a, w, bias, y, (size_t)M, K, N, act, a_dtype, w_dtype, y_dtype, stream);
+}
+
 chela_status_t chela_async_status(const void *workspace, cudaStream_t stream)
 {
     if (!workspace) return CHELA_ERR_INVALID_ARG;

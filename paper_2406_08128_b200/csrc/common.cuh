@@ -13,7 +13,7 @@ inline chela_status_t last_launch_status() { return cuda_status(cudaGetLastError
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int next_pow2(int x) { int p = 1; while (p < x) p <<= 1; return p; }
-inline size_t dtype_size(chela_dtype_t t) { return t == CHELA_BF16 ? 2 : 4; }
+inline size_t dtype_size(chela_dtype_t t) { return t == CHELA_F32 ? 4 : (t == CHELA_BF16 ? 2 : 4); }  // pair: two bf16 planes
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 __device__ __forceinline__ float silu_f(float u) { return u / (1.0f + __expf(-u)); }
@@ -70,6 +70,10 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
 chela_status_t launch_gemm_simt(const void *a, const void *w, const float *bias, void *y, size_t M, int K,
                                 int N, int act, chela_dtype_t a_dtype, chela_dtype_t w_dtype,
                                 chela_dtype_t y_dtype, cudaStream_t stream);
+// tcgen05 GEMM: a bf16 or bf16 pair, w bf16, y bf16 or bf16 pair
+bool gemm_sm100_supported(size_t M, int K, int N, chela_dtype_t a_dtype, chela_dtype_t w_dtype, chela_dtype_t y_dtype);
+chela_status_t launch_gemm_sm100(const void *a, const void *w, const float *bias, void *y, size_t M, int K, int N,
+                                 int act, chela_dtype_t a_dtype, chela_dtype_t y_dtype, int *status, cudaStream_t stream);
 // y[m,c] = alpha[c] * z[m,c] + beta[c]
 chela_status_t launch_affine(const float *z, const void *alpha, const float *beta, float *y, size_t M, int D,
                              chela_dtype_t alpha_dtype, cudaStream_t stream);

@@ -1,0 +1,262 @@
+// Dense projection on the sm_100a tensor cores for the Q/K/V formation of the mixer (Eqs. 10-12 in
+// their dense form): Y = act(A W + bias), fp32 accumulation in TMEM.
+//
+// A [M, K] is bf16, or a bf16 pair (A = A_hi + A_lo, two planes): the long-convolution output and the
+// resulting Q, K must keep about 16 mantissa bits, because the normalised attention output loses its
+// leading digits to cancellation in Q K^T.  W [K, N] is bf16.  Y [M, N] is written as bf16 or as a
+// bf16 pair (hi = round(y), lo = round(y - hi)).
+//
+// Persistent kernel, one CTA per SM, 128 x 128 output tiles, K blocks of 64:
+//   warp 4 lane 0 : TMA producer (A_hi, A_lo: [128 rows] x 128 B K-major tiles; W: two [64 k-rows] x 128 B
+//                   atoms, MN-major), 3-stage ring
+//   warp 5 lane 0 : tcgen05.mma issuer, M = 128, N = 128 (64 cycles per instruction: full rate);
+//                   accumulators double-buffered in TMEM (2 x 128 columns)
+//   warps 0-3     : epilogue: TMEM -> bias, activation, hi/lo split -> swizzled staging -> TMA store,
+//                   32 rows x 64 columns per warp and box, ping-pong staging
+// Every wait is bounded; a timeout records CHELA_ERR_TIMEOUT in the status word and ends the CTA cleanly.
+#include "sm100_ptx.cuh"
+
+namespace chela {
+namespace {
+
+using namespace sm100;
+
+constexpr int BM = 128, BN = 128, BK = 64;
+constexpr int kStages = 3;
+constexpr int kThreads = 192;
+constexpr int kATile = BM * 128;        // 16 KB
+constexpr int kBTile = BK * 128 * 2;    // two 64-column atoms, 16 KB
+constexpr int kStageBytes = 2 * kATile + kBTile;
+constexpr int kStagingWarp = 4 * 32 * 128;   // per warp: 2 buffers x (hi, lo) x [32 rows x 128 B]
+
+struct Smem {
+    static constexpr int offStage = 0;
+    static constexpr int offStaging = kStages * kStageBytes;
+    static constexpr int offBar = offStaging + 4 * kStagingWarp;   // full[3], empty[3], tfull[2], tempty[2]
+    static constexpr int offTmem = offBar + 8 * (2 * kStages + 4);
+    static constexpr int offAbort = offTmem + 8;
+    static constexpr int bytes = offAbort + 8;
+};
+
+template <bool kAPair, bool kYPair>
+__global__ void __launch_bounds__(kThreads)
+gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_constant__ CUtensorMap tm_a_lo,
+                  const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y_hi,
+                  const __grid_constant__ CUtensorMap tm_y_lo, const float *__restrict__ bias, int M, int N, int K,
+                  int act, int *__restrict__ status)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {
+        if (threadIdx.x == 0) atomicExch(status, (int)CHELA_ERR_CUDA);
+        return;
+    }
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t bar_full0 = sbase + Smem::offBar, bar_empty0 = bar_full0 + 8 * kStages,
+                   bar_tfull0 = bar_empty0 + 8 * kStages, bar_tempty0 = bar_tfull0 + 16;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + Smem::offTmem);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + Smem::offAbort);
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full0 + 8 * s, 1);
+            mbar_init(bar_empty0 + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_tfull0 + 8 * b, 1);
+            mbar_init(bar_tempty0 + 8 * b, 4);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tm_a_hi);
+        tma_prefetch_desc(&tm_w);
+        tma_prefetch_desc(&tm_y_hi);
+    }
+    if (warp == 0) {
+        tmem_alloc(sbase + Smem::offTmem, 256);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int n_tiles = N / BN, m_tiles = (M + BM - 1) / BM, tiles = n_tiles * m_tiles, kblocks = K / BK;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int it = 0, issued = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x) {
+                const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    ok = mbar_wait(bar_empty0 + 8 * s, ((it / kStages) & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    const uint32_t bar = bar_full0 + 8 * s, dst = sbase + Smem::offStage + s * kStageBytes;
+                    mbar_expect_tx(bar, (kAPair ? 2 : 1) * kATile + kBTile);
+                    tma_load_2d(dst, &tm_a_hi, bar, kb * BK, m0);
+                    if (kAPair) tma_load_2d(dst + kATile, &tm_a_lo, bar, kb * BK, m0);
+                    tma_load_2d(dst + 2 * kATile, &tm_w, bar, n0, kb * BK);
+                    tma_load_2d(dst + 2 * kATile + BK * 128, &tm_w, bar, n0 + 64, kb * BK);
+                    issued = it + 1;
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+                // loads still in flight land in this CTA's shared memory: wait for them (bounded)
+                for (int c = issued > kStages ? issued - kStages : 0; c < issued; ++c) mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1, nullptr);
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(BM, BN, 0, 1);
+            int it = 0, ti = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
+                const int buf = ti & 1;
+                ok = mbar_wait(bar_tempty0 + 8 * buf, ((ti >> 1) & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d = tmem + buf * BN;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    ok = mbar_wait(bar_full0 + 8 * s, (it / kStages) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t st = sbase + Smem::offStage + s * kStageBytes;
+                    const uint32_t a_hi = desc_lo(st), a_lo = desc_lo(st + kATile), w_lo = desc_lo(st + 2 * kATile, BK * 128);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        umma_bf16(d, a_hi + 2 * k, w_lo + 128 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        if (kAPair) umma_bf16(d, a_lo + 2 * k, w_lo + 128 * k, idesc, 1u);
+                    }
+                    umma_commit(bar_empty0 + 8 * s);
+                }
+                if (ok) umma_commit(bar_tfull0 + 8 * buf);
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        // thread = accumulator row (TMEM lane); warp w stores rows 32w..32w+31 of the tile
+        uint8_t *stg = smem + Smem::offStaging + warp * kStagingWarp;
+        const uint32_t stg_u32 = sbase + Smem::offStaging + warp * kStagingWarp;
+        int ti = 0, nbox = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++ti) {
+            const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN, buf = ti & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull0 + 8 * buf, (ti >> 1) & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16) + buf * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 64; ++c, ++nbox) {
+                float acc[64];
+                tmem_ld32(trow + c * 64, *reinterpret_cast<float(*)[32]>(&acc[0]));
+                tmem_ld32(trow + c * 64 + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
+                tmem_ld_wait();
+                if (c == BN / 64 - 1) {
+                    // the accumulator is in registers: hand the TMEM buffer back to the issuer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_tempty0 + 8 * buf);
+                }
+                // staging buffer (nbox & 1) is free once the store issued two boxes ago has been read
+                if (lane == 0) bulk_wait_read1();
+                __syncwarp();
+                uint8_t *hi = stg + (nbox & 1) * (2 * 32 * 128), *lo = hi + 32 * 128;
+#pragma unroll
+                for (int j8 = 0; j8 < 8; ++j8) {
+                    uint32_t wh[4], wl[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int col = j8 * 8 + e * 2;
+                        float x0 = acc[col], x1 = acc[col + 1];
+                        if (bias) {
+                            x0 += bias[n0 + c * 64 + col];
+                            x1 += bias[n0 + c * 64 + col + 1];
+                        }
+                        if (act) {
+                            x0 = silu_f(x0);
+                            x1 = silu_f(x1);
+                        }
+                        const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                        wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                        if (kYPair) {
+                            const float2 hf = __bfloat1622float2(hh);
+                            wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                        }
+                    }
+                    const uint32_t off = sw128(lane, j8);
+                    *reinterpret_cast<uint4 *>(hi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                    if (kYPair) *reinterpret_cast<uint4 *>(lo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {   // rows past M are clipped by the copy engine
+                    const uint32_t src = stg_u32 + (nbox & 1) * (2 * 32 * 128);
+                    tma_store_2d(&tm_y_hi, src, n0 + c * 64, m0 + warp * 32);
+                    if (kYPair) tma_store_2d(&tm_y_lo, src + 32 * 128, n0 + c * 64, m0 + warp * 32);
+                    bulk_commit();
+                }
+            }
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+        }
+        if (lane == 0) bulk_wait0();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 256);
+}
+
+bool map_2d(CUtensorMap *map, const void *ptr, size_t rows, int cols, int box_cols, int box_rows)
+{
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    return make_map_sw128(map, ptr, false, 2, dims, strides, box);
+}
+
+}  // namespace
+
+bool gemm_sm100_supported(size_t M, int K, int N, chela_dtype_t a_dtype, chela_dtype_t w_dtype, chela_dtype_t y_dtype)
+{
+    return M >= 1 && M < (1ull << 31) && K % BK == 0 && N % BN == 0 && w_dtype == CHELA_BF16 &&
+           (a_dtype == CHELA_BF16 || a_dtype == CHELA_BF16_PAIR) && (y_dtype == CHELA_BF16 || y_dtype == CHELA_BF16_PAIR);
+}
+
+// a, y: for a bf16 pair the low plane follows the high plane (M*K resp. M*N elements later).
+chela_status_t launch_gemm_sm100(const void *a, const void *w, const float *bias, void *y, size_t M, int K, int N,
+                                 int act, chela_dtype_t a_dtype, chela_dtype_t y_dtype, int *status, cudaStream_t stream)
+{
+    const bool a_pair = a_dtype == CHELA_BF16_PAIR, y_pair = y_dtype == CHELA_BF16_PAIR;
+    const __nv_bfloat16 *a_hi = (const __nv_bfloat16 *)a, *a_lo = a_pair ? a_hi + M * K : a_hi;
+    __nv_bfloat16 *y_hi = (__nv_bfloat16 *)y, *y_lo = y_pair ? y_hi + M * N : y_hi;
+    CUtensorMap ma_hi, ma_lo, mw, my_hi, my_lo;
+    if (!map_2d(&ma_hi, a_hi, M, K, BK, BM) || !map_2d(&ma_lo, a_lo, M, K, BK, BM) || !map_2d(&mw, w, K, N, 64, BK) ||
+        !map_2d(&my_hi, y_hi, M, N, 64, 32) || !map_2d(&my_lo, y_lo, M, N, 64, 32))
+        return CHELA_ERR_CUDA;
+    int sms = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+    const long long tiles = (long long)((M + BM - 1) / BM) * (N / BN);
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float *, int, int, int, int, int *) =
+        a_pair ? (y_pair ? gemm_sm100_kernel<true, true> : gemm_sm100_kernel<true, false>)
+               : (y_pair ? gemm_sm100_kernel<false, true> : gemm_sm100_kernel<false, false>);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes) != cudaSuccess) return CHELA_ERR_CUDA;
+    kern<<<grid, kThreads, Smem::bytes, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status);
+    return last_launch_status();
+}
+
+}  // namespace chela
