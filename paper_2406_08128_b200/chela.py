@@ -141,14 +141,18 @@ def linattn_workspace_bytes(B, H, L, d_k, d_v, chunk) -> int:
     return int(lib().chela_linattn_workspace_bytes(B, H, L, d_k, d_v, chunk))
 
 
-def linattn_fwd(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale=1.0, out=None, workspace=None):
-    """q,k [B,L,H,d_k], v [B,L,H,d_v] -> o [B,L,H,d_v] of out_dtype."""
-    B, L, H, d_k = q.shape
-    d_v = v.shape[3]
+def linattn_fwd(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale=1.0, out=None, workspace=None,
+                in_dtype=None):
+    """q,k [B,L,H,d_k], v [B,L,H,d_v] -> o [B,L,H,d_v] of out_dtype.
+
+    With in_dtype=BF16_PAIR q, k, v are [2,B,L,H,d] bf16 tensors (high plane, low plane)."""
+    in_dtype = _dt(q) if in_dtype is None else in_dtype
+    B, L, H, d_k = q.shape[-4:]
+    d_v = v.shape[-1]
     o = torch.empty((B, L, H, d_v), dtype=_tdtype(out_dtype), device=q.device) if out is None else out
     if workspace is None:
         workspace = _workspace(linattn_workspace_bytes(B, H, L, d_k, d_v, chunk), q.device)
-    _check(lib().chela_linattn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, L, d_k, d_v, chunk, _dt(q), _dt(o),
+    _check(lib().chela_linattn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, L, d_k, d_v, chunk, in_dtype, _dt(o),
                                    int(norm), float(eps), float(scale), _ptr(workspace), workspace.numel(),
                                    _stream()), "chela_linattn_fwd")
     return o

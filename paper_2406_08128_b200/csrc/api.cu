@@ -49,10 +49,10 @@ int chela_version(void) { return 100; }
 int chela_linattn_kernel_kind(int B, int H, int L, int d_k, int d_v, int chunk, chela_dtype_t in_dtype,
                               chela_dtype_t out_dtype)
 {
-    if (B < 1 || H < 1 || L < 1 || !dtype_ok(in_dtype) || !dtype_ok(out_dtype)) return 0;
+    if (B < 1 || H < 1 || L < 1 || !(dtype_ok(in_dtype) || in_dtype == CHELA_BF16_PAIR) || !dtype_ok(out_dtype)) return 0;
     if (d_k != d_v || (d_k != 64 && d_k != 128) || (chunk != 64 && chunk != 128)) return 0;
     if (linattn_sm100_supported(B, H, L, d_k, chunk, in_dtype, out_dtype)) return 2;
-    return 1;
+    return in_dtype == CHELA_BF16_PAIR ? 0 : 1;
 }
 
 chela_status_t chela_shortconv_fwd(const void *x, const float *w, const float *bias, void *y, int B, int L,
@@ -98,7 +98,7 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
                                  void *workspace, size_t workspace_bytes, cudaStream_t stream)
 {
     if (!q || !k || !v || !o || B < 1 || H < 1 || L < 1 || d_k < 1 || d_v < 1 || chunk < 1 ||
-        !dtype_ok(in_dtype) || !dtype_ok(out_dtype) || (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) ||
+        !(dtype_ok(in_dtype) || in_dtype == CHELA_BF16_PAIR) || !dtype_ok(out_dtype) || (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) ||
         !(norm_eps >= 0.f))
         return CHELA_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(workspace))

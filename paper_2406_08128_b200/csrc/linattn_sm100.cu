@@ -33,18 +33,21 @@ constexpr int kThreads = 160;            // 4 compute warps + 1 issuer warp
 // ------------------------------------------------------------------------------- kernel
 
 constexpr int kC = 64;       // tokens per tile
-constexpr int kStages = 3;
 constexpr int kTile = kC * 128;   // one 64-row x 128-byte tile
 
-template <typename TOut>
+// kPair: Q, K, V arrive as bf16 pairs (hi + lo planes); every product then takes three tensor-core
+// terms (hi*hi + hi*lo + lo*hi) and the score tile is kept as a pair too.
+template <typename TOut, bool kPair>
 struct Smem {
+    static constexpr int kStages = kPair ? 2 : 3;
+    static constexpr int kTilesPerStage = kPair ? 6 : 3;  // Q, K, V (hi), then Q, K, V (lo); adjacent
     static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as 128-byte wide boxes
-    static constexpr int offPT = 0;                       // masked scores, transposed: rows = s, 64 t per row
-    static constexpr int offShi = offPT + kTile;          // state, bf16 high part: rows = d_k
+    static constexpr int offPT = 0;                       // masked scores, transposed: rows = s, 64 t per row (hi, lo)
+    static constexpr int offShi = offPT + (kPair ? 2 : 1) * kTile;   // state, bf16 high part: rows = d_k
     static constexpr int offSlo = offShi + kTile;         // state, bf16 low part
     static constexpr int offO = offSlo + kTile;           // output staging
-    static constexpr int offStage = offO + kOBoxes * kTile;   // per stage: Q, K, V tiles, adjacent
-    static constexpr int offBar = offStage + kStages * 3 * kTile;   // full[kStages], p, o, pt, s
+    static constexpr int offStage = offO + kOBoxes * kTile;
+    static constexpr int offBar = offStage + kStages * kTilesPerStage * kTile;   // full[kStages], p, o, pt, s
     static constexpr int offTmem = offBar + 8 * (kStages + 4);
     static constexpr int offAbort = offTmem + 8;
     static constexpr int bytes = offAbort + 8;
@@ -63,7 +66,7 @@ constexpr int kColPT = 64;   // rows 64..127: transposed scores; 64 columns
 #define TDUMP(slot)
 #endif
 
-template <typename TOut>
+template <typename TOut, bool kPair>
 __global__ void __launch_bounds__(kThreads)
 linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
@@ -72,7 +75,9 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 {
     // Grid: one CTA per (batch*head, group).  Group g covers chunks [g*cpg, (g+1)*cpg) of its sequence and
     // starts from the state sum_{g' < g} s_part[bh][g'] (per-group K^T V sums written by the state kernel).
-    using SM = Smem<TOut>;
+    using SM = Smem<TOut, kPair>;
+    constexpr int kStages = SM::kStages;
+    constexpr int kTPS = SM::kTilesPerStage;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     if (sbase & 1023u) {  // swizzled tiles need a 1024-byte aligned base: report instead of corrupting
@@ -120,13 +125,16 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         // =========================================== issuer: TMA loads and every tcgen05.mma ==========
         if (lane == 0) {
             TDECL;
-            auto stage_base = [&](int chunk) { return sbase + SM::offStage + (chunk % kStages) * 3 * kTile; };
+            auto stage_base = [&](int chunk) { return sbase + SM::offStage + (chunk % kStages) * kTPS * kTile; };
             auto issue_load = [&](int chunk) {
                 const uint32_t bar = bar_full0 + 8 * (chunk % kStages), dst = stage_base(chunk);
-                mbar_expect_tx(bar, 3 * kTile);
-                tma_load_4d(dst, &tm_q, bar, 0, h, (c0 + chunk) * kC, b);
-                tma_load_4d(dst + kTile, &tm_k, bar, 0, h, (c0 + chunk) * kC, b);
-                tma_load_4d(dst + 2 * kTile, &tm_v, bar, 0, h, (c0 + chunk) * kC, b);
+                mbar_expect_tx(bar, kTPS * kTile);
+#pragma unroll
+                for (int pl = 0; pl < (kPair ? 2 : 1); ++pl) {
+                    tma_load_5d(dst + (3 * pl) * kTile, &tm_q, bar, 0, h, (c0 + chunk) * kC, b, pl);
+                    tma_load_5d(dst + (3 * pl + 1) * kTile, &tm_k, bar, 0, h, (c0 + chunk) * kC, b, pl);
+                    tma_load_5d(dst + (3 * pl + 2) * kTile, &tm_v, bar, 0, h, (c0 + chunk) * kC, b, pl);
+                }
             };
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [Q;K] (K-major) x Q^T (K-major)
             constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;K] (K-major) x S (MN-major)
@@ -138,6 +146,13 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const uint32_t qk_lo = desc_lo(stage_base(chunk));
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk_lo + 2 * k, qk_lo + 2 * k, idescG1, k > 0);
+                if (kPair) {   // + K_hi Q_lo^T + K_lo Q_hi^T
+                    const uint32_t qk2_lo = desc_lo(stage_base(chunk) + 3 * kTile);
+#pragma unroll
+                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk_lo + 2 * k, qk2_lo + 2 * k, idescG1, 1);
+#pragma unroll
+                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk2_lo + 2 * k, qk_lo + 2 * k, idescG1, 1);
+                }
                 umma_commit(bar_p);
                 return true;
             };
@@ -161,6 +176,11 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, shi_lo + 128 * k, idescG2, k > 0, 1);
 #pragma unroll
                     for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, slo_lo + 128 * k, idescG2, 1, 1);
+                    if (kPair) {   // + Q_lo S_hi
+                        const uint32_t qk2_lo = desc_lo(st + 3 * kTile);
+#pragma unroll
+                        for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk2_lo + 2 * k, shi_lo + 128 * k, idescG2, 1, 1);
+                    }
                     TMARK(1);
                 }
                 // G3: OS += [P^T | K]^T V; atom 0 = score tile, atom 1 = K tile of this stage
@@ -172,6 +192,14 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k)
                     umma_bf16(tmem + kColOS, a_lo + 128 * k, v_lo + 128 * k, idescG3, (i > 0 || has_init || k > 0) ? 1u : 0u);
+                if (kPair) {   // + [P_hi^T | K_hi]^T V_lo + [P_lo^T | K_lo]^T V_hi
+                    const uint32_t v2_lo = desc_lo(st + 5 * kTile);
+                    const uint32_t a2_lo = desc_lo(sbase + SM::offPT + kTile, st + 4 * kTile - (sbase + SM::offPT + kTile));
+#pragma unroll
+                    for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS, a_lo + 128 * k, v2_lo + 128 * k, idescG3, 1);
+#pragma unroll
+                    for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS, a2_lo + 128 * k, v_lo + 128 * k, idescG3, 1);
+                }
                 umma_commit(bar_o);
                 if (i + 1 < nchunks) {
                     ok = issue_scores(i + 1);
@@ -270,15 +298,21 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const bool live = cb == 1 || warp == 2;
 #pragma unroll
                     for (int c8 = 0; c8 < 4; ++c8) {
-                        uint32_t w[4];
+                        uint32_t w[4], w2[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int t = cb * 32 + c8 * 8 + e * 2;
-                            const float lo = (live && t >= r) ? p[cb][c8 * 8 + e * 2] : 0.f;
-                            const float hi = (live && t + 1 >= r) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
-                            w[e] = pack_bf16(lo, hi);
+                            const float x0 = (live && t >= r) ? p[cb][c8 * 8 + e * 2] : 0.f;
+                            const float x1 = (live && t + 1 >= r) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
+                            const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                            w[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                            if (kPair) {
+                                const float2 hf = __bfloat1622float2(hh);
+                                w2[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                            }
                         }
                         *reinterpret_cast<uint4 *>(sP + sw128(r, cb * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                        if (kPair) *reinterpret_cast<uint4 *>(sP + kTile + sw128(r, cb * 4 + c8)) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
                     }
                 }
                 fence_proxy_async();
@@ -330,8 +364,8 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (lane == 0) {
 #pragma unroll
                     for (int bx = 0; bx < SM::kOBoxes; ++bx)
-                        tma_store_4d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
-                                     (c0 + i) * kC + warp * 32, b);
+                        tma_store_5d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
+                                     (c0 + i) * kC + warp * 32, b, 0);   // the map's rank is 5 (plane = 0)
                     bulk_commit();
                 }
                 TMARK(3);
@@ -371,19 +405,23 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 // One tcgen05.mma group per chunk: A = [K_i | V_i] (MN-major, two atoms), B = V_i; rows 0..63 of the
 // accumulator are K^T V, rows 64..127 (V^T V) are ignored.
 constexpr int kStStages = 4;
+template <bool kPair>
 struct SmemState {
-    static constexpr int offStage = 0;                              // per stage: K, V tiles, adjacent
-    static constexpr int offBar = kStStages * 2 * kTile;            // full[kStStages], empty[kStStages], done
+    static constexpr int kTilesPerStage = kPair ? 4 : 2;           // K, V (hi) then K, V (lo); adjacent
+    static constexpr int offStage = 0;
+    static constexpr int offBar = kStStages * kTilesPerStage * kTile;   // full[kStStages], empty[kStStages], done
     static constexpr int offTmem = offBar + 8 * (2 * kStStages + 1);
     static constexpr int offAbort = offTmem + 8;
     static constexpr int bytes = offAbort + 8;
 };
 
+template <bool kPair>
 __global__ void __launch_bounds__(kThreads)
 linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                      float *__restrict__ s_part, int H, int G, int cpg, int *__restrict__ status)
 {
-    using SM = SmemState;
+    using SM = SmemState<kPair>;
+    constexpr int kTPS = SM::kTilesPerStage;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     if (sbase & 1023u) {
@@ -422,10 +460,13 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     if (warp == 4) {
         if (lane == 0) {
             auto issue_load = [&](int chunk) {
-                const uint32_t bar = bar_full0 + 8 * (chunk % kStStages), dst = sbase + SM::offStage + (chunk % kStStages) * 2 * kTile;
-                mbar_expect_tx(bar, 2 * kTile);
-                tma_load_4d(dst, &tm_k, bar, 0, h, (c0 + chunk) * kC, b);
-                tma_load_4d(dst + kTile, &tm_v, bar, 0, h, (c0 + chunk) * kC, b);
+                const uint32_t bar = bar_full0 + 8 * (chunk % kStStages), dst = sbase + SM::offStage + (chunk % kStStages) * kTPS * kTile;
+                mbar_expect_tx(bar, kTPS * kTile);
+#pragma unroll
+                for (int pl = 0; pl < (kPair ? 2 : 1); ++pl) {
+                    tma_load_5d(dst + 2 * pl * kTile, &tm_k, bar, 0, h, (c0 + chunk) * kC, b, pl);
+                    tma_load_5d(dst + (2 * pl + 1) * kTile, &tm_v, bar, 0, h, (c0 + chunk) * kC, b, pl);
+                }
             };
             constexpr uint32_t idesc = make_idesc(128, kD, 1, 1);
             int loads_issued = 0, consumed = 0;
@@ -436,10 +477,17 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 ok = mbar_wait(bar_full0 + 8 * stage, (i / kStStages) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t st = sbase + SM::offStage + stage * 2 * kTile;
+                const uint32_t st = sbase + SM::offStage + stage * kTPS * kTile;
                 const uint32_t a_lo = desc_lo(st, kTile), v_lo = desc_lo(st + kTile);
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem, a_lo + 128 * k, v_lo + 128 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                if (kPair) {   // + K_hi^T V_lo + K_lo^T V_hi
+                    const uint32_t a2_lo = desc_lo(st + 2 * kTile, kTile), v2_lo = desc_lo(st + 3 * kTile);
+#pragma unroll
+                    for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem, a_lo + 128 * k, v2_lo + 128 * k, idesc, 1);
+#pragma unroll
+                    for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem, a2_lo + 128 * k, v_lo + 128 * k, idesc, 1);
+                }
                 umma_commit(bar_empty0 + 8 * stage);
                 consumed = i + 1;
                 if (i + kStStages < nchunks) {
@@ -484,22 +532,24 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 // [B, L, H, 64] viewed as a rank-4 tensor (d, H, L, B); box = (128 bytes of d) x 1 x C x 1, 128-byte
 // swizzle.  Loads: rows past L are out of bounds for the copy engine and arrive as zeros.  Stores: rows
 // past L are clipped.
-bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int C, bool f32)
+// `planes` = 2 for a bf16 pair (the low plane follows the high plane), else 1: always a rank-5 map.
+bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int C, bool f32, int planes)
 {
     const cuuint64_t es = f32 ? 4 : 2;
-    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)kD * es, (cuuint64_t)H * kD * es, (cuuint64_t)L * H * kD * es};
-    const cuuint32_t box[4] = {(cuuint32_t)(128 / es), 1, (cuuint32_t)C, 1};
-    return make_map_sw128(map, ptr, f32, 4, dims, strides, box);
+    const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B, (cuuint64_t)planes};
+    const cuuint64_t strides[4] = {(cuuint64_t)kD * es, (cuuint64_t)H * kD * es, (cuuint64_t)L * H * kD * es,
+                                   (cuuint64_t)B * L * H * kD * es};
+    const cuuint32_t box[5] = {(cuuint32_t)(128 / es), 1, (cuuint32_t)C, 1, 1};
+    return make_map_sw128(map, ptr, f32, 5, dims, strides, box);
 }
 
-// How a call is split along L.  The grid holds B*H*G CTAs, at most two per SM so that all of them are
-// resident at once; a group never has fewer than 8 chunks.
+// How a call is split along L.  The grid holds B*H*G CTAs, no more than are resident at once (two per SM,
+// one per SM for bf16-pair inputs); a group never has fewer than 8 chunks.
 struct SplitPlan {
     int G, cpg;
     size_t part_bytes;
 };
-SplitPlan split_plan(int B, int H, int L)
+SplitPlan split_plan(int B, int H, int L, bool pair)
 {
     int sms = 0;
     int dev = 0;
@@ -508,9 +558,10 @@ SplitPlan split_plan(int B, int H, int L)
         sms = 148;
     const long long bh = (long long)B * H;
     const int nchunks = (L + kC - 1) / kC;
+    const long long slots = (pair ? 1LL : 2LL) * sms;   // resident CTAs: shared memory allows 2 per SM, 1 for pairs
     int G = 1;
-    if (bh < 2LL * sms) {
-        G = (int)((2LL * sms) / bh);
+    if (bh < slots) {
+        G = (int)(slots / bh);
         if (G > nchunks / 8) G = nchunks / 8;
         if (G < 1) G = 1;
     }
@@ -522,26 +573,28 @@ SplitPlan split_plan(int B, int H, int L)
 }
 constexpr size_t kWsHeader = 512;   // word 0: asynchronous status; the rest: diagnostics
 
-template <typename TOut>
+template <typename TOut, bool kPair>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
                         float scale, void *workspace, cudaStream_t stream)
 {
     CUtensorMap mq, mk, mv, mo;
-    if (!make_map(&mq, q, B, H, L, kC, false) || !make_map(&mk, k, B, H, L, kC, false) ||
-        !make_map(&mv, v, B, H, L, kC, false) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4))
+    const int planes = kPair ? 2 : 1;
+    if (!make_map(&mq, q, B, H, L, kC, false, planes) || !make_map(&mk, k, B, H, L, kC, false, planes) ||
+        !make_map(&mv, v, B, H, L, kC, false, planes) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4, 1))
         return CHELA_ERR_CUDA;
-    const SplitPlan plan = split_plan(B, H, L);
+    const SplitPlan plan = split_plan(B, H, L, kPair);
     int *status = (int *)workspace;
     float *s_part = (float *)((char *)workspace + kWsHeader);
     if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
     if (plan.G > 1) {
-        if (cudaFuncSetAttribute(linattn_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemState::bytes) != cudaSuccess)
+        auto skern = linattn_state_kernel<kPair>;
+        if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemState<kPair>::bytes) != cudaSuccess)
             return CHELA_ERR_CUDA;
-        linattn_state_kernel<<<B * H * (plan.G - 1), kThreads, SmemState::bytes, stream>>>(mk, mv, s_part, H, plan.G, plan.cpg, status);
+        skern<<<B * H * (plan.G - 1), kThreads, SmemState<kPair>::bytes, stream>>>(mk, mv, s_part, H, plan.G, plan.cpg, status);
         if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
     }
-    auto kern = linattn_sm100_kernel<TOut>;
-    const int smem = Smem<TOut>::bytes;
+    auto kern = linattn_sm100_kernel<TOut, kPair>;
+    const int smem = Smem<TOut, kPair>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return CHELA_ERR_CUDA;
     kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg);
@@ -550,28 +603,35 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
 
 }  // namespace
 
-bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_t in_dtype, chela_dtype_t)
+bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype)
 {
     (void)B; (void)H; (void)L;
-    return in_dtype == CHELA_BF16 && d == kD && (chunk == 64 || chunk == 128);
+    return (in_dtype == CHELA_BF16 || in_dtype == CHELA_BF16_PAIR) && (out_dtype == CHELA_F32 || out_dtype == CHELA_BF16) &&
+           d == kD && (chunk == 64 || chunk == 128);
 }
 
 // Header (word 0 = asynchronous status of the last launch that used this workspace) followed by the
 // per-group state sums [B*H][G-1][64][64] fp32 of a call that is split along L.
 size_t linattn_sm100_workspace_bytes(int B, int H, int L, int d, int)
 {
-    return d == kD ? kWsHeader + split_plan(B, H, L).part_bytes : 0;
+    if (d != kD) return 0;
+    const size_t a = split_plan(B, H, L, false).part_bytes, b = split_plan(B, H, L, true).part_bytes;
+    return kWsHeader + (a > b ? a : b);   // the query does not know the input dtype: cover both plans
 }
 
 chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int d,
-                                    int chunk, chela_dtype_t, chela_dtype_t out_dtype, int norm, float eps,
+                                    int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps,
                                     float scale, void *workspace, cudaStream_t stream)
 {
     (void)d;
     // The result does not depend on the chunk size: both supported values run on 64-token tiles.
     (void)chunk;
-    if (out_dtype == CHELA_F32) return launch_t<float>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
-    return launch_t<__nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
+    if (in_dtype == CHELA_BF16_PAIR) {
+        if (out_dtype == CHELA_F32) return launch_t<float, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
+        return launch_t<__nv_bfloat16, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
+    }
+    if (out_dtype == CHELA_F32) return launch_t<float, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
+    return launch_t<__nv_bfloat16, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
 }
 
 }  // namespace chela
