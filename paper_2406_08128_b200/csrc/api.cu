@@ -127,7 +127,7 @@ chela_status_t chela_dense_fwd(const void *a, const void *w, const float *bias, 
         return CHELA_ERR_INVALID_ARG;
     if (!aligned16(a) || !aligned16(w) || !aligned16(y) || !aligned16(workspace)) return CHELA_ERR_INVALID_ARG;
     if (!workspace || workspace_bytes < chela_dense_workspace_bytes()) return CHELA_ERR_WORKSPACE;
-    if (cudaMemsetAsync(workspace, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+    if (cudaMemsetAsync(workspace, 0, 2 * sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
     if (gemm_sm100_supported((size_t)M, K, N, a_dtype, w_dtype, y_dtype))
         return launch_gemm_sm100(a, w, bias, y, (size_t)M, K, N, act, a_dtype, y_dtype, (int *)workspace, stream);
     if (a_dtype == CHELA_BF16_PAIR || y_dtype == CHELA_BF16_PAIR) return CHELA_ERR_UNSUPPORTED;
@@ -137,11 +137,13 @@ chela_status_t chela_dense_fwd(const void *a, const void *w, const float *bias, 
 chela_status_t chela_async_status(const void *workspace, cudaStream_t stream)
 {
     if (!workspace) return CHELA_ERR_INVALID_ARG;
-    int word = 0;
-    if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+    int word[2] = {0, 0};   // word 0: attention kernels (or the only kernel of the call); word 1: the mixer's GEMMs
+    if (cudaMemcpyAsync(word, workspace, sizeof(word), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess)
         return CHELA_ERR_CUDA;
-    return word == (int)CHELA_ERR_TIMEOUT ? CHELA_ERR_TIMEOUT : CHELA_OK;
+    if (word[0] == (int)CHELA_ERR_TIMEOUT || word[1] == (int)CHELA_ERR_TIMEOUT) return CHELA_ERR_TIMEOUT;
+    if (word[0] == (int)CHELA_ERR_CUDA || word[1] == (int)CHELA_ERR_CUDA) return CHELA_ERR_CUDA;
+    return CHELA_OK;
 }
 
 size_t chela_mixer_workspace_bytes(int B, int L, int D, int H, int chunk, chela_dtype_t)
@@ -175,9 +177,36 @@ chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_wi
           *vv = (float *)(ws + p.off_v);
     const size_t M = (size_t)B * L;
 
-    // Z = K_l(silu(K_s(X)))  (Eq. 7), kept in fp32
-    chela_status_t st = launch_longconv(x, k_long, w_short, short_width, z, B, L, D, in_dtype, CHELA_F32,
-                                        ws + p.off_conv, stream);
+    const size_t n = M * D;
+    // Tensor-core path: every intermediate (Z, Q, K, V) is a bf16 pair (hi + lo, about 16 mantissa bits) and
+    // every product takes three tensor-core terms; single bf16 intermediates would cost the normalised
+    // output its leading digits (cancellation in Q K^T on rows with a small pre-norm RMS).
+    const bool tensor_path = in_dtype == CHELA_BF16 && d == 64 &&
+                             gemm_sm100_supported(M, D, D, CHELA_BF16_PAIR, CHELA_BF16, CHELA_BF16_PAIR);
+    chela_status_t st;
+    if (tensor_path) {
+        __nv_bfloat16 *zp = (__nv_bfloat16 *)z, *qp = (__nv_bfloat16 *)qq, *kp = (__nv_bfloat16 *)kk, *vp = (__nv_bfloat16 *)vv;
+        int *status = (int *)ws + 1;   // word 1 of the header: the GEMMs; word 0: the attention kernels
+        st = launch_longconv(x, k_long, w_short, short_width, zp, B, L, D, in_dtype, CHELA_BF16_PAIR, ws + p.off_conv, stream);
+        if (st != CHELA_OK) return st;
+        if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+        if (qk_diag) {
+            st = launch_affine_pair(zp, w_q, b_q, qp, M, D, in_dtype, stream);
+            if (st == CHELA_OK) st = launch_affine_pair(zp, w_k, b_k, kp, M, D, in_dtype, stream);
+        } else {
+            st = launch_gemm_sm100(zp, w_q, b_q, qp, M, D, D, 0, CHELA_BF16_PAIR, CHELA_BF16_PAIR, status, stream);
+            if (st == CHELA_OK) st = launch_gemm_sm100(zp, w_k, b_k, kp, M, D, D, 0, CHELA_BF16_PAIR, CHELA_BF16_PAIR, status, stream);
+        }
+        if (st != CHELA_OK) return st;
+        st = launch_gemm_sm100(x, w_v, b_v, vp, M, D, D, v_silu ? 1 : 0, CHELA_BF16, CHELA_BF16_PAIR, status, stream);
+        if (st != CHELA_OK) return st;
+        return launch_linattn_sm100(qp, kp, vp, o, B, H, L, d, chunk, CHELA_BF16_PAIR, out_dtype, (int)norm, norm_eps, 1.0f,
+                                    ws + p.off_attn, stream);
+    }
+    (void)n;
+    // fp32 path.  Z = K_l(silu(K_s(X)))  (Eq. 7), kept in fp32
+    st = launch_longconv(x, k_long, w_short, short_width, z, B, L, D, in_dtype, CHELA_F32,
+                         ws + p.off_conv, stream);
     if (st != CHELA_OK) return st;
     // Q, K from Z (Eqs. 10-11, or dense projections), V from X (Eq. 12)
     if (qk_diag) {

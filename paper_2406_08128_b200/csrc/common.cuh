@@ -78,4 +78,8 @@ chela_status_t launch_gemm_sm100(const void *a, const void *w, const float *bias
 chela_status_t launch_affine(const float *z, const void *alpha, const float *beta, float *y, size_t M, int D,
                              chela_dtype_t alpha_dtype, cudaStream_t stream);
 
+// the same on bf16 pairs ([2][M*D] bf16 in and out)
+chela_status_t launch_affine_pair(const void *z, const void *alpha, const float *beta, void *y, size_t M, int D,
+                                  chela_dtype_t alpha_dtype, cudaStream_t stream);
+
 }  // namespace chela

@@ -85,8 +85,9 @@ __global__ void conv_transpose_kernel(const T *__restrict__ x, const float *__re
 }
 
 // zt[B,D,Ls] fp32 -> z[B,L,D].  Tile: 64 channels x 32 tokens.
+// lo_offset != 0: z is a bf16 pair; the low plane (z + lo_offset) receives round(value - high part).
 template <typename T>
-__global__ void transpose_out_kernel(const float *__restrict__ zt, T *__restrict__ z, int L, int D, int Ls)
+__global__ void transpose_out_kernel(const float *__restrict__ zt, T *__restrict__ z, int L, int D, int Ls, size_t lo_offset)
 {
     __shared__ float tile[64][33];
     const int b = blockIdx.z, t0 = blockIdx.x * 32, c0 = blockIdx.y * 64;
@@ -100,7 +101,12 @@ __global__ void transpose_out_kernel(const float *__restrict__ zt, T *__restrict
         const int t = t0 + tt;
         if (t >= L) continue;
         for (int cc = lane; cc < 64; cc += 32)
-            if (c0 + cc < D) store1(z + ((size_t)b * L + t) * D + c0 + cc, tile[cc][tt]);
+            if (c0 + cc < D) {
+                const size_t idx = ((size_t)b * L + t) * D + c0 + cc;
+                const float val = tile[cc][tt];
+                store1(z + idx, val);
+                if (lo_offset) store1(z + lo_offset + idx, val - load1(z + idx));
+            }
     }
 }
 
@@ -344,10 +350,11 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
     fft_conv_kernel<1><<<B * D, threads, smem, stream>>>(at, p.Ls, L, D, p.M, p.logM, tw, spec);
 
     dim3 g2((L + 31) / 32, (D + 63) / 64, B);
-    if (out_dtype == CHELA_BF16)
-        transpose_out_kernel<__nv_bfloat16><<<g2, 256, 0, stream>>>(at, (__nv_bfloat16 *)z, L, D, p.Ls);
+    if (out_dtype == CHELA_BF16 || out_dtype == CHELA_BF16_PAIR)
+        transpose_out_kernel<__nv_bfloat16><<<g2, 256, 0, stream>>>(at, (__nv_bfloat16 *)z, L, D, p.Ls,
+                                                                    out_dtype == CHELA_BF16_PAIR ? (size_t)B * L * D : 0);
     else
-        transpose_out_kernel<float><<<g2, 256, 0, stream>>>(at, (float *)z, L, D, p.Ls);
+        transpose_out_kernel<float><<<g2, 256, 0, stream>>>(at, (float *)z, L, D, p.Ls, 0);
     return last_launch_status();
 }
 

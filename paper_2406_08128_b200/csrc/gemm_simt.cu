@@ -81,7 +81,35 @@ __global__ void affine_kernel(const float *__restrict__ z, const TW *__restrict_
     }
 }
 
+// bf16-pair version: z, y are [2][n] bf16 (high plane, low plane)
+template <typename TW>
+__global__ void affine_pair_kernel(const __nv_bfloat16 *__restrict__ z, const TW *__restrict__ alpha,
+                                   const float *__restrict__ beta, __nv_bfloat16 *__restrict__ y, size_t n, int D)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % D);
+        const float v = fmaf(load1(alpha + c), __bfloat162float(z[i]) + __bfloat162float(z[n + i]), beta ? beta[c] : 0.f);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+        y[i] = hi;
+        y[n + i] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
+}
+
 }  // namespace
+
+chela_status_t launch_affine_pair(const void *z, const void *alpha, const float *beta, void *y, size_t M, int D,
+                                  chela_dtype_t alpha_dtype, cudaStream_t stream)
+{
+    const size_t n = M * D;
+    const int blocks = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
+    if (alpha_dtype == CHELA_BF16)
+        affine_pair_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>((const __nv_bfloat16 *)z, (const __nv_bfloat16 *)alpha, beta,
+                                                                      (__nv_bfloat16 *)y, n, D);
+    else
+        affine_pair_kernel<float><<<blocks, 256, 0, stream>>>((const __nv_bfloat16 *)z, (const float *)alpha, beta,
+                                                              (__nv_bfloat16 *)y, n, D);
+    return last_launch_status();
+}
 
 chela_status_t launch_gemm_simt(const void *a, const void *w, const float *bias, void *y, size_t M, int K,
                                 int N, int act, chela_dtype_t a_dtype, chela_dtype_t w_dtype,
