@@ -128,76 +128,181 @@ __device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(
 __device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
 __device__ __forceinline__ float2 cconj(float2 a) { return make_float2(a.x, -a.y); }
 
-// Forward M-point FFT in shared memory, decimation in frequency: natural order in, bit-reversed
-// order out.  tw[j] = exp(-2 pi i j / (2M)), so exp(-2 pi i k / len) = tw[k * (2M / len)].
-__device__ void fft_forward_dif(float2 *s, const float2 *__restrict__ tw, int M, int logM)
+// ---- in-shared-memory FFT: up to four radix-2 stages fused per pass in registers ---------------------
+//
+// Element e of the M-point array lives at phys(e): 16-byte chunks (two complex values) are XOR-swizzled
+// inside groups of eight, so both access patterns of the passes are free of bank conflicts: lanes
+// reading consecutive elements, and lanes reading 16 consecutive elements each (the contiguous pass).
+__device__ __forceinline__ int phys(int e)
 {
-    int len = M, st = 2;  // st = 2M / len
-    int stages = logM;
-    for (; stages >= 2; stages -= 2, len >>= 2, st <<= 2) {
-        const int quarter = len >> 2;
-        for (int g = threadIdx.x; g < (M >> 2); g += blockDim.x) {
-            const int k = g & (quarter - 1);
-            const int i0 = ((g - k) << 2) + k;
-            float2 a = s[i0], b = s[i0 + quarter], c = s[i0 + 2 * quarter], d = s[i0 + 3 * quarter];
-            // stage "len": pairs (a,c) twiddle k, (b,d) twiddle k + quarter
-            float2 a1 = cadd(a, c), c1 = cmul(csub(a, c), tw[k * st]);
-            float2 b1 = cadd(b, d), d1 = cmul(csub(b, d), tw[(k + quarter) * st]);
-            // stage "len/2": pairs (a1,b1) and (c1,d1), both twiddle k (at stride 2*st)
-            const float2 w2 = tw[k * 2 * st];
-            s[i0] = cadd(a1, b1);
-            s[i0 + quarter] = cmul(csub(a1, b1), w2);
-            s[i0 + 2 * quarter] = cadd(c1, d1);
-            s[i0 + 3 * quarter] = cmul(csub(c1, d1), w2);
-        }
-        __syncthreads();
-    }
-    if (stages == 1) {  // len == 2
-        for (int g = threadIdx.x; g < (M >> 1); g += blockDim.x) {
-            float2 a = s[2 * g], b = s[2 * g + 1];
-            s[2 * g] = cadd(a, b);
-            s[2 * g + 1] = csub(a, b);
-        }
-        __syncthreads();
+    const int c = e >> 1;
+    return ((c ^ ((c >> 3) & 7)) << 1) | (e & 1);
+}
+
+// exp(-2 pi i m / 16), m = 0..7
+__device__ __forceinline__ float2 root16(int m)
+{
+    switch (m) {
+        case 0: return make_float2(1.f, 0.f);
+        case 1: return make_float2(0.92387953251128674f, -0.38268343236508977f);
+        case 2: return make_float2(0.70710678118654752f, -0.70710678118654752f);
+        case 3: return make_float2(0.38268343236508977f, -0.92387953251128674f);
+        case 4: return make_float2(0.f, -1.f);
+        case 5: return make_float2(-0.38268343236508977f, -0.92387953251128674f);
+        case 6: return make_float2(-0.70710678118654752f, -0.70710678118654752f);
+        default: return make_float2(-0.92387953251128674f, -0.38268343236508977f);
     }
 }
 
-// Inverse (unscaled) M-point FFT, decimation in time: bit-reversed order in, natural order out.
-__device__ void fft_inverse_dit(float2 *s, const float2 *__restrict__ tw, int M, int logM)
+// Two-level twiddle table in shared memory: exp(-2 pi i j / 2M) = T1[j & 127] * T2[j >> 7], j < M.
+struct Twiddles {
+    const float2 *t1, *t2;
+    __device__ __forceinline__ float2 operator()(int j) const { return cmul(t1[j & 127], t2[j >> 7]); }
+};
+
+// One decimation-in-frequency pass: R radix-2 stages of sub-lengths len, len/2, ..., fused on the 2^R
+// elements i0 + j * (len >> R) that they keep among themselves.  In place; after all passes element
+// of frequency f sits at the bit-reversed position.
+template <int R, bool kContiguous>
+__device__ __forceinline__ void dif_pass(float2 *s, const Twiddles &tw, int M, int len)
 {
-    int len = 2;
-    int stages = logM;
-    if (stages & 1) {
-        for (int g = threadIdx.x; g < (M >> 1); g += blockDim.x) {
-            float2 a = s[2 * g], b = s[2 * g + 1];
-            s[2 * g] = cadd(a, b);
-            s[2 * g + 1] = csub(a, b);
+    constexpr int G = 1 << R;
+    const int q = len >> R, tws = (2 * M) / len;
+    for (int g = threadIdx.x; g < (M >> R); g += blockDim.x) {
+        const int k = g & (q - 1);
+        const int i0 = ((g - k) << R) + k;
+        float2 v[G];
+        if (kContiguous) {   // q == 1, G == 16: eight 16-byte chunks per thread
+#pragma unroll
+            for (int c = 0; c < G / 2; ++c) {
+                const float4 t = *reinterpret_cast<const float4 *>(s + phys(i0 + 2 * c));
+                v[2 * c] = make_float2(t.x, t.y);
+                v[2 * c + 1] = make_float2(t.z, t.w);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < G; ++j) v[j] = s[phys(i0 + j * q)];
         }
-        __syncthreads();
-        len = 4;
-        --stages;
+#pragma unroll
+        for (int st = 0; st < R; ++st) {
+            const int h = G >> (st + 1);
+            // W_len^(k 2^st): base twiddle of this stage; the rest of the exponent is a 16th root of unity
+            const float2 wb = kContiguous ? make_float2(1.f, 0.f) : tw((k << st) * tws);
+#pragma unroll
+            for (int blk = 0; blk < (1 << st); ++blk)
+#pragma unroll
+                for (int jj = 0; jj < h; ++jj) {
+                    const int ia = blk * 2 * h + jj, ib = ia + h;
+                    const float2 a = v[ia], b = v[ib];
+                    v[ia] = cadd(a, b);
+                    const float2 w = (jj == 0) ? wb : (kContiguous ? root16((jj << st) * (16 / G)) : cmul(wb, root16((jj << st) * (16 / G))));
+                    v[ib] = (kContiguous && jj == 0) ? csub(a, b) : cmul(csub(a, b), w);
+                }
+        }
+        if (kContiguous) {
+#pragma unroll
+            for (int c = 0; c < G / 2; ++c)
+                *reinterpret_cast<float4 *>(s + phys(i0 + 2 * c)) = make_float4(v[2 * c].x, v[2 * c].y, v[2 * c + 1].x, v[2 * c + 1].y);
+        } else {
+#pragma unroll
+            for (int j = 0; j < G; ++j) s[phys(i0 + j * q)] = v[j];
+        }
     }
-    // fused pairs of stages: first "len", then "2*len"
-    for (; stages >= 2; stages -= 2, len <<= 2) {
-        const int half = len >> 1;          // butterfly span of the first stage
-        const int st1 = (2 * M) / len;      // twiddle stride of the first stage
-        const int st2 = st1 >> 1;           // of the second stage (length 2*len)
-        for (int g = threadIdx.x; g < (M >> 2); g += blockDim.x) {
-            const int k = g & (half - 1);
-            const int i0 = ((g - k) << 2) + k;
-            float2 a = s[i0], b = s[i0 + half], c = s[i0 + 2 * half], d = s[i0 + 3 * half];
-            // first stage (length len): pairs (a,b) and (c,d), twiddle conj(w_len^k)
-            const float2 w1 = tw[k * st1];
-            const float2 bt = cmulc(b, w1), dt = cmulc(d, w1);
-            const float2 a1 = cadd(a, bt), b1 = csub(a, bt), c1 = cadd(c, dt), d1 = csub(c, dt);
-            // second stage (length 2*len): pairs (a1,c1) twiddle k, (b1,d1) twiddle k + half
-            const float2 ct = cmulc(c1, tw[k * st2]), dtt = cmulc(d1, tw[(k + half) * st2]);
-            s[i0] = cadd(a1, ct);
-            s[i0 + 2 * half] = csub(a1, ct);
-            s[i0 + half] = cadd(b1, dtt);
-            s[i0 + 3 * half] = csub(b1, dtt);
+    __syncthreads();
+}
+
+// One decimation-in-time pass of the inverse transform: R stages of sub-lengths len0, 2 len0, ..., on the
+// 2^R elements i0 + j * (len0 / 2).  Consumes the bit-reversed order the forward passes leave.
+template <int R, bool kContiguous>
+__device__ __forceinline__ void dit_pass(float2 *s, const Twiddles &tw, int M, int len0)
+{
+    constexpr int G = 1 << R;
+    const int h0 = len0 >> 1;
+    for (int g = threadIdx.x; g < (M >> R); g += blockDim.x) {
+        const int k = g & (h0 - 1);
+        const int i0 = ((g - k) << R) + k;
+        float2 v[G];
+        if (kContiguous) {   // len0 == 2, G == 16
+#pragma unroll
+            for (int c = 0; c < G / 2; ++c) {
+                const float4 t = *reinterpret_cast<const float4 *>(s + phys(i0 + 2 * c));
+                v[2 * c] = make_float2(t.x, t.y);
+                v[2 * c + 1] = make_float2(t.z, t.w);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < G; ++j) v[j] = s[phys(i0 + j * h0)];
         }
-        __syncthreads();
+#pragma unroll
+        for (int st = 0; st < R; ++st) {
+            const int d = 1 << st;
+            const float2 wb = kContiguous ? make_float2(1.f, 0.f) : tw(k * ((2 * M) / (len0 << st)));
+#pragma unroll
+            for (int j = 0; j < G; ++j) {
+                if (j & d) continue;
+                const int jj = j & (d - 1);
+                const float2 a = v[j];
+                float2 bt;
+                if (kContiguous && jj == 0) bt = v[j + d];
+                else {
+                    const float2 w = (jj == 0) ? wb : (kContiguous ? root16(jj * (16 >> (st + 1))) : cmul(wb, root16(jj * (16 >> (st + 1)))));
+                    bt = cmulc(v[j + d], w);
+                }
+                v[j] = cadd(a, bt);
+                v[j + d] = csub(a, bt);
+            }
+        }
+        if (kContiguous) {
+#pragma unroll
+            for (int c = 0; c < G / 2; ++c)
+                *reinterpret_cast<float4 *>(s + phys(i0 + 2 * c)) = make_float4(v[2 * c].x, v[2 * c].y, v[2 * c + 1].x, v[2 * c + 1].y);
+        } else {
+#pragma unroll
+            for (int j = 0; j < G; ++j) s[phys(i0 + j * h0)] = v[j];
+        }
+    }
+    __syncthreads();
+}
+
+template <bool kForward>
+__device__ __forceinline__ void pass_r(int R, float2 *s, const Twiddles &tw, int M, int len)
+{
+    if (kForward) {
+        if (R == 1) dif_pass<1, false>(s, tw, M, len);
+        else if (R == 2) dif_pass<2, false>(s, tw, M, len);
+        else if (R == 3) dif_pass<3, false>(s, tw, M, len);
+        else dif_pass<4, false>(s, tw, M, len);
+    } else {
+        if (R == 1) dit_pass<1, false>(s, tw, M, len);
+        else if (R == 2) dit_pass<2, false>(s, tw, M, len);
+        else if (R == 3) dit_pass<3, false>(s, tw, M, len);
+        else dit_pass<4, false>(s, tw, M, len);
+    }
+}
+
+// Forward M-point FFT (M >= 16): natural order in, bit-reversed order out.  Stages are grouped
+// r0, 4, 4, ..., 4 with r0 = logM mod 4 (4 if that is 0); the last pass works on 16 contiguous elements.
+__device__ void fft_forward_dif(float2 *s, const Twiddles &tw, int M, int logM)
+{
+    const int r0 = ((logM - 1) & 3) + 1;
+    int len = M;
+    if (logM > 4) {
+        pass_r<true>(r0, s, tw, M, len);
+        len >>= r0;
+        for (; len > 16; len >>= 4) dif_pass<4, false>(s, tw, M, len);
+    }
+    dif_pass<4, true>(s, tw, M, 16);
+}
+
+// Inverse (unscaled) M-point FFT: bit-reversed order in, natural order out (mirror of the forward passes).
+__device__ void fft_inverse_dit(float2 *s, const Twiddles &tw, int M, int logM)
+{
+    const int r0 = ((logM - 1) & 3) + 1;
+    dit_pass<4, true>(s, tw, M, 2);
+    if (logM > 4) {
+        int len0 = 32;
+        for (; (len0 << 3) <= (M >> r0); len0 <<= 4) dit_pass<4, false>(s, tw, M, len0);
+        pass_r<false>(r0, s, tw, M, len0);
     }
 }
 
@@ -207,10 +312,16 @@ __device__ __forceinline__ int bitrev(int f, int logM) { return (int)(__brev((un
 // mode 1: rows = sequences at[B*D][Ls]; multiplies with spec[row % D] and writes the causal
 //         convolution back over the row.
 template <int MODE>
-__global__ void fft_conv_kernel(float *__restrict__ rows, int row_stride, int L, int D, int M, int logM,
-                                const float2 *__restrict__ tw, float2 *__restrict__ spec)
+__global__ void __launch_bounds__(512) fft_conv_kernel(float *__restrict__ rows, int row_stride, int L, int D, int M, int logM,
+                                const float2 *__restrict__ tw_global, float2 *__restrict__ spec)
 {
-    extern __shared__ __align__(16) float2 s[];
+    extern __shared__ __align__(16) float2 s[];   // M data points (swizzled), then the two twiddle tables
+    float2 *t1 = s + M, *t2 = t1 + 128;
+    for (int j = threadIdx.x; j < 128; j += blockDim.x) {
+        t1[j] = (j < M) ? tw_global[j] : make_float2(1.f, 0.f);
+        t2[j] = (128 * j < M) ? tw_global[128 * j] : make_float2(1.f, 0.f);
+    }
+    const Twiddles tw = {t1, t2};
     const int row = blockIdx.x;
     float *x = rows + (size_t)row * row_stride;
     // pack: s[n] = x[2n] + i x[2n+1], zero beyond L
@@ -226,7 +337,7 @@ __global__ void fft_conv_kernel(float *__restrict__ rows, int row_stride, int L,
             if (t < L) re = x[t];
             if (t + 1 < L) im = x[t + 1];
         }
-        s[n] = make_float2(re, im);
+        s[phys(n)] = make_float2(re, im);
     }
     __syncthreads();
     fft_forward_dif(s, tw, M, logM);
@@ -236,10 +347,11 @@ __global__ void fft_conv_kernel(float *__restrict__ rows, int row_stride, int L,
     float2 *kspec = spec + (size_t)(MODE == 1 ? row % D : row) * (M + 1);
     for (int f = threadIdx.x; f <= (M >> 1); f += blockDim.x) {
         const int pf = bitrev(f, logM), pm = bitrev((M - f) & (M - 1), logM);
-        const float2 Cf = s[pf], Cm = s[pm];
+        const float2 Cf = s[phys(pf)], Cm = s[phys(pm)];
         const float2 E = make_float2(0.5f * (Cf.x + Cm.x), 0.5f * (Cf.y - Cm.y));
         const float2 O = make_float2(0.5f * (Cf.y + Cm.y), -0.5f * (Cf.x - Cm.x));
-        const float2 wO = cmul(tw[f], O);
+        const float2 wf = tw(f);
+        const float2 wO = cmul(wf, O);
         float2 Xf = cadd(E, wO), Xm = cconj(csub(E, wO));
         if (MODE == 0) {
             if (f == 0) {
@@ -263,9 +375,9 @@ __global__ void fft_conv_kernel(float *__restrict__ rows, int row_stride, int L,
             }
             const float2 Ep = make_float2(0.5f * (Yf.x + Ym.x), 0.5f * (Yf.y - Ym.y));
             const float2 Dp = make_float2(0.5f * (Yf.x - Ym.x), 0.5f * (Yf.y + Ym.y));
-            const float2 Op = cmulc(Dp, tw[f]);
-            s[pf] = make_float2(Ep.x - Op.y, Ep.y + Op.x);          // E' + i O'
-            if (pm != pf) s[pm] = make_float2(Ep.x + Op.y, -Ep.y + Op.x);  // conj(E') + i conj(O')
+            const float2 Op = cmulc(Dp, wf);
+            s[phys(pf)] = make_float2(Ep.x - Op.y, Ep.y + Op.x);          // E' + i O'
+            if (pm != pf) s[phys(pm)] = make_float2(Ep.x + Op.y, -Ep.y + Op.x);  // conj(E') + i conj(O')
         }
     }
     if (MODE == 0) return;
@@ -274,7 +386,7 @@ __global__ void fft_conv_kernel(float *__restrict__ rows, int row_stride, int L,
     const float inv = 1.0f / (float)M;
     for (int n = threadIdx.x; 2 * n < row_stride; n += blockDim.x) {
         const int t = 2 * n;
-        float2 p = (n < M) ? s[n] : make_float2(0.f, 0.f);
+        float2 p = (n < M) ? s[phys(n)] : make_float2(0.f, 0.f);
         p.x = (t < L) ? p.x * inv : 0.f;
         p.y = (t + 1 < L) ? p.y * inv : 0.f;
         *reinterpret_cast<float2 *>(x + t) = p;
@@ -339,9 +451,9 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
         conv_transpose_kernel<float><<<g1, 256, 0, stream>>>((const float *)x, w_short, short_width, at, L, D, p.Ls);
     twiddle_kernel<<<(p.M + 255) / 256, 256, 0, stream>>>(tw, p.M);
 
-    const size_t smem = (size_t)p.M * sizeof(float2);
-    int threads = p.M / 4;
-    threads = threads < 32 ? 32 : (threads > 1024 ? 1024 : threads);
+    const size_t smem = (size_t)(p.M + 256) * sizeof(float2);
+    int threads = p.M / 16;
+    threads = threads < 32 ? 32 : (threads > 512 ? 512 : threads);
     cudaError_t e = cudaFuncSetAttribute(fft_conv_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(fft_conv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
