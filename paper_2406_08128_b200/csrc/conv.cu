@@ -312,7 +312,7 @@ __device__ __forceinline__ int bitrev(int f, int logM) { return (int)(__brev((un
 // mode 1: rows = sequences at[B*D][Ls]; multiplies with spec[row % D] and writes the causal
 //         convolution back over the row.
 template <int MODE>
-__global__ void __launch_bounds__(512) fft_conv_kernel(float *__restrict__ rows, int row_stride, int L, int D, int M, int logM,
+__global__ void __launch_bounds__(1024) fft_conv_kernel(float *__restrict__ rows, int row_stride, int L, int D, int M, int logM,
                                 const float2 *__restrict__ tw_global, float2 *__restrict__ spec)
 {
     extern __shared__ __align__(16) float2 s[];   // M data points (swizzled), then the two twiddle tables
@@ -344,9 +344,14 @@ __global__ void __launch_bounds__(512) fft_conv_kernel(float *__restrict__ rows,
     // C[f] sits at s[bitrev(f)].  Spectrum of the real length-2M sequence:
     //   E = (C[f] + conj C[M-f]) / 2, O = -i (C[f] - conj C[M-f]) / 2,
     //   X[f] = E + w^f O,  X[M-f] = conj(E - w^f O),  w = exp(-2 pi i / 2M); X[M] = E[0] - O[0].
+    // The kernel spectrum is kept in the same bit-reversed order as the data (entry p holds K[bitrev(p)];
+    // entry M holds the Nyquist term), and the loop runs over positions p rather than frequencies: lanes
+    // then touch consecutive shared-memory and global addresses instead of one bank.
     float2 *kspec = spec + (size_t)(MODE == 1 ? row % D : row) * (M + 1);
-    for (int f = threadIdx.x; f <= (M >> 1); f += blockDim.x) {
-        const int pf = bitrev(f, logM), pm = bitrev((M - f) & (M - 1), logM);
+    for (int pf = threadIdx.x; pf < M; pf += blockDim.x) {
+        const int f = bitrev(pf, logM);
+        if (f > (M >> 1)) continue;   // the pair (f, M-f) is handled by its smaller member
+        const int pm = bitrev((M - f) & (M - 1), logM);
         const float2 Cf = s[phys(pf)], Cm = s[phys(pm)];
         const float2 E = make_float2(0.5f * (Cf.x + Cm.x), 0.5f * (Cf.y - Cm.y));
         const float2 O = make_float2(0.5f * (Cf.y + Cm.y), -0.5f * (Cf.x - Cm.x));
@@ -358,8 +363,8 @@ __global__ void __launch_bounds__(512) fft_conv_kernel(float *__restrict__ rows,
                 kspec[0] = make_float2(E.x + O.x, 0.f);
                 kspec[M] = make_float2(E.x - O.x, 0.f);
             } else {
-                kspec[f] = Xf;
-                kspec[M - f] = Xm;
+                kspec[pf] = Xf;
+                kspec[pm] = Xm;
             }
         } else {
             // Y = X K, then the packed spectrum of y: C'[f] = E' + i O',
@@ -370,8 +375,8 @@ __global__ void __launch_bounds__(512) fft_conv_kernel(float *__restrict__ rows,
                 Yf = make_float2((E.x + O.x) * kspec[0].x, 0.f);
                 Ym = make_float2((E.x - O.x) * kspec[M].x, 0.f);
             } else {
-                Yf = cmul(Xf, kspec[f]);
-                Ym = cmul(Xm, kspec[M - f]);
+                Yf = cmul(Xf, kspec[pf]);
+                Ym = cmul(Xm, kspec[pm]);
             }
             const float2 Ep = make_float2(0.5f * (Yf.x + Ym.x), 0.5f * (Yf.y - Ym.y));
             const float2 Dp = make_float2(0.5f * (Yf.x - Ym.x), 0.5f * (Yf.y + Ym.y));
@@ -453,7 +458,7 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
 
     const size_t smem = (size_t)(p.M + 256) * sizeof(float2);
     int threads = p.M / 16;
-    threads = threads < 32 ? 32 : (threads > 512 ? 512 : threads);
+    threads = threads < 32 ? 32 : (threads > 1024 ? 1024 : threads);
     cudaError_t e = cudaFuncSetAttribute(fft_conv_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(fft_conv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
