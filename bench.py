@@ -332,6 +332,28 @@ def main():
         if chela.async_status(ws) != chela.OK:
             raise RuntimeError("device-side wait timed out in the extras")
         del sets
+        # ---- token mixer forward (configs 3 and 4): short conv + SiLU, long conv, Q/K/V, attention --------
+        # roofline: bf16 tensor peak over the algorithmic flops (3 dense projections + the attention tiles)
+        mixers = []
+        for (mb, ml, md, mh, mc) in ((4, 16384, 512, 8, 64), (8, 8192, 1024, 8, 128)):
+            x = torch.randn(mb, ml, md, device=dev, generator=gen).to(torch.bfloat16)
+            w_s = torch.randn(md, 3, device=dev, generator=gen) / 3 ** 0.5
+            k_l = torch.randn(md, ml, device=dev, generator=gen) * torch.exp(-0.001 * torch.arange(ml, device=dev))[None, :]
+            w_q, w_k, w_v = [(torch.randn(md, md, device=dev, generator=gen) / md ** 0.5).to(torch.bfloat16) for _ in range(3)]
+            mws = torch.zeros(chela.mixer_workspace_bytes(mb, ml, md, mh, mc), dtype=torch.uint8, device=dev)
+            mo = torch.empty(mb, ml, md, device=dev)
+            ms = timed(lambda: chela.mixer_fwd(x, w_s, k_l, w_q, w_k, w_v, mh, chunk=mc, out=mo, workspace=mws), 5, warm=2)
+            if chela.async_status(mws) != chela.OK:
+                raise RuntimeError("device-side wait timed out in the mixer")
+            d_head = md // mh
+            flops_tok = 3 * 2 * md * md + mh * (4 * mc * d_head + 4 * d_head * d_head)
+            mixers.append({"B": mb, "L": ml, "D": md, "H": mh, "chunk": mc, "ms": ms,
+                           "tokens_per_s": mb * ml / (ms * 1e-3),
+                           "tensor_frac": flops_tok * mb * ml / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                           "attention_kernel_kind": chela.linattn_kernel_kind(mb, mh, ml, d_head, d_head, mc,
+                                                                              chela.BF16_PAIR if d_head == 64 else chela.F32)})
+            del x, k_l, mws, mo
+        line["mixer"] = mixers
         # ---- CPU oracle on the host cores, bounded sample -----------------------------------------------
         import oracle
         oracle.build()

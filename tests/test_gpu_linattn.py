@@ -125,3 +125,24 @@ def test_workspace_too_small_is_rejected():
     with pytest.raises(chela.ChelaError) as e:
         chela.linattn_fwd(q, k, v, workspace=ws)
     assert e.value.status == chela.ERR_WORKSPACE
+
+
+def _pair(a):
+    import torch
+    hi = inputs.round_bf16(a.astype(np.float32))
+    lo = inputs.round_bf16((a.astype(np.float64) - hi).astype(np.float32))
+    return torch.stack([to_device(hi, "bf16"), to_device(lo, "bf16")]).contiguous(), hi.astype(np.float64) + lo
+
+
+@pytest.mark.parametrize("B,L,H", [(1, 64, 1), (1, 200, 2), (2, 1000, 3), (1, 8192, 2), (3, 4096, 8)])
+@pytest.mark.parametrize("norm", [True, False])
+def test_bf16_pair_inputs_reach_fp32_like_accuracy(B, L, H, norm):
+    """Q, K, V as bf16 pairs (hi + lo planes): three-term tensor-core products, error far below the
+    single-bf16 bound (this is the mixer's attention path)."""
+    rng = np.random.default_rng(B + L + H)
+    q, k, v = (rng.standard_normal((B, L, H, 64), dtype=np.float32) * 2 for _ in range(3))
+    (qd, qv), (kd, kv), (vd, vv) = _pair(q), _pair(k), _pair(v)
+    assert chela.linattn_kernel_kind(B, H, L, 64, 64, 64, chela.BF16_PAIR, chela.F32) == 2
+    o = chela.linattn_fwd(qd, kd, vd, chunk=64, norm=chela.NORM_RMS if norm else chela.NORM_NONE, in_dtype=chela.BF16_PAIR)
+    ref = oracle.linattn_recurrent(qv, kv, vv, norm=norm)
+    assert rel_err(to_numpy(o), ref) <= 5e-4
