@@ -181,7 +181,7 @@ chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_wi
     // Tensor-core path: every intermediate (Z, Q, K, V) is a bf16 pair (hi + lo, about 16 mantissa bits) and
     // every product takes three tensor-core terms; single bf16 intermediates would cost the normalised
     // output its leading digits (cancellation in Q K^T on rows with a small pre-norm RMS).
-    const bool tensor_path = in_dtype == CHELA_BF16 && d == 64 &&
+    const bool tensor_path = in_dtype == CHELA_BF16 && (d == 64 || d == 128) &&
                              gemm_sm100_supported(M, D, D, CHELA_BF16_PAIR, CHELA_BF16, CHELA_BF16_PAIR);
     chela_status_t st;
     if (tensor_path) {

@@ -607,13 +607,14 @@ bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_
 {
     (void)B; (void)H; (void)L;
     return (in_dtype == CHELA_BF16 || in_dtype == CHELA_BF16_PAIR) && (out_dtype == CHELA_F32 || out_dtype == CHELA_BF16) &&
-           d == kD && (chunk == 64 || chunk == 128);
+           (d == kD || d == 128) && (chunk == 64 || chunk == 128);
 }
 
 // Header (word 0 = asynchronous status of the last launch that used this workspace) followed by the
 // per-group state sums [B*H][G-1][64][64] fp32 of a call that is split along L.
 size_t linattn_sm100_workspace_bytes(int B, int H, int L, int d, int)
 {
+    if (d == 128) return kWsHeader;   // the 128-wide kernel does not split sequences
     if (d != kD) return 0;
     const size_t a = split_plan(B, H, L, false).part_bytes, b = split_plan(B, H, L, true).part_bytes;
     return kWsHeader + (a > b ? a : b);   // the query does not know the input dtype: cover both plans
@@ -623,7 +624,7 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
                                     int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps,
                                     float scale, void *workspace, cudaStream_t stream)
 {
-    (void)d;
+    if (d == 128) return launch_linattn_sm100_d128(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, workspace, stream);
     // The result does not depend on the chunk size: both supported values run on 64-token tiles.
     (void)chunk;
     if (in_dtype == CHELA_BF16_PAIR) {

@@ -1,0 +1,386 @@
+// Chunked causal linear attention on sm_100a for head dimension 128 (d_k = d_v = 128): the same
+// tcgen05 / TMEM / TMA scheme as the 64-wide kernel, with N = 128 instructions (64 cycles each, the
+// tensor core's full rate) wherever d_v is the N dimension.
+//
+// One CTA (issuer warp + 4 compute warps) walks one (batch, head) sequence in tiles of 64 tokens.  Per tile
+// and per input plane the TMA ring holds six [64 rows] x 128 B tiles: Q_a, K_a, Q_b, K_b (the two halves of
+// d_k, Q and K of a half adjacent) and V_a, V_b (the two halves of d_v, adjacent).
+//   G1 : PT   = [Q_a;K_a] Q_a^T + [Q_b;K_b] Q_b^T         rows 64..127 = P^T = K Q^T           (N = 64)
+//   G2 : OS_a rows 0..63 = sum_x [Q_x;K_x] (S_x,hi + S_x,lo)   lanes 64..127 write-disabled     (N = 128)
+//   G3 : OS_a += [P^T | K_a]^T [V_a|V_b]   rows 0..63 += P V, rows 64..127 += K_a^T V (state rows d_k < 64)
+//        S_b  += [P^T | K_b]^T [V_a|V_b]   lanes 0..63 write-disabled: state rows d_k >= 64      (N = 128)
+// TMEM: OS_a 128 columns, S_b 128 columns, PT 64 columns.  The fp32 state (128 x 128) never leaves the SM;
+// it is fed back as bf16 hi + lo tiles.  With bf16-pair inputs every product takes three terms
+// (hi*hi + hi*lo + lo*hi) and the score tile is kept as a pair (the mixer's fp32-like path).
+// Sequences are not split along L here (one CTA per (batch, head)).
+// Every wait is bounded; a timeout records CHELA_ERR_TIMEOUT, drains outstanding loads, frees TMEM.
+#include "sm100_ptx.cuh"
+
+namespace chela {
+namespace {
+
+using namespace sm100;
+
+constexpr int kD = 128;
+constexpr int kC = 64;
+constexpr int kThreads = 160;
+constexpr int kTile = kC * 128;
+
+template <typename TOut, bool kPair>
+struct Smem {
+    static constexpr int kStages = kPair ? 1 : 2;
+    static constexpr int kPlanes = kPair ? 2 : 1;
+    static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;
+    static constexpr int offPT = 0;                                   // score tile (hi, lo)
+    static constexpr int offS = offPT + kPlanes * kTile;              // S_a hi, S_b hi, S_a lo, S_b lo: 2 tiles each
+    static constexpr int offO = offS + 8 * kTile;
+    static constexpr int offStage = offO + kOBoxes * kTile;           // per stage and plane: Qa Ka Qb Kb Va Vb
+    static constexpr int offBar = offStage + kStages * kPlanes * 6 * kTile;   // full[kStages], p, o, pt, s
+    static constexpr int offTmem = offBar + 8 * (kStages + 4);
+    static constexpr int offAbort = offTmem + 8;
+    static constexpr int bytes = offAbort + 8;
+};
+constexpr int kTmemCols = 512;
+constexpr int kColOS = 0, kColSb = 128, kColPT = 256;
+
+template <typename TOut, bool kPair>
+__global__ void __launch_bounds__(kThreads)
+linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                          const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
+                          float scale, int norm, float eps, int *__restrict__ status)
+{
+    using SM = Smem<TOut, kPair>;
+    constexpr int kStages = SM::kStages, kPlanes = SM::kPlanes;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {
+        if (threadIdx.x == 0) atomicExch(status, (int)CHELA_ERR_CUDA);
+        return;
+    }
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.x / H, h = blockIdx.x % H;
+    const int nchunks = (L + kC - 1) / kC;
+
+    const uint32_t bar_full0 = sbase + SM::offBar;
+    const uint32_t bar_p = bar_full0 + 8 * kStages, bar_o = bar_p + 8, bar_pt = bar_o + 8, bar_s = bar_pt + 8;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(bar_full0 + 8 * s, 1);
+        mbar_init(bar_p, 1);
+        mbar_init(bar_o, 1);
+        mbar_init(bar_pt, 2);
+        mbar_init(bar_s, 4);
+        *abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_o);
+    }
+    if (warp == 0) {
+        tmem_alloc(sbase + SM::offTmem, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            // tile t (0 Qa, 1 Ka, 2 Qb, 3 Kb, 4 Va, 5 Vb) of plane pl of the stage of `chunk`
+            auto tile = [&](int chunk, int pl, int t) {
+                return sbase + SM::offStage + (((chunk % kStages) * kPlanes + pl) * 6 + t) * kTile;
+            };
+            auto issue_load = [&](int chunk) {
+                const uint32_t bar = bar_full0 + 8 * (chunk % kStages);
+                mbar_expect_tx(bar, kPlanes * 6 * kTile);
+#pragma unroll
+                for (int pl = 0; pl < kPlanes; ++pl)
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        tma_load_5d(tile(chunk, pl, 2 * x), &tm_q, bar, 64 * x, h, chunk * kC, b, pl);
+                        tma_load_5d(tile(chunk, pl, 2 * x + 1), &tm_k, bar, 64 * x, h, chunk * kC, b, pl);
+                        tma_load_5d(tile(chunk, pl, 4 + x), &tm_v, bar, 64 * x, h, chunk * kC, b, pl);
+                    }
+            };
+            constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);
+            constexpr uint32_t idescG2 = make_idesc(128, 128, 0, 1);
+            constexpr uint32_t idescG3 = make_idesc(128, 128, 1, 1);
+            // G1; false if the chunk's tiles never arrived
+            auto issue_scores = [&](int chunk) -> bool {
+                if (!mbar_wait(bar_full0 + 8 * (chunk % kStages), (chunk / kStages) & 1, abort_flag)) return false;
+                tc_fence_after();
+                uint32_t acc = 0;
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    const uint32_t qk_hi = desc_lo(tile(chunk, 0, 2 * x));
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) { umma_bf16(tmem + kColPT, qk_hi + 2 * k, qk_hi + 2 * k, idescG1, acc); acc = 1; }
+                    if (kPair) {
+                        const uint32_t qk_lo = desc_lo(tile(chunk, 1, 2 * x));
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColPT, qk_hi + 2 * k, qk_lo + 2 * k, idescG1, 1);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColPT, qk_lo + 2 * k, qk_hi + 2 * k, idescG1, 1);
+                    }
+                }
+                umma_commit(bar_p);
+                return true;
+            };
+            int loads_issued = 0, consumed = 0;
+            for (; loads_issued < kStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued);
+            bool ok = issue_scores(0);
+            uint32_t par_s = 0;
+            for (int i = 0; ok && i < nchunks; ++i) {
+                if (i > 0) {
+                    ok = mbar_wait(bar_s, par_s, abort_flag);
+                    par_s ^= 1;
+                    if (!ok) break;
+                    tc_fence_after();
+                    uint32_t acc = 0;
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        // state tiles of d_k half x: hi at offS + x*2 tiles, lo at offS + (4 + x*2) tiles; two d_v atoms each
+                        const uint32_t s_hi = desc_lo(sbase + SM::offS + (2 * x) * kTile, kTile),
+                                       s_lo = desc_lo(sbase + SM::offS + (4 + 2 * x) * kTile, kTile);
+                        const uint32_t qk_hi = desc_lo(tile(i, 0, 2 * x));
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) { umma_bf16(tmem + kColOS, qk_hi + 2 * k, s_hi + 128 * k, idescG2, acc, 1); acc = 1; }
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColOS, qk_hi + 2 * k, s_lo + 128 * k, idescG2, 1, 1);
+                        if (kPair) {
+                            const uint32_t qk_lo = desc_lo(tile(i, 1, 2 * x));
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, s_hi + 128 * k, idescG2, 1, 1);
+                        }
+                    }
+                }
+                ok = mbar_wait(bar_pt, i & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                {
+                    const uint32_t pt_hi = sbase + SM::offPT, pt_lo = pt_hi + kTile;
+                    const uint32_t v_hi = desc_lo(tile(i, 0, 4), kTile);
+                    // OS_a: [P^T | K_a]; S_b: [P^T | K_b] with the lower lanes write-disabled
+                    const uint32_t a_a = desc_lo(pt_hi, tile(i, 0, 1) - pt_hi), a_b = desc_lo(pt_hi, tile(i, 0, 3) - pt_hi);
+                    const uint32_t first = i > 0 ? 1u : 0u;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColOS, a_a + 128 * k, v_hi + 128 * k, idescG3, (first || k > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColSb, a_b + 128 * k, v_hi + 128 * k, idescG3, (first || k > 0) ? 1u : 0u, 2);
+                    if (kPair) {
+                        const uint32_t v_lo = desc_lo(tile(i, 1, 4), kTile);
+                        const uint32_t a2_a = desc_lo(pt_lo, tile(i, 1, 1) - pt_lo), a2_b = desc_lo(pt_lo, tile(i, 1, 3) - pt_lo);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColOS, a_a + 128 * k, v_lo + 128 * k, idescG3, 1);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColOS, a2_a + 128 * k, v_hi + 128 * k, idescG3, 1);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColSb, a_b + 128 * k, v_lo + 128 * k, idescG3, 1, 2);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColSb, a2_b + 128 * k, v_hi + 128 * k, idescG3, 1, 2);
+                    }
+                    umma_commit(bar_o);
+                }
+                if (kStages > 1 && i + 1 < nchunks) {
+                    ok = issue_scores(i + 1);
+                    if (!ok) break;
+                }
+                ok = mbar_wait(bar_o, i & 1, abort_flag);
+                if (!ok) break;
+                consumed = i + 1;
+                if (i + kStages < nchunks) {
+                    issue_load(i + kStages);
+                    ++loads_issued;
+                }
+                if (kStages == 1 && i + 1 < nchunks) {
+                    ok = issue_scores(i + 1);
+                    if (!ok) break;
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+                for (int c = consumed; c < loads_issued; ++c)
+                    mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1, nullptr);
+            }
+        }
+    } else {
+        const bool upper = warp >= 2;
+        const int r = tid & 63;
+        const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
+        bool ok = true;
+        for (int i = 0; i < nchunks; ++i) {
+            if (upper) {
+                // ---- P^T_i: TMEM -> causal mask (t >= s) -> bf16 (pair) -> shared, rows = s ---------------
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_p, i & 1, abort_flag));
+                if (!ok) break;
+                tc_fence_after();
+                float p[2][32];
+                if (warp == 2) tmem_ld32(tmem_warp + kColPT, p[0]);
+                tmem_ld32(tmem_warp + kColPT + 32, p[1]);
+                tmem_ld_wait();
+                uint8_t *sP = smem + SM::offPT;
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    const bool live = cb == 1 || warp == 2;
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        uint32_t w[4], w2[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int t = cb * 32 + c8 * 8 + e * 2;
+                            const float x0 = (live && t >= r) ? p[cb][c8 * 8 + e * 2] : 0.f;
+                            const float x1 = (live && t + 1 >= r) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
+                            const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                            w[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                            if (kPair) {
+                                const float2 hf = __bfloat1622float2(hh);
+                                w2[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                            }
+                        }
+                        *reinterpret_cast<uint4 *>(sP + sw128(r, cb * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                        if (kPair) *reinterpret_cast<uint4 *>(sP + kTile + sw128(r, cb * 4 + c8)) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+                    }
+                }
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_pt);
+            }
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            if (!upper) {
+                // ---- output row t (128 values): scale, normaliser -> swizzled staging -> TMA store ------------
+                float acc[kD];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld32(tmem_warp + kColOS + 32 * c, *reinterpret_cast<float(*)[32]>(&acc[32 * c]));
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar_s);
+                    bulk_wait_read0();
+                }
+                __syncwarp();
+                float ss = 0.f;
+#pragma unroll
+                for (int j = 0; j < kD; ++j) {
+                    acc[j] *= scale;
+                    ss = fmaf(acc[j], acc[j], ss);
+                }
+                const float inv = norm ? rsqrtf(ss * (1.0f / kD) + eps) : 1.0f;
+                uint8_t *sO = smem + SM::offO;
+                if (sizeof(TOut) == 4) {
+#pragma unroll
+                    for (int j = 0; j < kD; j += 4)
+                        *reinterpret_cast<float4 *>(sO + (j / 32) * kTile + sw128(r, (j % 32) / 4)) =
+                            make_float4(acc[j] * inv, acc[j + 1] * inv, acc[j + 2] * inv, acc[j + 3] * inv);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kD; j += 8)
+                        *reinterpret_cast<uint4 *>(sO + (j / 64) * kTile + sw128(r, (j % 64) / 8)) =
+                            make_uint4(pack_bf16(acc[j] * inv, acc[j + 1] * inv), pack_bf16(acc[j + 2] * inv, acc[j + 3] * inv),
+                                       pack_bf16(acc[j + 4] * inv, acc[j + 5] * inv), pack_bf16(acc[j + 6] * inv, acc[j + 7] * inv));
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+#pragma unroll
+                    for (int bx = 0; bx < SM::kOBoxes; ++bx)
+                        tma_store_5d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
+                                     i * kC + warp * 32, b, 0);
+                    bulk_commit();
+                }
+            } else if (i + 1 < nchunks) {
+                // ---- state rows d_k = r (from OS_a) and d_k = 64 + r (from S_b): bf16 hi + lo -> shared --------
+#pragma unroll
+                for (int x = 0; x < 2; ++x)
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        float sv[64];
+                        const uint32_t col = (x == 0 ? kColOS : kColSb) + 64 * half;
+                        tmem_ld32(tmem_warp + col, *reinterpret_cast<float(*)[32]>(&sv[0]));
+                        tmem_ld32(tmem_warp + col + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+                        tmem_ld_wait();
+                        uint8_t *sHi = smem + SM::offS + (2 * x + half) * kTile, *sLo = sHi + 4 * kTile;
+#pragma unroll
+                        for (int c8 = 0; c8 < 8; ++c8) {
+                            uint32_t wh[4], wl[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float x0 = sv[c8 * 8 + e * 2], x1 = sv[c8 * 8 + e * 2 + 1];
+                                const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                                const float2 hf = __bfloat1622float2(hh);
+                                wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                                wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                            }
+                            const uint32_t off = sw128(r, c8);
+                            *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                            *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                        }
+                    }
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_s);
+            }
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+        }
+        if (!upper && lane == 0) bulk_wait0();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int box_rows, bool f32, int planes)
+{
+    const cuuint64_t es = f32 ? 4 : 2;
+    const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B, (cuuint64_t)planes};
+    const cuuint64_t strides[4] = {(cuuint64_t)kD * es, (cuuint64_t)H * kD * es, (cuuint64_t)L * H * kD * es,
+                                   (cuuint64_t)B * L * H * kD * es};
+    const cuuint32_t box[5] = {(cuuint32_t)(128 / es), 1, (cuuint32_t)box_rows, 1, 1};
+    return make_map_sw128(map, ptr, f32, 5, dims, strides, box);
+}
+
+template <typename TOut, bool kPair>
+chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
+                        float scale, int *status, cudaStream_t stream)
+{
+    CUtensorMap mq, mk, mv, mo;
+    const int planes = kPair ? 2 : 1;
+    if (!make_map(&mq, q, B, H, L, kC, false, planes) || !make_map(&mk, k, B, H, L, kC, false, planes) ||
+        !make_map(&mv, v, B, H, L, kC, false, planes) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4, 1))
+        return CHELA_ERR_CUDA;
+    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+    auto kern = linattn_sm100_d128_kernel<TOut, kPair>;
+    const int smem = Smem<TOut, kPair>::bytes;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
+    kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status);
+    return last_launch_status();
+}
+
+}  // namespace
+
+chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
+                                         chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
+                                         void *workspace, cudaStream_t stream)
+{
+    int *status = (int *)workspace;
+    if (in_dtype == CHELA_BF16_PAIR) {
+        if (out_dtype == CHELA_F32) return launch_t<float, true>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+        return launch_t<__nv_bfloat16, true>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+    }
+    if (out_dtype == CHELA_F32) return launch_t<float, false>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+    return launch_t<__nv_bfloat16, false>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+}
+
+}  // namespace chela

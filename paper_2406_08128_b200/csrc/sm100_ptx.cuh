@@ -152,18 +152,19 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, 
 }
 
 // D[tmem] (+)= A[smem] * B[smem], bf16 operands, fp32 accumulate; issued by a single thread.
-// upper_off != 0 write-disables TMEM lanes 64..127 (rows 64..127 of an M = 128 result).
+// lane_mask: 0 = write all 128 TMEM lanes, 1 = write-disable lanes 64..127 (rows 64..127 of an M = 128
+// result), 2 = write-disable lanes 0..63.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate,
-                                          uint32_t upper_off = 0)
+                                          uint32_t lane_mask = 0)
 {
-    const uint32_t m = upper_off ? 0xFFFFFFFFu : 0u;
+    const uint32_t m_lo = lane_mask == 2 ? 0xFFFFFFFFu : 0u, m_hi = lane_mask == 1 ? 0xFFFFFFFFu : 0u;
     asm volatile(
         "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "mov.b64 da, {%1, %5};\n\t"
         "mov.b64 db, {%2, %5};\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, {%6, %6, %7, %7}, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi), "r"(0u), "r"(m)
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi), "r"(m_lo), "r"(m_hi)
         : "memory");
 }
 

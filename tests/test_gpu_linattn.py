@@ -110,6 +110,8 @@ def test_sequences_split_along_length(B, L, H):
 def test_async_status_is_ok_and_tensor_core_path_is_used():
     import torch
     assert chela.linattn_kernel_kind(2, 2, 256, 64, 64, 64, chela.BF16, chela.F32) == 2
+    assert chela.linattn_kernel_kind(2, 2, 256, 128, 128, 128, chela.BF16, chela.F32) == 2
+    assert chela.linattn_kernel_kind(2, 2, 256, 128, 128, 128, chela.F32, chela.F32) == 1
     assert chela.linattn_kernel_kind(2, 2, 256, 64, 64, 64, chela.F32, chela.F32) == 1
     q, k, v = inputs.qkv(3, 2, 256, 2, 64, 64, "bf16")
     ws = torch.zeros(chela.linattn_workspace_bytes(2, 2, 256, 64, 64, 64), dtype=torch.uint8, device="cuda")
@@ -136,13 +138,14 @@ def _pair(a):
 
 @pytest.mark.parametrize("B,L,H", [(1, 64, 1), (1, 200, 2), (2, 1000, 3), (1, 8192, 2), (3, 4096, 8)])
 @pytest.mark.parametrize("norm", [True, False])
-def test_bf16_pair_inputs_reach_fp32_like_accuracy(B, L, H, norm):
+@pytest.mark.parametrize("d", [64, 128])
+def test_bf16_pair_inputs_reach_fp32_like_accuracy(B, L, H, norm, d):
     """Q, K, V as bf16 pairs (hi + lo planes): three-term tensor-core products, error far below the
     single-bf16 bound (this is the mixer's attention path)."""
     rng = np.random.default_rng(B + L + H)
-    q, k, v = (rng.standard_normal((B, L, H, 64), dtype=np.float32) * 2 for _ in range(3))
+    q, k, v = (rng.standard_normal((B, L, H, d), dtype=np.float32) * 2 for _ in range(3))
     (qd, qv), (kd, kv), (vd, vv) = _pair(q), _pair(k), _pair(v)
-    assert chela.linattn_kernel_kind(B, H, L, 64, 64, 64, chela.BF16_PAIR, chela.F32) == 2
+    assert chela.linattn_kernel_kind(B, H, L, d, d, 64, chela.BF16_PAIR, chela.F32) == 2
     o = chela.linattn_fwd(qd, kd, vd, chunk=64, norm=chela.NORM_RMS if norm else chela.NORM_NONE, in_dtype=chela.BF16_PAIR)
     ref = oracle.linattn_recurrent(qv, kv, vv, norm=norm)
     assert rel_err(to_numpy(o), ref) <= 5e-4

@@ -50,6 +50,15 @@ def test_mixer_qk_diag_biases_and_no_silu():
     assert rel_err(to_numpy(o), ref) <= TOL
 
 
+def test_mixer_config4_shape_reduced_length():
+    """Config 4 layer (D=1024, H=8, head dim 128, C=128) at L=2048 so that the oracle finishes in seconds."""
+    B, L, D, H = 1, 2048, 1024, 8
+    m = inputs.mixer(3, B, L, D)
+    got = run_mixer(m, H, 128)
+    ref = oracle.mixer(m["x"], m["w_short"], m["k_long"], m["w_q"], m["w_k"], m["w_v"], H)
+    assert rel_err(got, ref) <= TOL
+
+
 def test_mixer_config3_shape_one_batch():
     """Config 3 layer (D=512, H=8, L=16384, C=64) on one batch row: the oracle's FFT form finishes in seconds."""
     B, L, D, H = 1, 16384, 512, 8
