@@ -167,6 +167,48 @@ def workload_config():
             "l2": "inputs+outputs %.2f GB per step, larger than L2: no flush needed" % (BYTES_PER_TOKEN_HEAD * TOTAL_TOKENS * H / 1e9)}
 
 
+def run_mixer_mode(args):
+    """--mixer: one step = one chela_mixer_fwd call; prints one JSON line (tokens/s, share of the bf16 tensor peak)."""
+    import torch
+    from paper_2406_08128_b200 import build as _build, chela
+    _build.build()
+    mb, ml, md, mh, mc = (int(x) for x in args.mixer.split(","))
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device=dev).manual_seed(2)
+    x = torch.randn(mb, ml, md, device=dev, generator=gen).to(torch.bfloat16)
+    w_s = torch.randn(md, 3, device=dev, generator=gen) / 3 ** 0.5
+    k_l = torch.randn(md, ml, device=dev, generator=gen) * torch.exp(-0.001 * torch.arange(ml, device=dev))[None, :]
+    w_q, w_k, w_v = [(torch.randn(md, md, device=dev, generator=gen) / md ** 0.5).to(torch.bfloat16) for _ in range(3)]
+    ws = torch.zeros(chela.mixer_workspace_bytes(mb, ml, md, mh, mc), dtype=torch.uint8, device=dev)
+    out = torch.empty(mb, ml, md, device=dev)
+    step = lambda: chela.mixer_fwd(x, w_s, k_l, w_q, w_k, w_v, mh, chunk=mc, out=out, workspace=ws)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    if chela.async_status(ws) != chela.OK:
+        raise RuntimeError("device-side wait timed out")
+    ms = e0.elapsed_time(e1) / args.steps
+    peaks, peak_kind = measured_peaks()
+    d_head = md // mh
+    flops_tok = 3 * 2 * md * md + mh * (4 * 64 * d_head + 4 * d_head * d_head)
+    achieved = flops_tok * mb * ml / (ms * 1e-3) / 1e12
+    print(json.dumps({"metric": "mixer_fwd_tokens_per_s", "value": mb * ml / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "token mixer forward B=%d L=%d D=%d H=%d chunk=%d, bf16 in, fp32 out" % (mb, ml, md, mh, mc)},
+                      "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                   "frac": achieved / peaks["bf16_tflops"], "traffic": None, "peak_source": peak_kind,
+                                   "note": "algorithmic flops (3 dense projections + attention tiles) over the whole call; "
+                                           "the long convolution (fp32 FFT on the plain ALUs) is inside the time"}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -176,7 +218,12 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the sweep / config-2 / mixer / CPU-oracle extras")
     ap.add_argument("--tokens", type=int, default=TOTAL_TOKENS, help="B*L of the timed step (profiling captures use a smaller case)")
     ap.add_argument("--L", type=int, default=L_MAIN, help="sequence length of the timed step")
+    ap.add_argument("--mixer", default=None, metavar="B,L,D,H,chunk",
+                    help="time the whole token mixer (short conv, long conv, Q/K/V, attention) on this shape instead, "
+                         "e.g. 4,16384,512,8,64 (config 3) or 8,8192,1024,8,128 (config 4); single GPU")
     args = ap.parse_args()
+    if args.mixer:
+        return run_mixer_mode(args)
     if (args.tokens, args.L) != (TOTAL_TOKENS, L_MAIN):
         globals().update(TOTAL_TOKENS=args.tokens, L_MAIN=args.L)
         args.no_extras = True

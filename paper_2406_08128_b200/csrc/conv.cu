@@ -84,6 +84,72 @@ __global__ void conv_transpose_kernel(const T *__restrict__ x, const float *__re
     }
 }
 
+// Fast form of conv_transpose_kernel for bf16 input and W <= 4 taps (W = 0: plain transpose): a
+// 64-channel x 64-token tile; each lane owns two adjacent channels (4-byte loads, 128 B per warp row) and
+// walks 8 consecutive tokens with the previous W-1 inputs in registers.
+template <int W>
+__global__ void __launch_bounds__(256)
+conv_transpose_bf16_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ w, float *__restrict__ at, int L,
+                           int D, int Ls)
+{
+    __shared__ float tile[64][65];
+    const int b = blockIdx.z, t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
+    const int lane = threadIdx.x & 31, wrp = threadIdx.x >> 5;
+    const int c = c0 + 2 * lane;
+    constexpr int WW = W > 0 ? W : 1;
+    float w0[WW], w1[WW];
+#pragma unroll
+    for (int j = 0; j < WW; ++j) {
+        w0[j] = (W > 0 && c < D) ? w[c * W + j] : 0.f;
+        w1[j] = (W > 0 && c + 1 < D) ? w[(c + 1) * W + j] : 0.f;
+    }
+    float2 hist[WW];   // hist[j] = x[t - j]
+#pragma unroll
+    for (int j = 0; j < WW; ++j) hist[j] = make_float2(0.f, 0.f);
+    const int ts = t0 + wrp * 8;
+    auto load = [&](int t) -> float2 {
+        if (t < 0 || t >= L || c >= D) return make_float2(0.f, 0.f);   // D is even: c + 1 < D whenever c < D
+        return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(x + ((size_t)b * L + t) * D + c));
+    };
+#pragma unroll
+    for (int j = 1; j < WW; ++j) hist[j] = load(ts - j);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        hist[0] = load(ts + i);
+        float2 y;
+        if (W > 0) {
+            y = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < WW; ++j) {
+                y.x = fmaf(w0[j], hist[j].x, y.x);
+                y.y = fmaf(w1[j], hist[j].y, y.y);
+            }
+            y.x = silu_f(y.x);
+            y.y = silu_f(y.y);
+        } else {
+            y = hist[0];
+        }
+        tile[2 * lane][wrp * 8 + i] = y.x;
+        tile[2 * lane + 1][wrp * 8 + i] = y.y;
+#pragma unroll
+        for (int j = WW - 1; j > 0; --j) hist[j] = hist[j - 1];
+    }
+    __syncthreads();
+    // rows of at: 64 tokens = 256 B per channel; a half-warp writes one row with float4 stores
+    const int half = lane >> 4, l16 = lane & 15;
+    for (int cc = wrp * 2 + half; cc < 64; cc += 16) {
+        if (c0 + cc >= D) continue;
+        const int t = t0 + 4 * l16;
+        if (t >= Ls) continue;   // Ls is a multiple of 8: a float4 is either inside or outside
+        float4 v = make_float4(tile[cc][4 * l16], tile[cc][4 * l16 + 1], tile[cc][4 * l16 + 2], tile[cc][4 * l16 + 3]);
+        if (t + 0 >= L) v.x = 0.f;
+        if (t + 1 >= L) v.y = 0.f;
+        if (t + 2 >= L) v.z = 0.f;
+        if (t + 3 >= L) v.w = 0.f;
+        *reinterpret_cast<float4 *>(at + ((size_t)b * D + c0 + cc) * Ls + t) = v;
+    }
+}
+
 // zt[B,D,Ls] fp32 -> z[B,L,D].  Tile: 64 channels x 32 tokens.
 // lo_offset != 0: z is a bf16 pair; the low plane (z + lo_offset) receives round(value - high part).
 template <typename T>
@@ -107,6 +173,41 @@ __global__ void transpose_out_kernel(const float *__restrict__ zt, T *__restrict
                 store1(z + idx, val);
                 if (lo_offset) store1(z + lo_offset + idx, val - load1(z + idx));
             }
+    }
+}
+
+// Fast form for bf16 (pair) output: 64 channels x 64 tokens; float4 loads along tokens, 4-byte stores of
+// two adjacent channels (128 B per warp row).
+__global__ void __launch_bounds__(256)
+transpose_out_bf16_kernel(const float *__restrict__ zt, __nv_bfloat16 *__restrict__ z, int L, int D, int Ls, size_t lo_offset)
+{
+    __shared__ float tile[64][65];
+    const int b = blockIdx.z, t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
+    const int lane = threadIdx.x & 31, wrp = threadIdx.x >> 5;
+    const int half = lane >> 4, l16 = lane & 15;
+    for (int cc = wrp * 2 + half; cc < 64; cc += 16) {
+        const int t = t0 + 4 * l16;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c0 + cc < D && t < Ls) v = *reinterpret_cast<const float4 *>(zt + ((size_t)b * D + c0 + cc) * Ls + t);
+        tile[cc][4 * l16] = v.x;
+        tile[cc][4 * l16 + 1] = v.y;
+        tile[cc][4 * l16 + 2] = v.z;
+        tile[cc][4 * l16 + 3] = v.w;
+    }
+    __syncthreads();
+    const int c = c0 + 2 * lane;
+    if (c >= D) return;
+    for (int tt = wrp; tt < 64; tt += 8) {
+        const int t = t0 + tt;
+        if (t >= L) break;
+        const float v0 = tile[2 * lane][tt], v1 = tile[2 * lane + 1][tt];
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(v0, v1);
+        const size_t idx = ((size_t)b * L + t) * D + c;
+        *reinterpret_cast<__nv_bfloat162 *>(z + idx) = hi;
+        if (lo_offset) {
+            const float2 hf = __bfloat1622float2(hi);
+            *reinterpret_cast<__nv_bfloat162 *>(z + lo_offset + idx) = __floats2bfloat162_rn(v0 - hf.x, v1 - hf.y);
+        }
     }
 }
 
@@ -168,9 +269,12 @@ __device__ __forceinline__ void dif_pass(float2 *s, const Twiddles &tw, int M, i
 {
     constexpr int G = 1 << R;
     const int q = len >> R, tws = (2 * M) / len;
+    // a stride of whole 128-element blocks leaves the swizzle pattern of the group's elements unchanged
+    const bool aligned = (q & 127) == 0;
     for (int g = threadIdx.x; g < (M >> R); g += blockDim.x) {
         const int k = g & (q - 1);
         const int i0 = ((g - k) << R) + k;
+        const int p0 = phys(i0);
         float2 v[G];
         if (kContiguous) {   // q == 1, G == 16: eight 16-byte chunks per thread
 #pragma unroll
@@ -179,6 +283,9 @@ __device__ __forceinline__ void dif_pass(float2 *s, const Twiddles &tw, int M, i
                 v[2 * c] = make_float2(t.x, t.y);
                 v[2 * c + 1] = make_float2(t.z, t.w);
             }
+        } else if (aligned) {
+#pragma unroll
+            for (int j = 0; j < G; ++j) v[j] = s[p0 + j * q];
         } else {
 #pragma unroll
             for (int j = 0; j < G; ++j) v[j] = s[phys(i0 + j * q)];
@@ -203,6 +310,9 @@ __device__ __forceinline__ void dif_pass(float2 *s, const Twiddles &tw, int M, i
 #pragma unroll
             for (int c = 0; c < G / 2; ++c)
                 *reinterpret_cast<float4 *>(s + phys(i0 + 2 * c)) = make_float4(v[2 * c].x, v[2 * c].y, v[2 * c + 1].x, v[2 * c + 1].y);
+        } else if (aligned) {
+#pragma unroll
+            for (int j = 0; j < G; ++j) s[p0 + j * q] = v[j];
         } else {
 #pragma unroll
             for (int j = 0; j < G; ++j) s[phys(i0 + j * q)] = v[j];
@@ -218,9 +328,11 @@ __device__ __forceinline__ void dit_pass(float2 *s, const Twiddles &tw, int M, i
 {
     constexpr int G = 1 << R;
     const int h0 = len0 >> 1;
+    const bool aligned = (h0 & 127) == 0;
     for (int g = threadIdx.x; g < (M >> R); g += blockDim.x) {
         const int k = g & (h0 - 1);
         const int i0 = ((g - k) << R) + k;
+        const int p0 = phys(i0);
         float2 v[G];
         if (kContiguous) {   // len0 == 2, G == 16
 #pragma unroll
@@ -229,6 +341,9 @@ __device__ __forceinline__ void dit_pass(float2 *s, const Twiddles &tw, int M, i
                 v[2 * c] = make_float2(t.x, t.y);
                 v[2 * c + 1] = make_float2(t.z, t.w);
             }
+        } else if (aligned) {
+#pragma unroll
+            for (int j = 0; j < G; ++j) v[j] = s[p0 + j * h0];
         } else {
 #pragma unroll
             for (int j = 0; j < G; ++j) v[j] = s[phys(i0 + j * h0)];
@@ -256,6 +371,9 @@ __device__ __forceinline__ void dit_pass(float2 *s, const Twiddles &tw, int M, i
 #pragma unroll
             for (int c = 0; c < G / 2; ++c)
                 *reinterpret_cast<float4 *>(s + phys(i0 + 2 * c)) = make_float4(v[2 * c].x, v[2 * c].y, v[2 * c + 1].x, v[2 * c + 1].y);
+        } else if (aligned) {
+#pragma unroll
+            for (int j = 0; j < G; ++j) s[p0 + j * h0] = v[j];
         } else {
 #pragma unroll
             for (int j = 0; j < G; ++j) s[phys(i0 + j * h0)] = v[j];
@@ -449,7 +567,18 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
     float2 *spec = (float2 *)(ws + p.off_spec);
 
     dim3 g1((L + 63) / 64, (D + 31) / 32, B);
-    if (in_dtype == CHELA_BF16)
+    const int wfast = w_short ? short_width : 0;
+    if (in_dtype == CHELA_BF16 && wfast <= 4) {
+        dim3 gf((L + 63) / 64, (D + 63) / 64, B);
+        const __nv_bfloat16 *xb = (const __nv_bfloat16 *)x;
+        switch (wfast) {
+            case 0: conv_transpose_bf16_kernel<0><<<gf, 256, 0, stream>>>(xb, w_short, at, L, D, p.Ls); break;
+            case 1: conv_transpose_bf16_kernel<1><<<gf, 256, 0, stream>>>(xb, w_short, at, L, D, p.Ls); break;
+            case 2: conv_transpose_bf16_kernel<2><<<gf, 256, 0, stream>>>(xb, w_short, at, L, D, p.Ls); break;
+            case 3: conv_transpose_bf16_kernel<3><<<gf, 256, 0, stream>>>(xb, w_short, at, L, D, p.Ls); break;
+            default: conv_transpose_bf16_kernel<4><<<gf, 256, 0, stream>>>(xb, w_short, at, L, D, p.Ls); break;
+        }
+    } else if (in_dtype == CHELA_BF16)
         conv_transpose_kernel<__nv_bfloat16><<<g1, 256, 0, stream>>>((const __nv_bfloat16 *)x, w_short, short_width,
                                                                      at, L, D, p.Ls);
     else
@@ -467,10 +596,11 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
     fft_conv_kernel<1><<<B * D, threads, smem, stream>>>(at, p.Ls, L, D, p.M, p.logM, tw, spec);
 
     dim3 g2((L + 31) / 32, (D + 63) / 64, B);
-    if (out_dtype == CHELA_BF16 || out_dtype == CHELA_BF16_PAIR)
-        transpose_out_kernel<__nv_bfloat16><<<g2, 256, 0, stream>>>(at, (__nv_bfloat16 *)z, L, D, p.Ls,
-                                                                    out_dtype == CHELA_BF16_PAIR ? (size_t)B * L * D : 0);
-    else
+    if (out_dtype == CHELA_BF16 || out_dtype == CHELA_BF16_PAIR) {
+        dim3 gf((L + 63) / 64, (D + 63) / 64, B);
+        transpose_out_bf16_kernel<<<gf, 256, 0, stream>>>(at, (__nv_bfloat16 *)z, L, D, p.Ls,
+                                                          out_dtype == CHELA_BF16_PAIR ? (size_t)B * L * D : 0);
+    } else
         transpose_out_kernel<float><<<g2, 256, 0, stream>>>(at, (float *)z, L, D, p.Ls, 0);
     return last_launch_status();
 }
