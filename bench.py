@@ -398,7 +398,7 @@ def main():
                            "tokens_per_s": mb * ml / (ms * 1e-3),
                            "tensor_frac": flops_tok * mb * ml / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                            "attention_kernel_kind": chela.linattn_kernel_kind(mb, mh, ml, d_head, d_head, mc,
-                                                                              chela.BF16_PAIR if d_head == 64 else chela.F32)})
+                                                                              chela.BF16_PAIR)})
             del x, k_l, mws, mo
         line["mixer"] = mixers
         # ---- CPU oracle on the host cores, bounded sample -----------------------------------------------

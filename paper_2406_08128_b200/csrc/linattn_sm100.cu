@@ -544,7 +544,7 @@ bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int C, boo
 }
 
 // How a call is split along L.  The grid holds B*H*G CTAs, no more than are resident at once (two per SM,
-// one per SM for bf16-pair inputs); a group never has fewer than 8 chunks.
+// one per SM for bf16-pair inputs); a group never has fewer than 16 chunks.
 struct SplitPlan {
     int G, cpg;
     size_t part_bytes;
@@ -559,10 +559,12 @@ SplitPlan split_plan(int B, int H, int L, bool pair)
     const long long bh = (long long)B * H;
     const int nchunks = (L + kC - 1) / kC;
     const long long slots = (pair ? 1LL : 2LL) * sms;   // resident CTAs: shared memory allows 2 per SM, 1 for pairs
+    // Measured on B200: with fewer (batch, head) pairs than SMs, fill the resident slots (a lone CTA per SM is
+    // bound by its own dependency chain, two per SM by HBM), but keep at least 16 chunks per group.
     int G = 1;
-    if (bh < slots) {
+    if (bh < sms) {
         G = (int)(slots / bh);
-        if (G > nchunks / 8) G = nchunks / 8;
+        if (G > nchunks / 16) G = nchunks / 16;
         if (G < 1) G = 1;
     }
     SplitPlan p;

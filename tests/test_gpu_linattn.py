@@ -95,7 +95,7 @@ def test_sweep_shapes_sampled(B, L):
     assert bool(torch.isfinite(o).all())
 
 
-@pytest.mark.parametrize("B,L,H", [(1, 8192, 2), (1, 5000, 3), (1, 1100, 1), (2, 4096, 1)])
+@pytest.mark.parametrize("B,L,H", [(1, 8192, 2), (1, 5000, 3), (1, 2100, 1), (2, 4096, 1)])
 def test_sequences_split_along_length(B, L, H):
     """Few (batch, head) pairs: the tensor-core path splits each sequence into groups of chunks whose
     initial states come from a separate K^T V pass; the result must still match the oracle."""
