@@ -104,6 +104,23 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
                                  void *workspace, size_t workspace_bytes, cudaStream_t stream);
 
 /*
+ * chela_linattn_fwd with the running state carried across calls, for segment-wise sequential evaluation
+ * and decoding (Sec. 5, language modelling: "process each segment sequentially"; the state is the
+ * intermediate variable of Sec. 4.1):
+ *   S_{-1} = state_in (zero if NULL);  outputs as chela_linattn_fwd;  state_out = S after the last token.
+ * Evaluating a sequence in consecutive segments with the state carried gives the result of one call over
+ * the whole sequence (up to rounding).  state_in, state_out : [B, H, d_k, d_v] fp32, nullable, may alias
+ * each other.  Supported: everything chela_linattn_fwd supports except bf16(-pair) inputs with d = 128
+ * (CHELA_ERR_UNSUPPORTED; fp32 inputs with d = 128 are fine).
+ */
+chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void *v, void *o,
+                                       const float *state_in, float *state_out,
+                                       int B, int H, int L, int d_k, int d_v, int chunk,
+                                       chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                                       chela_norm_t norm, float norm_eps, float scale,
+                                       void *workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/*
  * Dense projection with optional SiLU, the building block of the Q/K/V formation (Eq. 12; Eqs. 10-11 in
  * their dense form): y = act(a w + bias), fp32 accumulation.
  * a : [M, K], a_dtype in {F32, BF16, BF16_PAIR}.  w : [K, N] row-major, w_dtype in {F32, BF16}.

@@ -36,6 +36,8 @@ _SIGNATURES = {
     "chela_linattn_workspace_bytes": (_c_size_t, [_c_int] * 6),
     "chela_linattn_fwd": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                    _c_float, _vp, _c_size_t, _vp]),
+    "chela_linattn_carry_fwd": (_c_int, [_vp, _vp, _vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
+                                         _c_float, _vp, _c_size_t, _vp]),
     "chela_dense_workspace_bytes": (_c_size_t, []),
     "chela_dense_fwd": (_c_int, [_vp, _vp, _vp, _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _vp,
                                  _c_size_t, _vp]),
@@ -156,6 +158,23 @@ def linattn_fwd(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale
                                    int(norm), float(eps), float(scale), _ptr(workspace), workspace.numel(),
                                    _stream()), "chela_linattn_fwd")
     return o
+
+
+def linattn_carry_fwd(q, k, v, state_in=None, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale=1.0, out=None,
+                      state_out=None, workspace=None, in_dtype=None):
+    """chela_linattn_carry_fwd: returns (o, state_out); state tensors are [B,H,d_k,d_v] fp32."""
+    in_dtype = _dt(q) if in_dtype is None else in_dtype
+    B, L, H, d_k = q.shape[-4:]
+    d_v = v.shape[-1]
+    o = torch.empty((B, L, H, d_v), dtype=_tdtype(out_dtype), device=q.device) if out is None else out
+    if state_out is None:
+        state_out = torch.empty((B, H, d_k, d_v), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = _workspace(linattn_workspace_bytes(B, H, L, d_k, d_v, chunk), q.device)
+    _check(lib().chela_linattn_carry_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(state_in), _ptr(state_out), B, H, L,
+                                         d_k, d_v, chunk, in_dtype, _dt(o), int(norm), float(eps), float(scale),
+                                         _ptr(workspace), workspace.numel(), _stream()), "chela_linattn_carry_fwd")
+    return o, state_out
 
 
 def linattn_fwd_static_ws(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale=1.0, out=None):

@@ -92,27 +92,39 @@ size_t chela_linattn_workspace_bytes(int B, int H, int L, int d_k, int d_v, int 
     return linattn_sm100_workspace_bytes(B, H, L, d_k, chunk);
 }
 
+chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void *v, void *o, const float *state_in,
+                                       float *state_out, int B, int H, int L, int d_k, int d_v, int chunk,
+                                       chela_dtype_t in_dtype, chela_dtype_t out_dtype, chela_norm_t norm,
+                                       float norm_eps, float scale, void *workspace, size_t workspace_bytes,
+                                       cudaStream_t stream)
+{
+    if (!q || !k || !v || !o || B < 1 || H < 1 || L < 1 || d_k < 1 || d_v < 1 || chunk < 1 ||
+        !(dtype_ok(in_dtype) || in_dtype == CHELA_BF16_PAIR) || !dtype_ok(out_dtype) ||
+        (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) || !(norm_eps >= 0.f))
+        return CHELA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(workspace) ||
+        !aligned16(state_in) || !aligned16(state_out))
+        return CHELA_ERR_INVALID_ARG;
+    const int kind = chela_linattn_kernel_kind(B, H, L, d_k, d_v, chunk, in_dtype, out_dtype);
+    if (kind == 0) return CHELA_ERR_UNSUPPORTED;
+    if (kind == 2) {
+        if (d_k == 128 && (state_in || state_out)) return CHELA_ERR_UNSUPPORTED;
+        const size_t need = linattn_sm100_workspace_bytes(B, H, L, d_k, chunk);
+        if (need && (!workspace || workspace_bytes < need)) return CHELA_ERR_WORKSPACE;
+        return launch_linattn_sm100(q, k, v, o, B, H, L, d_k, chunk, in_dtype, out_dtype, (int)norm, norm_eps,
+                                    scale, workspace, stream, state_in, state_out);
+    }
+    return launch_linattn_simt(q, k, v, o, B, H, L, d_k, chunk, in_dtype, out_dtype, (int)norm, norm_eps, scale,
+                               stream, state_in, state_out);
+}
+
 chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                                  int d_k, int d_v, int chunk, chela_dtype_t in_dtype,
                                  chela_dtype_t out_dtype, chela_norm_t norm, float norm_eps, float scale,
                                  void *workspace, size_t workspace_bytes, cudaStream_t stream)
 {
-    if (!q || !k || !v || !o || B < 1 || H < 1 || L < 1 || d_k < 1 || d_v < 1 || chunk < 1 ||
-        !(dtype_ok(in_dtype) || in_dtype == CHELA_BF16_PAIR) || !dtype_ok(out_dtype) || (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) ||
-        !(norm_eps >= 0.f))
-        return CHELA_ERR_INVALID_ARG;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(workspace))
-        return CHELA_ERR_INVALID_ARG;
-    const int kind = chela_linattn_kernel_kind(B, H, L, d_k, d_v, chunk, in_dtype, out_dtype);
-    if (kind == 0) return CHELA_ERR_UNSUPPORTED;
-    if (kind == 2) {
-        const size_t need = linattn_sm100_workspace_bytes(B, H, L, d_k, chunk);
-        if (need && (!workspace || workspace_bytes < need)) return CHELA_ERR_WORKSPACE;
-        return launch_linattn_sm100(q, k, v, o, B, H, L, d_k, chunk, in_dtype, out_dtype, (int)norm, norm_eps,
-                                    scale, workspace, stream);
-    }
-    return launch_linattn_simt(q, k, v, o, B, H, L, d_k, chunk, in_dtype, out_dtype, (int)norm, norm_eps, scale,
-                               stream);
+    return chela_linattn_carry_fwd(q, k, v, o, nullptr, nullptr, B, H, L, d_k, d_v, chunk, in_dtype, out_dtype, norm,
+                                   norm_eps, scale, workspace, workspace_bytes, stream);
 }
 
 size_t chela_dense_workspace_bytes(void) { return 256; }

@@ -47,7 +47,7 @@ __device__ __forceinline__ void store1(__nv_bfloat16 *p, float v) { *p = __float
 chela_status_t launch_linattn_simt(const void *q, const void *k, const void *v, void *o, int B, int H,
                                    int L, int d, int chunk, chela_dtype_t in_dtype,
                                    chela_dtype_t out_dtype, int norm, float eps, float scale,
-                                   cudaStream_t stream);
+                                   cudaStream_t stream, const float *state_in = nullptr, float *state_out = nullptr);
 
 // tcgen05/TMEM/TMA kernel for bf16 inputs
 bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_t in_dtype,
@@ -56,7 +56,8 @@ size_t linattn_sm100_workspace_bytes(int B, int H, int L, int d, int chunk);
 chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v, void *o, int B, int H,
                                     int L, int d, int chunk, chela_dtype_t in_dtype,
                                     chela_dtype_t out_dtype, int norm, float eps, float scale,
-                                    void *workspace, cudaStream_t stream);
+                                    void *workspace, cudaStream_t stream, const float *state_in = nullptr,
+                                    float *state_out = nullptr);
 
 chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                                          chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,

@@ -21,7 +21,8 @@ struct SimtSmem {
 template <int D, int C, typename TIn, typename TOut>
 __global__ void __launch_bounds__(kThreads)
 linattn_simt_kernel(const TIn *__restrict__ q, const TIn *__restrict__ k, const TIn *__restrict__ v,
-                    TOut *__restrict__ o, int H, int L, float scale, int norm, float eps)
+                    TOut *__restrict__ o, int H, int L, float scale, int norm, float eps,
+                    const float *__restrict__ state_in, float *__restrict__ state_out)
 {
     extern __shared__ __align__(16) float smem[];
     constexpr int KS = SimtSmem<D, C>::KS;
@@ -36,7 +37,8 @@ linattn_simt_kernel(const TIn *__restrict__ q, const TIn *__restrict__ k, const 
     const size_t row_stride = (size_t)H * D;
     const size_t base = ((size_t)b * L * H + h) * D;
 
-    for (int i = tid; i < D * D; i += kThreads) sS[i] = 0.f;
+    // running state: zero, or the caller's initial state [B*H][D][D]
+    for (int i = tid; i < D * D; i += kThreads) sS[i] = state_in ? state_in[(size_t)blockIdx.x * D * D + i] : 0.f;
 
     for (int t0 = 0; t0 < L; t0 += C) {
         const int n = min(C, L - t0);
@@ -147,33 +149,35 @@ linattn_simt_kernel(const TIn *__restrict__ q, const TIn *__restrict__ k, const 
         }
         __syncthreads();
     }
+    if (state_out)
+        for (int i = tid; i < D * D; i += kThreads) state_out[(size_t)blockIdx.x * D * D + i] = sS[i];
 }
 
 template <int D, int C, typename TIn, typename TOut>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
-                        int norm, float eps, float scale, cudaStream_t stream)
+                        int norm, float eps, float scale, cudaStream_t stream, const float *state_in, float *state_out)
 {
     auto kern = linattn_simt_kernel<D, C, TIn, TOut>;
     const size_t smem = sizeof(float) * SimtSmem<D, C>::floats;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return CHELA_ERR_CUDA;
     kern<<<B * H, kThreads, smem, stream>>>((const TIn *)q, (const TIn *)k, (const TIn *)v, (TOut *)o, H, L,
-                                           scale, norm, eps);
+                                           scale, norm, eps, state_in, state_out);
     return last_launch_status();
 }
 
 template <int D, int C>
 chela_status_t launch_d(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                         chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
-                        cudaStream_t stream)
+                        cudaStream_t stream, const float *state_in, float *state_out)
 {
     if (in_dtype == CHELA_F32 && out_dtype == CHELA_F32)
-        return launch_t<D, C, float, float>(q, k, v, o, B, H, L, norm, eps, scale, stream);
+        return launch_t<D, C, float, float>(q, k, v, o, B, H, L, norm, eps, scale, stream, state_in, state_out);
     if (in_dtype == CHELA_BF16 && out_dtype == CHELA_F32)
-        return launch_t<D, C, __nv_bfloat16, float>(q, k, v, o, B, H, L, norm, eps, scale, stream);
+        return launch_t<D, C, __nv_bfloat16, float>(q, k, v, o, B, H, L, norm, eps, scale, stream, state_in, state_out);
     if (in_dtype == CHELA_BF16 && out_dtype == CHELA_BF16)
-        return launch_t<D, C, __nv_bfloat16, __nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, stream);
-    return launch_t<D, C, float, __nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, stream);
+        return launch_t<D, C, __nv_bfloat16, __nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, stream, state_in, state_out);
+    return launch_t<D, C, float, __nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, stream, state_in, state_out);
 }
 
 }  // namespace
@@ -183,11 +187,11 @@ chela_status_t launch_d(const void *q, const void *k, const void *v, void *o, in
 chela_status_t launch_linattn_simt(const void *q, const void *k, const void *v, void *o, int B, int H,
                                    int L, int d, int chunk, chela_dtype_t in_dtype,
                                    chela_dtype_t out_dtype, int norm, float eps, float scale,
-                                   cudaStream_t stream)
+                                   cudaStream_t stream, const float *state_in, float *state_out)
 {
-    if (d == 64 && chunk == 64) return launch_d<64, 64>(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, stream);
-    if (d == 64 && chunk == 128) return launch_d<64, 128>(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, stream);
-    if (d == 128) return launch_d<128, 64>(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, stream);
+    if (d == 64 && chunk == 64) return launch_d<64, 64>(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, stream, state_in, state_out);
+    if (d == 64 && chunk == 128) return launch_d<64, 128>(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, stream, state_in, state_out);
+    if (d == 128) return launch_d<128, 64>(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, stream, state_in, state_out);
     return CHELA_ERR_UNSUPPORTED;
 }
 

@@ -71,10 +71,11 @@ __global__ void __launch_bounds__(kThreads)
 linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
                      float scale, int norm, float eps, int *__restrict__ status, const float *__restrict__ s_part,
-                     int G, int cpg)
+                     int G, int cpg, const float *__restrict__ state_in, float *__restrict__ state_out)
 {
     // Grid: one CTA per (batch*head, group).  Group g covers chunks [g*cpg, (g+1)*cpg) of its sequence and
-    // starts from the state sum_{g' < g} s_part[bh][g'] (per-group K^T V sums written by the state kernel).
+    // starts from the state sum_{g' < g} s_part[bh][g'] (per-group K^T V sums written by the state kernel),
+    // plus the caller's initial state state_in[bh] if given; the last group writes the final state.
     using SM = Smem<TOut, kPair>;
     constexpr int kStages = SM::kStages;
     constexpr int kTPS = SM::kTilesPerStage;
@@ -89,7 +90,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const int b = bh / H, h = bh % H;
     const int c0 = g * cpg;                                        // first chunk of this group
     const int nchunks = min(cpg, (L + kC - 1) / kC - c0);          // chunks of this group
-    const bool has_init = g > 0;
+    const bool has_init = g > 0 || state_in != nullptr;
 
     const uint32_t bar_full0 = sbase + SM::offBar;
     const uint32_t bar_p = bar_full0 + 8 * kStages;   // G1 of a chunk has completed (tensor core -> warps 2,3)
@@ -262,6 +263,14 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 float sv[kD];
 #pragma unroll
                 for (int j = 0; j < kD; ++j) sv[j] = 0.f;
+                if (state_in) {
+                    const float4 *src = reinterpret_cast<const float4 *>(state_in + ((size_t)bh * kD + r) * kD);
+#pragma unroll
+                    for (int j = 0; j < kD / 4; ++j) {
+                        const float4 x = src[j];
+                        sv[4 * j] = x.x; sv[4 * j + 1] = x.y; sv[4 * j + 2] = x.z; sv[4 * j + 3] = x.w;
+                    }
+                }
                 for (int gp = 0; gp < g; ++gp) {
                     const float4 *src = reinterpret_cast<const float4 *>(s_part + (((size_t)bh * (G - 1) + gp) * kD + r) * kD);
 #pragma unroll
@@ -380,6 +389,14 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_s);
+                } else if (state_out && g == G - 1) {
+                    // last chunk of the sequence: the fp32 state leaves the SM once, for the caller
+                    tmem_ld32(tmem_warp + kColOS, *reinterpret_cast<float(*)[32]>(&acc[0]));
+                    tmem_ld32(tmem_warp + kColOS + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
+                    tmem_ld_wait();
+                    float4 *dst = reinterpret_cast<float4 *>(state_out + ((size_t)bh * kD + r) * kD);
+#pragma unroll
+                    for (int j = 0; j < kD / 4; ++j) dst[j] = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
                 }
                 TMARK(3);
             }
@@ -577,7 +594,7 @@ constexpr size_t kWsHeader = 512;   // word 0: asynchronous status; the rest: di
 
 template <typename TOut, bool kPair>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
-                        float scale, void *workspace, cudaStream_t stream)
+                        float scale, void *workspace, const float *state_in, float *state_out, cudaStream_t stream)
 {
     CUtensorMap mq, mk, mv, mo;
     const int planes = kPair ? 2 : 1;
@@ -599,7 +616,8 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
     const int smem = Smem<TOut, kPair>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return CHELA_ERR_CUDA;
-    kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg);
+    kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg,
+                                                     state_in, state_out);
     return last_launch_status();
 }
 
@@ -624,17 +642,19 @@ size_t linattn_sm100_workspace_bytes(int B, int H, int L, int d, int)
 
 chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int d,
                                     int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps,
-                                    float scale, void *workspace, cudaStream_t stream)
+                                    float scale, void *workspace, cudaStream_t stream, const float *state_in,
+                                    float *state_out)
 {
+    if (d == 128 && (state_in || state_out)) return CHELA_ERR_UNSUPPORTED;   // the caller routes these elsewhere
     if (d == 128) return launch_linattn_sm100_d128(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, workspace, stream);
     // The result does not depend on the chunk size: both supported values run on 64-token tiles.
     (void)chunk;
     if (in_dtype == CHELA_BF16_PAIR) {
-        if (out_dtype == CHELA_F32) return launch_t<float, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
-        return launch_t<__nv_bfloat16, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
+        if (out_dtype == CHELA_F32) return launch_t<float, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+        return launch_t<__nv_bfloat16, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
     }
-    if (out_dtype == CHELA_F32) return launch_t<float, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
-    return launch_t<__nv_bfloat16, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, stream);
+    if (out_dtype == CHELA_F32) return launch_t<float, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+    return launch_t<__nv_bfloat16, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
 }
 
 }  // namespace chela
