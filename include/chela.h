@@ -124,7 +124,7 @@ chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void 
  * Dense projection with optional SiLU, the building block of the Q/K/V formation (Eq. 12; Eqs. 10-11 in
  * their dense form): y = act(a w + bias), fp32 accumulation.
  * a : [M, K], a_dtype in {F32, BF16, BF16_PAIR}.  w : [K, N] row-major, w_dtype in {F32, BF16}.
- * bias : [N] fp32 or NULL.  y : [M, N], y_dtype in {F32, BF16, BF16_PAIR}.  act : 0 identity, 1 SiLU.
+ * bias : [N] fp32 or NULL.  y : [M, N], y_dtype in {F32, BF16, BF16_PAIR}.  act : 0 identity, 1 SiLU, 2 sigmoid.
  * Tensor-core path (tcgen05): a BF16 or BF16_PAIR, w BF16, y BF16 or BF16_PAIR, K a multiple of 64, N a
  * multiple of 128.  Other combinations without a pair run on an fp32 SIMT kernel; pairs outside the
  * tensor-core path are CHELA_ERR_UNSUPPORTED.  The workspace holds the asynchronous status word
@@ -195,6 +195,24 @@ chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_wi
                                int D, int H, int chunk, chela_dtype_t in_dtype,
                                chela_dtype_t out_dtype, chela_norm_t norm, float norm_eps,
                                void *workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/*
+ * Token mixer forward with the gates (Eqs. 8, 9, 13, 14): with O the output of chela_mixer_fwd,
+ *   G_a = silu(Z W_a + b_a),  G_o = sigmoid(Z W_o + b_o),  U = O . G_a . G_o + X . (1 - G_o).
+ * (Eq. 9 prints the gate weight with the same symbol as the value projection; it is read as a weight of
+ * its own, w_a.)  w_a, w_o : [D, D] row-major, in_dtype.  b_a, b_o : [D] fp32 or NULL.  u : [B, L, D]
+ * out_dtype.  Everything else as chela_mixer_fwd; the workspace is larger (three more [B, L, D] buffers).
+ */
+size_t chela_mixer_gated_workspace_bytes(int B, int L, int D, int H, int chunk, chela_dtype_t in_dtype);
+chela_status_t chela_mixer_gated_fwd(const void *x, const float *w_short, int short_width,
+                                     const float *k_long, const void *w_q, const void *w_k,
+                                     const void *w_v, const float *b_q, const float *b_k,
+                                     const float *b_v, const void *w_a, const float *b_a,
+                                     const void *w_o, const float *b_o, int qk_diag, int v_silu,
+                                     void *u, int B, int L, int D, int H, int chunk,
+                                     chela_dtype_t in_dtype, chela_dtype_t out_dtype, chela_norm_t norm,
+                                     float norm_eps, void *workspace, size_t workspace_bytes,
+                                     cudaStream_t stream);
 
 #ifdef __cplusplus
 }

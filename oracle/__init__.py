@@ -154,3 +154,19 @@ def dense(x, w, bias=None, act=False):
     y = np.empty((M, N))
     _load().oracle_dense(_p(x), _p(w), _p(b), _p(y), ctypes.c_size_t(M), K, N, int(bool(act)))
     return y
+
+
+def mixer_gated(x, w_short, k_long, w_q, w_k, w_v, w_a, w_o, H, b_q=None, b_k=None, b_v=None, b_a=None, b_o=None,
+                qk_diag=False, v_silu=True, norm=True, eps=1e-6, use_fft=True):
+    """Mixer with gates: U = O . silu(Z W_a + b_a) . sigmoid(Z W_o + b_o) + X . (1 - sigmoid(...)) (Eqs. 8-9, 13-14)."""
+    x, w_short, k_long = _f64(x), _f64(w_short), _f64(k_long)
+    w_q, w_k, w_v, w_a, w_o = _f64(w_q), _f64(w_k), _f64(w_v), _f64(w_a), _f64(w_o)
+    B, L, D = x.shape
+    opt = lambda b: None if b is None else _f64(b)
+    bq, bk, bv, ba, bo = opt(b_q), opt(b_k), opt(b_v), opt(b_a), opt(b_o)
+    u = np.empty_like(x)
+    _load().oracle_mixer_gated(_p(x), _p(w_short), w_short.shape[1], _p(k_long), _p(w_q), _p(w_k), _p(w_v),
+                               _p(bq), _p(bk), _p(bv), _p(w_a), _p(ba), _p(w_o), _p(bo), int(bool(qk_diag)),
+                               int(bool(v_silu)), _p(u), B, L, D, H, int(bool(norm)), ctypes.c_double(eps),
+                               int(bool(use_fft)))
+    return u

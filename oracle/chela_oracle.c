@@ -327,3 +327,27 @@ void oracle_mixer(const double *x, const double *w_short, int width, const doubl
     oracle_linattn_recurrent(qq, kk, vv, o, B, H, L, D / H, D / H, 1.0, norm, eps, NULL, NULL);
     free(a); free(z); free(qq); free(kk); free(vv);
 }
+
+/* Gated mixer (Eqs. 8, 9, 13, 14): with O = oracle_mixer(...) and Z its short-long convolution output,
+ *   G_a = silu(Z W_a + b_a), G_o = sigmoid(Z W_o + b_o), U = O . G_a . G_o + X . (1 - G_o). */
+void oracle_mixer_gated(const double *x, const double *w_short, int width, const double *k_long,
+                        const double *w_q, const double *w_k, const double *w_v,
+                        const double *b_q, const double *b_k, const double *b_v,
+                        const double *w_a, const double *b_a, const double *w_o, const double *b_o,
+                        int qk_diag, int v_silu, double *u,
+                        int B, int L, int D, int H, int norm, double eps, int use_fft)
+{
+    size_t M = (size_t)B * L, n = M * D;
+    double *o = (double *)malloc(sizeof(double) * n);
+    double *z = (double *)malloc(sizeof(double) * n);
+    double *ga = (double *)malloc(sizeof(double) * n);
+    double *go = (double *)malloc(sizeof(double) * n);
+    oracle_mixer(x, w_short, width, k_long, w_q, w_k, w_v, b_q, b_k, b_v, qk_diag, v_silu, o, z, B, L, D, H, norm, eps, use_fft);
+    oracle_dense(z, w_a, b_a, ga, M, D, D, 1);
+    oracle_dense(z, w_o, b_o, go, M, D, D, 0);
+    for (size_t i = 0; i < n; ++i) {
+        double g = 1.0 / (1.0 + exp(-go[i]));
+        u[i] = o[i] * ga[i] * g + x[i] * (1.0 - g);
+    }
+    free(o); free(z); free(ga); free(go);
+}

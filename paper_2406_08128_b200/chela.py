@@ -45,6 +45,10 @@ _SIGNATURES = {
     "chela_linattn_fwd_static_ws": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                              _c_float, _vp]),
     "chela_mixer_workspace_bytes": (_c_size_t, [_c_int] * 5 + [_c_int]),
+    "chela_mixer_gated_workspace_bytes": (_c_size_t, [_c_int] * 5 + [_c_int]),
+    "chela_mixer_gated_fwd": (_c_int, [_vp, _vp, _c_int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _c_int, _c_int,
+                                       _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_float,
+                                       _vp, _c_size_t, _vp]),
     "chela_mixer_fwd": (_c_int, [_vp, _vp, _c_int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _c_int, _c_int, _vp,
                                  _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_float,
                                  _vp, _c_size_t, _vp]),
@@ -203,7 +207,7 @@ def dense_fwd(a, w, bias=None, act=False, a_dtype=None, y_dtype=BF16, out=None, 
         out = torch.empty(shape, dtype=torch.float32 if y_dtype == F32 else torch.bfloat16, device=a.device)
     if workspace is None:
         workspace = _workspace(int(lib().chela_dense_workspace_bytes()), a.device)
-    _check(lib().chela_dense_fwd(_ptr(a), _ptr(w), _ptr(bias), _ptr(out), M, K, N, int(bool(act)), a_dtype, _dt(w),
+    _check(lib().chela_dense_fwd(_ptr(a), _ptr(w), _ptr(bias), _ptr(out), M, K, N, int(act), a_dtype, _dt(w),
                                  y_dtype, _ptr(workspace), workspace.numel(), _stream()), "chela_dense_fwd")
     return out
 
@@ -229,3 +233,22 @@ def mixer_fwd(x, w_short, k_long, w_q, w_k, w_v, H, chunk=64, b_q=None, b_k=None
                                  int(bool(v_silu)), _ptr(o), B, L, D, H, chunk, _dt(x), _dt(o), int(norm),
                                  float(eps), _ptr(workspace), workspace.numel(), _stream()), "chela_mixer_fwd")
     return o
+
+
+def mixer_gated_workspace_bytes(B, L, D, H, chunk, in_dtype=BF16) -> int:
+    return int(lib().chela_mixer_gated_workspace_bytes(B, L, D, H, chunk, in_dtype))
+
+
+def mixer_gated_fwd(x, w_short, k_long, w_q, w_k, w_v, w_a, w_o, H, chunk=64, b_q=None, b_k=None, b_v=None, b_a=None,
+                    b_o=None, qk_diag=False, v_silu=True, out_dtype=F32, norm=NORM_RMS, eps=1e-6, out=None, workspace=None):
+    """x [B,L,D] -> u [B,L,D]: the mixer with its gates G_a, G_o and the residual mix."""
+    B, L, D = x.shape
+    u = torch.empty((B, L, D), dtype=_tdtype(out_dtype), device=x.device) if out is None else out
+    if workspace is None:
+        workspace = _workspace(mixer_gated_workspace_bytes(B, L, D, H, chunk, _dt(x)), x.device)
+    _check(lib().chela_mixer_gated_fwd(_ptr(x), _ptr(w_short), w_short.shape[1], _ptr(k_long), _ptr(w_q), _ptr(w_k), _ptr(w_v),
+                                       _ptr(b_q), _ptr(b_k), _ptr(b_v), _ptr(w_a), _ptr(b_a), _ptr(w_o), _ptr(b_o),
+                                       int(bool(qk_diag)), int(bool(v_silu)), _ptr(u), B, L, D, H, chunk, _dt(x), _dt(u),
+                                       int(norm), float(eps), _ptr(workspace), workspace.numel(), _stream()),
+           "chela_mixer_gated_fwd")
+    return u

@@ -8,10 +8,10 @@ namespace {
 bool dtype_ok(chela_dtype_t t) { return t == CHELA_F32 || t == CHELA_BF16; }
 
 struct MixerPlan {
-    size_t off_conv, off_z, off_q, off_k, off_v, off_attn, total;
+    size_t off_conv, off_z, off_q, off_k, off_v, off_attn, off_ga, off_go, off_o, total;
     size_t conv_bytes, attn_bytes;
 };
-MixerPlan mixer_plan(int B, int L, int D, int H, int chunk)
+MixerPlan mixer_plan(int B, int L, int D, int H, int chunk, bool gated)
 {
     MixerPlan p;
     const size_t act = align_up((size_t)B * L * D * sizeof(float), 256);
@@ -23,7 +23,10 @@ MixerPlan mixer_plan(int B, int L, int D, int H, int chunk)
     p.off_q = p.off_z + act;
     p.off_k = p.off_q + act;
     p.off_v = p.off_k + act;
-    p.total = p.off_v + act;
+    p.off_ga = p.off_v + act;                 // gated form only: G_a, G_o, un-gated attention output
+    p.off_go = p.off_ga + (gated ? act : 0);
+    p.off_o = p.off_go + (gated ? act : 0);
+    p.total = p.off_o + (gated ? act : 0);
     return p;
 }
 
@@ -134,7 +137,7 @@ chela_status_t chela_dense_fwd(const void *a, const void *w, const float *bias, 
                                size_t workspace_bytes, cudaStream_t stream)
 {
     auto any_dtype = [](chela_dtype_t t) { return t == CHELA_F32 || t == CHELA_BF16 || t == CHELA_BF16_PAIR; };
-    if (!a || !w || !y || M < 1 || K < 1 || N < 1 || (act != 0 && act != 1) || !any_dtype(a_dtype) || !dtype_ok(w_dtype) ||
+    if (!a || !w || !y || M < 1 || K < 1 || N < 1 || (act < 0 || act > 2) || !any_dtype(a_dtype) || !dtype_ok(w_dtype) ||
         !any_dtype(y_dtype))
         return CHELA_ERR_INVALID_ARG;
     if (!aligned16(a) || !aligned16(w) || !aligned16(y) || !aligned16(workspace)) return CHELA_ERR_INVALID_ARG;
@@ -161,28 +164,38 @@ chela_status_t chela_async_status(const void *workspace, cudaStream_t stream)
 size_t chela_mixer_workspace_bytes(int B, int L, int D, int H, int chunk, chela_dtype_t)
 {
     if (B < 1 || L < 1 || D < 1 || H < 1 || D % H != 0) return 0;
-    return mixer_plan(B, L, D, H, chunk).total;
+    return mixer_plan(B, L, D, H, chunk, false).total;
 }
 
-chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_width, const float *k_long,
-                               const void *w_q, const void *w_k, const void *w_v, const float *b_q,
-                               const float *b_k, const float *b_v, int qk_diag, int v_silu, void *o, int B,
-                               int L, int D, int H, int chunk, chela_dtype_t in_dtype,
-                               chela_dtype_t out_dtype, chela_norm_t norm, float norm_eps, void *workspace,
-                               size_t workspace_bytes, cudaStream_t stream)
+size_t chela_mixer_gated_workspace_bytes(int B, int L, int D, int H, int chunk, chela_dtype_t)
 {
+    if (B < 1 || L < 1 || D < 1 || H < 1 || D % H != 0) return 0;
+    return mixer_plan(B, L, D, H, chunk, true).total;
+}
+
+}  // extern "C"
+
+namespace {
+chela_status_t mixer_impl(const void *x, const float *w_short, int short_width, const float *k_long, const void *w_q,
+                          const void *w_k, const void *w_v, const float *b_q, const float *b_k, const float *b_v,
+                          const void *w_a, const float *b_a, const void *w_o, const float *b_o, int qk_diag, int v_silu,
+                          void *o, int B, int L, int D, int H, int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                          chela_norm_t norm, float norm_eps, void *workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    const bool gated = w_a != nullptr;
+    if (gated && !w_o) return CHELA_ERR_INVALID_ARG;
     if (!x || !w_short || !k_long || !w_q || !w_k || !w_v || !o || B < 1 || L < 1 || D < 1 || H < 1 ||
         !dtype_ok(in_dtype) || !dtype_ok(out_dtype) || (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) ||
         !(norm_eps >= 0.f))
         return CHELA_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(o) || !aligned16(w_q) || !aligned16(w_k) || !aligned16(w_v) ||
-        !aligned16(workspace))
+        !aligned16(workspace) || !aligned16(w_a) || !aligned16(w_o))
         return CHELA_ERR_INVALID_ARG;
     if (D % H != 0) return CHELA_ERR_INVALID_ARG;
     const int d = D / H;
     if ((d != 64 && d != 128) || (chunk != 64 && chunk != 128) || L > 16384 || short_width < 1 || short_width > 16)
         return CHELA_ERR_UNSUPPORTED;
-    const MixerPlan p = mixer_plan(B, L, D, H, chunk);
+    const MixerPlan p = mixer_plan(B, L, D, H, chunk, gated);
     if (!workspace || workspace_bytes < p.total) return CHELA_ERR_WORKSPACE;
     char *ws = (char *)workspace;
     float *z = (float *)(ws + p.off_z), *qq = (float *)(ws + p.off_q), *kk = (float *)(ws + p.off_k),
@@ -190,6 +203,9 @@ chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_wi
     const size_t M = (size_t)B * L;
 
     const size_t n = M * D;
+    // gated form: the attention output goes to scratch, then u = o . G_a . G_o + x . (1 - G_o)  (Eqs. 8, 9, 13, 14)
+    void *attn_out = gated ? (void *)(ws + p.off_o) : o;
+    const chela_dtype_t attn_dtype = gated ? CHELA_F32 : out_dtype;
     // Tensor-core path: every intermediate (Z, Q, K, V) is a bf16 pair (hi + lo, about 16 mantissa bits) and
     // every product takes three tensor-core terms; single bf16 intermediates would cost the normalised
     // output its leading digits (cancellation in Q K^T on rows with a small pre-norm RMS).
@@ -212,10 +228,17 @@ chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_wi
         if (st != CHELA_OK) return st;
         st = launch_gemm_sm100(x, w_v, b_v, vp, M, D, D, v_silu ? 1 : 0, CHELA_BF16, CHELA_BF16_PAIR, status, stream);
         if (st != CHELA_OK) return st;
-        return launch_linattn_sm100(qp, kp, vp, o, B, H, L, d, chunk, CHELA_BF16_PAIR, out_dtype, (int)norm, norm_eps, 1.0f,
-                                    ws + p.off_attn, stream);
+        if (gated) {   // G_a = silu(Z W_a + b_a), G_o = sigmoid(Z W_o + b_o), as bf16 pairs
+            st = launch_gemm_sm100(zp, w_a, b_a, ws + p.off_ga, M, D, D, 1, CHELA_BF16_PAIR, CHELA_BF16_PAIR, status, stream);
+            if (st == CHELA_OK) st = launch_gemm_sm100(zp, w_o, b_o, ws + p.off_go, M, D, D, 2, CHELA_BF16_PAIR, CHELA_BF16_PAIR, status, stream);
+            if (st != CHELA_OK) return st;
+        }
+        st = launch_linattn_sm100(qp, kp, vp, attn_out, B, H, L, d, chunk, CHELA_BF16_PAIR, attn_dtype, (int)norm, norm_eps, 1.0f,
+                                  ws + p.off_attn, stream);
+        if (st != CHELA_OK || !gated) return st;
+        return launch_gate_combine((const float *)attn_out, ws + p.off_ga, ws + p.off_go, CHELA_BF16_PAIR, x, in_dtype, o,
+                                   out_dtype, n, stream);
     }
-    (void)n;
     // fp32 path.  Z = K_l(silu(K_s(X)))  (Eq. 7), kept in fp32
     st = launch_longconv(x, k_long, w_short, short_width, z, B, L, D, in_dtype, CHELA_F32,
                          ws + p.off_conv, stream);
@@ -231,9 +254,45 @@ chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_wi
     if (st != CHELA_OK) return st;
     st = launch_gemm_simt(x, w_v, b_v, vv, M, D, D, v_silu ? 1 : 0, in_dtype, in_dtype, CHELA_F32, stream);
     if (st != CHELA_OK) return st;
+    if (gated) {
+        st = launch_gemm_simt(z, w_a, b_a, ws + p.off_ga, M, D, D, 1, CHELA_F32, in_dtype, CHELA_F32, stream);
+        if (st == CHELA_OK) st = launch_gemm_simt(z, w_o, b_o, ws + p.off_go, M, D, D, 2, CHELA_F32, in_dtype, CHELA_F32, stream);
+        if (st != CHELA_OK) return st;
+    }
     // [B,L,D] with head h = columns [h*d,(h+1)*d) is [B,L,H,d]
-    return chela_linattn_fwd(qq, kk, vv, o, B, H, L, d, d, chunk, CHELA_F32, out_dtype, norm, norm_eps, 1.0f,
-                             ws + p.off_attn, p.attn_bytes, stream);
+    st = chela_linattn_fwd(qq, kk, vv, attn_out, B, H, L, d, d, chunk, CHELA_F32, attn_dtype, norm, norm_eps, 1.0f,
+                           ws + p.off_attn, p.attn_bytes, stream);
+    if (st != CHELA_OK || !gated) return st;
+    return launch_gate_combine((const float *)attn_out, ws + p.off_ga, ws + p.off_go, CHELA_F32, x, in_dtype, o, out_dtype, n,
+                               stream);
+}
+}  // namespace
+
+extern "C" {
+
+chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_width, const float *k_long,
+                               const void *w_q, const void *w_k, const void *w_v, const float *b_q,
+                               const float *b_k, const float *b_v, int qk_diag, int v_silu, void *o, int B,
+                               int L, int D, int H, int chunk, chela_dtype_t in_dtype,
+                               chela_dtype_t out_dtype, chela_norm_t norm, float norm_eps, void *workspace,
+                               size_t workspace_bytes, cudaStream_t stream)
+{
+    return mixer_impl(x, w_short, short_width, k_long, w_q, w_k, w_v, b_q, b_k, b_v, nullptr, nullptr, nullptr, nullptr,
+                      qk_diag, v_silu, o, B, L, D, H, chunk, in_dtype, out_dtype, norm, norm_eps, workspace, workspace_bytes,
+                      stream);
+}
+
+chela_status_t chela_mixer_gated_fwd(const void *x, const float *w_short, int short_width, const float *k_long,
+                                     const void *w_q, const void *w_k, const void *w_v, const float *b_q,
+                                     const float *b_k, const float *b_v, const void *w_a, const float *b_a,
+                                     const void *w_o, const float *b_o, int qk_diag, int v_silu, void *u, int B, int L,
+                                     int D, int H, int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                                     chela_norm_t norm, float norm_eps, void *workspace, size_t workspace_bytes,
+                                     cudaStream_t stream)
+{
+    if (!w_a || !w_o) return CHELA_ERR_INVALID_ARG;
+    return mixer_impl(x, w_short, short_width, k_long, w_q, w_k, w_v, b_q, b_k, b_v, w_a, b_a, w_o, b_o, qk_diag, v_silu, u,
+                      B, L, D, H, chunk, in_dtype, out_dtype, norm, norm_eps, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

@@ -17,6 +17,9 @@ inline size_t dtype_size(chela_dtype_t t) { return t == CHELA_F32 ? 4 : (t == CH
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 __device__ __forceinline__ float silu_f(float u) { return u / (1.0f + __expf(-u)); }
+__device__ __forceinline__ float sigmoid_f(float u) { return 1.0f / (1.0f + __expf(-u)); }
+// activation codes of the dense kernels: 0 identity, 1 SiLU, 2 sigmoid
+__device__ __forceinline__ float activate(float u, int act) { return act == 1 ? silu_f(u) : (act == 2 ? sigmoid_f(u) : u); }
 
 // Load / store 4 consecutive elements as fp32.
 __device__ __forceinline__ float4 load4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
@@ -86,5 +89,9 @@ chela_status_t launch_affine(const float *z, const void *alpha, const float *bet
 // the same on bf16 pairs ([2][M*D] bf16 in and out)
 chela_status_t launch_affine_pair(const void *z, const void *alpha, const float *beta, void *y, size_t M, int D,
                                   chela_dtype_t alpha_dtype, cudaStream_t stream);
+
+// u = o * g_a * g_o + x * (1 - g_o)  (Eqs. 8, 14); o fp32, gates fp32 or bf16 pairs, x and u in their own dtypes
+chela_status_t launch_gate_combine(const float *o, const void *g_a, const void *g_o, chela_dtype_t gate_dtype, const void *x,
+                                   chela_dtype_t x_dtype, void *u, chela_dtype_t u_dtype, size_t n, cudaStream_t stream);
 
 }  // namespace chela

@@ -56,7 +56,7 @@ gemm_simt_kernel(const TA *__restrict__ a, const TW *__restrict__ w, const float
             const int n = n0 + tn + j;
             if (n >= N) continue;
             float r = acc[i][j] + (bias ? bias[n] : 0.f);
-            if (act) r = silu_f(r);
+            if (act) r = activate(r, act);
             store1(y + m * N + n, r);
         }
     }
@@ -109,6 +109,46 @@ chela_status_t launch_affine_pair(const void *z, const void *alpha, const float 
         affine_pair_kernel<float><<<blocks, 256, 0, stream>>>((const __nv_bfloat16 *)z, (const float *)alpha, beta,
                                                               (__nv_bfloat16 *)y, n, D);
     return last_launch_status();
+}
+
+namespace {
+template <typename TG, typename TX, typename TU>
+__global__ void gate_combine_kernel(const float *__restrict__ o, const TG *__restrict__ g_a, const TG *__restrict__ g_o,
+                                    const TX *__restrict__ x, TU *__restrict__ u, size_t n, int pair)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float ga = load1(g_a + i), go = load1(g_o + i);
+        if (pair) {   // bf16 pair: low plane n elements later
+            ga += load1(g_a + n + i);
+            go += load1(g_o + n + i);
+        }
+        store1(u + i, fmaf(o[i] * ga, go, load1(x + i) * (1.0f - go)));
+    }
+}
+template <typename TG>
+chela_status_t gate_combine_t(const float *o, const void *g_a, const void *g_o, int pair, const void *x, chela_dtype_t x_dtype,
+                              void *u, chela_dtype_t u_dtype, size_t n, cudaStream_t stream)
+{
+    typedef __nv_bfloat16 bf;
+    const int blocks = (int)((n + 255) / 256 < 148 * 32 ? (n + 255) / 256 : 148 * 32);
+    const TG *ga = (const TG *)g_a, *go = (const TG *)g_o;
+    if (x_dtype == CHELA_BF16 && u_dtype == CHELA_BF16)
+        gate_combine_kernel<TG, bf, bf><<<blocks, 256, 0, stream>>>(o, ga, go, (const bf *)x, (bf *)u, n, pair);
+    else if (x_dtype == CHELA_BF16)
+        gate_combine_kernel<TG, bf, float><<<blocks, 256, 0, stream>>>(o, ga, go, (const bf *)x, (float *)u, n, pair);
+    else if (u_dtype == CHELA_BF16)
+        gate_combine_kernel<TG, float, bf><<<blocks, 256, 0, stream>>>(o, ga, go, (const float *)x, (bf *)u, n, pair);
+    else
+        gate_combine_kernel<TG, float, float><<<blocks, 256, 0, stream>>>(o, ga, go, (const float *)x, (float *)u, n, pair);
+    return last_launch_status();
+}
+}  // namespace
+
+chela_status_t launch_gate_combine(const float *o, const void *g_a, const void *g_o, chela_dtype_t gate_dtype, const void *x,
+                                   chela_dtype_t x_dtype, void *u, chela_dtype_t u_dtype, size_t n, cudaStream_t stream)
+{
+    if (gate_dtype == CHELA_BF16_PAIR) return gate_combine_t<__nv_bfloat16>(o, g_a, g_o, 1, x, x_dtype, u, u_dtype, n, stream);
+    return gate_combine_t<float>(o, g_a, g_o, 0, x, x_dtype, u, u_dtype, n, stream);
 }
 
 chela_status_t launch_gemm_simt(const void *a, const void *w, const float *bias, void *y, size_t M, int K,

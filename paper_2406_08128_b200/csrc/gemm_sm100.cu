@@ -184,8 +184,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                             x1 += bias[n0 + c * 64 + col + 1];
                         }
                         if (act) {
-                            x0 = silu_f(x0);
-                            x1 = silu_f(x1);
+                            x0 = activate(x0, act);
+                            x1 = activate(x1, act);
                         }
                         const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
                         wh[e] = *reinterpret_cast<const uint32_t *>(&hh);

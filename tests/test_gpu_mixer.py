@@ -66,3 +66,17 @@ def test_mixer_config3_shape_one_batch():
     got = run_mixer(m, H, 64)
     ref = oracle.mixer(m["x"], m["w_short"], m["k_long"], m["w_q"], m["w_k"], m["w_v"], H)
     assert rel_err(got, ref) <= TOL
+
+
+@pytest.mark.parametrize("B,L,D,H,chunk,dtype", [(2, 300, 128, 2, 64, "bf16"), (1, 1000, 256, 2, 128, "bf16"),
+                                                 (1, 2048, 512, 8, 64, "bf16"), (1, 200, 64, 1, 64, "f32")])
+def test_gated_mixer(B, L, D, H, chunk, dtype):
+    m = inputs.mixer(5, B, L, D, dtype=dtype)
+    rng = np.random.default_rng(6)
+    w_a, w_o = (inputs.round_storage(rng.standard_normal((D, D), dtype=np.float32) / np.sqrt(D) / 12, dtype) for _ in range(2))
+    b_a, b_o = (rng.standard_normal(D, dtype=np.float32) * 0.5 for _ in range(2))
+    dev = lambda a: to_device(a, dtype)
+    u = chela.mixer_gated_fwd(dev(m["x"]), dev_f32(m["w_short"]), dev_f32(m["k_long"]), dev(m["w_q"]), dev(m["w_k"]),
+                              dev(m["w_v"]), dev(w_a), dev(w_o), H, chunk=chunk, b_a=dev_f32(b_a), b_o=dev_f32(b_o))
+    ref = oracle.mixer_gated(m["x"], m["w_short"], m["k_long"], m["w_q"], m["w_k"], m["w_v"], w_a, w_o, H, b_a=b_a, b_o=b_o)
+    assert rel_err(to_numpy(u), ref) <= TOL

@@ -303,3 +303,30 @@ def test_mixer_head_split_is_contiguous_column_blocks():
     wq1 = np.zeros((D, D)); wq1[:, 2:4] = wq[:, 2:4]
     o = oracle.mixer(x, ws, kl, wq1, wk, rnd(63, D, D), H, v_silu=False, norm=False)
     assert list(np.nonzero(np.abs(o).sum(axis=(0, 1)))[0]) == [2, 3]
+
+
+# ---------------------------------------------------------------- gates (Eqs. 8, 9, 13, 14)
+
+def test_gated_mixer_limits_and_numpy_composition():
+    B, L, D, H = 2, 24, 8, 2
+    x, ws, kl = rnd(70, B, L, D), rnd(71, D, 3), rnd(72, D, L) * np.exp(-0.05 * np.arange(L))
+    wq, wk, wv, wa, wo = (rnd(s, D, D) / np.sqrt(D) for s in (73, 74, 75, 76, 77))
+    ba, bo = rnd(78, D), rnd(79, D)
+    o, z = oracle.mixer(x, ws, kl, wq, wk, wv, H, return_z=True)
+    u = oracle.mixer_gated(x, ws, kl, wq, wk, wv, wa, wo, H, b_a=ba, b_o=bo)
+    ga = z @ wa + ba
+    ga = ga / (1 + np.exp(-ga))
+    go = 1 / (1 + np.exp(-(z @ wo + bo)))
+    assert np.allclose(u, o * ga * go + x * (1 - go), atol=1e-10)
+    zero = np.zeros((D, D))
+    # output gate closed (b_o -> -inf): U = X exactly
+    closed = oracle.mixer_gated(x, ws, kl, wq, wk, wv, wa, zero, H, b_a=ba, b_o=np.full(D, -800.0))
+    assert np.array_equal(closed, x)
+    # output gate open, attention gate constant silu(b) = 1 (b = 1.2784645...): U = O
+    b1 = 1.2784645427610738
+    assert abs(b1 / (1 + np.exp(-b1)) - 1.0) < 1e-15
+    opened = oracle.mixer_gated(x, ws, kl, wq, wk, wv, zero, zero, H, b_a=np.full(D, b1), b_o=np.full(D, 800.0))
+    assert np.allclose(opened, o, atol=1e-13)
+    # zero gate weights and biases: G_a = silu(0) = 0 and G_o = 1/2, so U = X / 2
+    half = oracle.mixer_gated(x, ws, kl, wq, wk, wv, zero, zero, H)
+    assert np.allclose(half, 0.5 * x, atol=1e-15)
