@@ -110,8 +110,7 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
  *   S_{-1} = state_in (zero if NULL);  outputs as chela_linattn_fwd;  state_out = S after the last token.
  * Evaluating a sequence in consecutive segments with the state carried gives the result of one call over
  * the whole sequence (up to rounding).  state_in, state_out : [B, H, d_k, d_v] fp32, nullable, may alias
- * each other.  Supported: everything chela_linattn_fwd supports except bf16(-pair) inputs with d = 128
- * (CHELA_ERR_UNSUPPORTED; fp32 inputs with d = 128 are fine).
+ * each other.  Supported: everything chela_linattn_fwd supports.
  */
 chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void *v, void *o,
                                        const float *state_in, float *state_out,

@@ -111,7 +111,6 @@ chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void 
     const int kind = chela_linattn_kernel_kind(B, H, L, d_k, d_v, chunk, in_dtype, out_dtype);
     if (kind == 0) return CHELA_ERR_UNSUPPORTED;
     if (kind == 2) {
-        if (d_k == 128 && (state_in || state_out)) return CHELA_ERR_UNSUPPORTED;
         const size_t need = linattn_sm100_workspace_bytes(B, H, L, d_k, chunk);
         if (need && (!workspace || workspace_bytes < need)) return CHELA_ERR_WORKSPACE;
         return launch_linattn_sm100(q, k, v, o, B, H, L, d_k, chunk, in_dtype, out_dtype, (int)norm, norm_eps,

@@ -62,9 +62,11 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
                                     void *workspace, cudaStream_t stream, const float *state_in = nullptr,
                                     float *state_out = nullptr);
 
+size_t linattn_sm100_d128_workspace_bytes(int B, int H, int L);
 chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                                          chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
-                                         void *workspace, cudaStream_t stream);
+                                         void *workspace, cudaStream_t stream, const float *state_in = nullptr,
+                                         float *state_out = nullptr);
 
 chela_status_t launch_shortconv(const void *x, const float *w, const float *bias, void *y, int B, int L,
                                 int D, int width, int act, chela_dtype_t io_dtype, cudaStream_t stream);

@@ -634,7 +634,7 @@ bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_
 // per-group state sums [B*H][G-1][64][64] fp32 of a call that is split along L.
 size_t linattn_sm100_workspace_bytes(int B, int H, int L, int d, int)
 {
-    if (d == 128) return kWsHeader;   // the 128-wide kernel does not split sequences
+    if (d == 128) return linattn_sm100_d128_workspace_bytes(B, H, L);
     if (d != kD) return 0;
     const size_t a = split_plan(B, H, L, false).part_bytes, b = split_plan(B, H, L, true).part_bytes;
     return kWsHeader + (a > b ? a : b);   // the query does not know the input dtype: cover both plans
@@ -645,8 +645,9 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
                                     float scale, void *workspace, cudaStream_t stream, const float *state_in,
                                     float *state_out)
 {
-    if (d == 128 && (state_in || state_out)) return CHELA_ERR_UNSUPPORTED;   // the caller routes these elsewhere
-    if (d == 128) return launch_linattn_sm100_d128(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, workspace, stream);
+    if (d == 128)
+        return launch_linattn_sm100_d128(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, workspace, stream, state_in,
+                                         state_out);
     // The result does not depend on the chunk size: both supported values run on 64-token tiles.
     (void)chunk;
     if (in_dtype == CHELA_BF16_PAIR) {

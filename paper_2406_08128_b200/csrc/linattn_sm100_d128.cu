@@ -47,8 +47,11 @@ template <typename TOut, bool kPair>
 __global__ void __launch_bounds__(kThreads)
 linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
-                          float scale, int norm, float eps, int *__restrict__ status)
+                          float scale, int norm, float eps, int *__restrict__ status, const float *__restrict__ s_part, int G,
+                          int cpg, const float *__restrict__ state_in, float *__restrict__ state_out)
 {
+    // Grid: one CTA per (batch*head, group); group g covers chunks [g*cpg, (g+1)*cpg) and starts from
+    // state_in[bh] + sum_{g' < g} s_part[bh][g'] (128 x 128 fp32 each); the last group writes state_out[bh].
     using SM = Smem<TOut, kPair>;
     constexpr int kStages = SM::kStages, kPlanes = SM::kPlanes;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -58,8 +61,11 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         return;
     }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int b = blockIdx.x / H, h = blockIdx.x % H;
-    const int nchunks = (L + kC - 1) / kC;
+    const int bh = blockIdx.x / G, g = blockIdx.x % G;
+    const int b = bh / H, h = bh % H;
+    const int c0 = g * cpg;
+    const int nchunks = min(cpg, (L + kC - 1) / kC - c0);
+    const bool has_init = g > 0 || state_in != nullptr;
 
     const uint32_t bar_full0 = sbase + SM::offBar;
     const uint32_t bar_p = bar_full0 + 8 * kStages, bar_o = bar_p + 8, bar_pt = bar_o + 8, bar_s = bar_pt + 8;
@@ -101,9 +107,9 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 for (int pl = 0; pl < kPlanes; ++pl)
 #pragma unroll
                     for (int x = 0; x < 2; ++x) {
-                        tma_load_5d(tile(chunk, pl, 2 * x), &tm_q, bar, 64 * x, h, chunk * kC, b, pl);
-                        tma_load_5d(tile(chunk, pl, 2 * x + 1), &tm_k, bar, 64 * x, h, chunk * kC, b, pl);
-                        tma_load_5d(tile(chunk, pl, 4 + x), &tm_v, bar, 64 * x, h, chunk * kC, b, pl);
+                        tma_load_5d(tile(chunk, pl, 2 * x), &tm_q, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
+                        tma_load_5d(tile(chunk, pl, 2 * x + 1), &tm_k, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
+                        tma_load_5d(tile(chunk, pl, 4 + x), &tm_v, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
                     }
             };
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);
@@ -135,7 +141,7 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             bool ok = issue_scores(0);
             uint32_t par_s = 0;
             for (int i = 0; ok && i < nchunks; ++i) {
-                if (i > 0) {
+                if (i > 0 || has_init) {
                     ok = mbar_wait(bar_s, par_s, abort_flag);
                     par_s ^= 1;
                     if (!ok) break;
@@ -166,7 +172,7 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     const uint32_t v_hi = desc_lo(tile(i, 0, 4), kTile);
                     // OS_a: [P^T | K_a]; S_b: [P^T | K_b] with the lower lanes write-disabled
                     const uint32_t a_a = desc_lo(pt_hi, tile(i, 0, 1) - pt_hi), a_b = desc_lo(pt_hi, tile(i, 0, 3) - pt_hi);
-                    const uint32_t first = i > 0 ? 1u : 0u;
+                    const uint32_t first = (i > 0 || has_init) ? 1u : 0u;
 #pragma unroll
                     for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColOS, a_a + 128 * k, v_hi + 128 * k, idescG3, (first || k > 0) ? 1u : 0u);
 #pragma unroll
@@ -213,6 +219,58 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         const int r = tid & 63;
         const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
         bool ok = true;
+        // state rows of this thread: d_k = r (accumulator OS_a) and d_k = 64 + r (accumulator S_b); hi/lo tiles per
+        // d_v half: tile index 2*x + half, low part four tiles later
+        auto write_state_tiles = [&](const float(&sv)[64], int x, int half) {
+            uint8_t *sHi = smem + SM::offS + (2 * x + half) * kTile, *sLo = sHi + 4 * kTile;
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) {
+                uint32_t wh[4], wl[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float x0 = sv[c8 * 8 + e * 2], x1 = sv[c8 * 8 + e * 2 + 1];
+                    const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                    const float2 hf = __bfloat1622float2(hh);
+                    wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                    wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                }
+                const uint32_t off = sw128(r, c8);
+                *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+            }
+        };
+        if (has_init) {
+            if (upper) {
+#pragma unroll
+                for (int x = 0; x < 2; ++x)
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        float sv[64];
+#pragma unroll
+                        for (int j = 0; j < 64; ++j) sv[j] = 0.f;
+                        const size_t row_off = (size_t)(64 * x + r) * kD + 64 * half;
+                        auto add_row = [&](const float *base) {
+                            const float4 *src = reinterpret_cast<const float4 *>(base + row_off);
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float4 t = src[j];
+                                sv[4 * j] += t.x; sv[4 * j + 1] += t.y; sv[4 * j + 2] += t.z; sv[4 * j + 3] += t.w;
+                            }
+                        };
+                        if (state_in) add_row(state_in + (size_t)bh * kD * kD);
+                        for (int gp = 0; gp < g; ++gp) add_row(s_part + ((size_t)bh * (G - 1) + gp) * kD * kD);
+                        const uint32_t col = (x == 0 ? kColOS : kColSb) + 64 * half;
+                        tmem_st32(tmem_warp + col, *reinterpret_cast<const float(*)[32]>(&sv[0]));
+                        tmem_st32(tmem_warp + col + 32, *reinterpret_cast<const float(*)[32]>(&sv[32]));
+                        tmem_st_wait();
+                        write_state_tiles(sv, x, half);
+                    }
+                fence_proxy_async();
+                tc_fence_before();
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_s);
+        }
         for (int i = 0; i < nchunks; ++i) {
             if (upper) {
                 // ---- P^T_i: TMEM -> causal mask (t >= s) -> bf16 (pair) -> shared, rows = s ---------------
@@ -293,7 +351,7 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
 #pragma unroll
                     for (int bx = 0; bx < SM::kOBoxes; ++bx)
                         tma_store_5d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
-                                     i * kC + warp * 32, b, 0);
+                                     (c0 + i) * kC + warp * 32, b, 0);
                     bulk_commit();
                 }
             } else if (i + 1 < nchunks) {
@@ -307,27 +365,27 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                         tmem_ld32(tmem_warp + col, *reinterpret_cast<float(*)[32]>(&sv[0]));
                         tmem_ld32(tmem_warp + col + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
                         tmem_ld_wait();
-                        uint8_t *sHi = smem + SM::offS + (2 * x + half) * kTile, *sLo = sHi + 4 * kTile;
-#pragma unroll
-                        for (int c8 = 0; c8 < 8; ++c8) {
-                            uint32_t wh[4], wl[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float x0 = sv[c8 * 8 + e * 2], x1 = sv[c8 * 8 + e * 2 + 1];
-                                const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
-                                const float2 hf = __bfloat1622float2(hh);
-                                wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
-                                wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
-                            }
-                            const uint32_t off = sw128(r, c8);
-                            *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
-                            *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-                        }
+                        write_state_tiles(sv, x, half);
                     }
                 fence_proxy_async();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_s);
+            } else if (state_out && g == G - 1) {
+                // last chunk of the sequence: the fp32 state leaves the SM once, for the caller
+#pragma unroll
+                for (int x = 0; x < 2; ++x)
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        float sv[64];
+                        const uint32_t col = (x == 0 ? kColOS : kColSb) + 64 * half;
+                        tmem_ld32(tmem_warp + col, *reinterpret_cast<float(*)[32]>(&sv[0]));
+                        tmem_ld32(tmem_warp + col + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+                        tmem_ld_wait();
+                        float4 *dst = reinterpret_cast<float4 *>(state_out + (size_t)bh * kD * kD + (size_t)(64 * x + r) * kD + 64 * half);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) dst[j] = make_float4(sv[4 * j], sv[4 * j + 1], sv[4 * j + 2], sv[4 * j + 3]);
+                    }
             }
         }
         if (!ok && lane == 0) {
@@ -341,6 +399,134 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
+// Per-group state sums for sequences split along L: CTA (batch*head, g), g < G-1, writes
+// s_part[bh][g] = sum over the group's chunks of K_i^T V_i (128 x 128 fp32).  One accumulator, M = N = 128:
+// A = [K_a | K_b] (MN-major, the two d_k halves are adjacent tiles), B = [V_a | V_b].
+template <bool kPair>
+struct SmemState {
+    static constexpr int kStages = kPair ? 2 : 3;
+    static constexpr int kPlanes = kPair ? 2 : 1;
+    static constexpr int offStage = 0;                                        // per stage and plane: Ka Kb Va Vb
+    static constexpr int offBar = kStages * kPlanes * 4 * kTile;              // full[], empty[], done
+    static constexpr int offTmem = offBar + 8 * (2 * kStages + 1);
+    static constexpr int offAbort = offTmem + 8;
+    static constexpr int bytes = offAbort + 8;
+};
+
+template <bool kPair>
+__global__ void __launch_bounds__(kThreads)
+linattn_state_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                          float *__restrict__ s_part, int H, int G, int cpg, int *__restrict__ status)
+{
+    using SM = SmemState<kPair>;
+    constexpr int kStages = SM::kStages, kPlanes = SM::kPlanes;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t sbase = smem_u32(smem);
+    if (sbase & 1023u) {
+        if (threadIdx.x == 0) atomicExch(status, (int)CHELA_ERR_CUDA);
+        return;
+    }
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int bh = blockIdx.x / (G - 1), g = blockIdx.x % (G - 1);
+    const int b = bh / H, h = bh % H;
+    const int c0 = g * cpg, nchunks = cpg;
+    const uint32_t bar_full0 = sbase + SM::offBar, bar_empty0 = bar_full0 + 8 * kStages, bar_done = bar_empty0 + 8 * kStages;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full0 + 8 * s, 1);
+            mbar_init(bar_empty0 + 8 * s, 1);
+        }
+        mbar_init(bar_done, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    if (warp == 0) {
+        tmem_alloc(sbase + SM::offTmem, 128);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            auto tile = [&](int chunk, int pl, int t) { return sbase + SM::offStage + (((chunk % kStages) * kPlanes + pl) * 4 + t) * kTile; };
+            auto issue_load = [&](int chunk) {
+                const uint32_t bar = bar_full0 + 8 * (chunk % kStages);
+                mbar_expect_tx(bar, kPlanes * 4 * kTile);
+#pragma unroll
+                for (int pl = 0; pl < kPlanes; ++pl)
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        tma_load_5d(tile(chunk, pl, x), &tm_k, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
+                        tma_load_5d(tile(chunk, pl, 2 + x), &tm_v, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
+                    }
+            };
+            constexpr uint32_t idesc = make_idesc(128, 128, 1, 1);
+            int loads_issued = 0, consumed = 0;
+            for (; loads_issued < kStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued);
+            bool ok = true;
+            for (int i = 0; i < nchunks; ++i) {
+                const int stage = i % kStages;
+                ok = mbar_wait(bar_full0 + 8 * stage, (i / kStages) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t k_hi = desc_lo(tile(i, 0, 0), kTile), v_hi = desc_lo(tile(i, 0, 2), kTile);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_bf16(tmem, k_hi + 128 * k, v_hi + 128 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                if (kPair) {
+                    const uint32_t k_lo = desc_lo(tile(i, 1, 0), kTile), v_lo = desc_lo(tile(i, 1, 2), kTile);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16(tmem, k_hi + 128 * k, v_lo + 128 * k, idesc, 1);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16(tmem, k_lo + 128 * k, v_hi + 128 * k, idesc, 1);
+                }
+                umma_commit(bar_empty0 + 8 * stage);
+                consumed = i + 1;
+                if (i + kStages < nchunks) {
+                    ok = mbar_wait(bar_empty0 + 8 * stage, (i / kStages) & 1, abort_flag);
+                    if (!ok) break;
+                    issue_load(i + kStages);
+                    ++loads_issued;
+                }
+            }
+            if (ok) umma_commit(bar_done);
+            else {
+                *abort_flag = 1;
+                atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+                for (int c = consumed; c < loads_issued; ++c) mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1, nullptr);
+            }
+        }
+    } else {
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_done, 0, abort_flag));
+        if (ok) {
+            tc_fence_after();
+            const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
+            float4 *dst = reinterpret_cast<float4 *>(s_part + (((size_t)bh * (G - 1) + g) * kD + tid) * kD);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                float sv[64];
+                tmem_ld32(tmem_warp + 64 * half, *reinterpret_cast<float(*)[32]>(&sv[0]));
+                tmem_ld32(tmem_warp + 64 * half + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) dst[16 * half + j] = make_float4(sv[4 * j], sv[4 * j + 1], sv[4 * j + 2], sv[4 * j + 3]);
+            }
+        } else if (lane == 0) {
+            *abort_flag = 1;
+            atomicExch(status, (int)CHELA_ERR_TIMEOUT);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 128);
+}
+
 bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int box_rows, bool f32, int planes)
 {
     const cuuint64_t es = f32 ? 4 : 2;
@@ -351,36 +537,74 @@ bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int box_ro
     return make_map_sw128(map, ptr, f32, 5, dims, strides, box);
 }
 
+// Split along L: one CTA per SM is resident (shared memory), at least 16 chunks per group.
+struct SplitPlan {
+    int G, cpg;
+    size_t part_bytes;
+};
+SplitPlan split_plan(int B, int H, int L)
+{
+    int sms = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+    const long long bh = (long long)B * H;
+    const int nchunks = (L + kC - 1) / kC;
+    int G = 1;
+    if (bh * 2 <= sms) {
+        G = (int)(sms / bh);
+        if (G > nchunks / 16) G = nchunks / 16;
+        if (G < 1) G = 1;
+    }
+    SplitPlan p;
+    p.cpg = (nchunks + G - 1) / G;
+    p.G = (nchunks + p.cpg - 1) / p.cpg;
+    p.part_bytes = (size_t)bh * (p.G - 1) * kD * kD * sizeof(float);
+    return p;
+}
+constexpr size_t kWsHeader = 512;
+
 template <typename TOut, bool kPair>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
-                        float scale, int *status, cudaStream_t stream)
+                        float scale, void *workspace, const float *state_in, float *state_out, cudaStream_t stream)
 {
     CUtensorMap mq, mk, mv, mo;
     const int planes = kPair ? 2 : 1;
     if (!make_map(&mq, q, B, H, L, kC, false, planes) || !make_map(&mk, k, B, H, L, kC, false, planes) ||
         !make_map(&mv, v, B, H, L, kC, false, planes) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4, 1))
         return CHELA_ERR_CUDA;
+    int *status = (int *)workspace;
+    float *s_part = (float *)((char *)workspace + kWsHeader);
+    const SplitPlan plan = split_plan(B, H, L);
     if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+    if (plan.G > 1) {
+        auto skern = linattn_state_d128_kernel<kPair>;
+        if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemState<kPair>::bytes) != cudaSuccess)
+            return CHELA_ERR_CUDA;
+        skern<<<B * H * (plan.G - 1), kThreads, SmemState<kPair>::bytes, stream>>>(mk, mv, s_part, H, plan.G, plan.cpg, status);
+        if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
+    }
     auto kern = linattn_sm100_d128_kernel<TOut, kPair>;
     const int smem = Smem<TOut, kPair>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
-    kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status);
+    kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg,
+                                                     state_in, state_out);
     return last_launch_status();
 }
 
 }  // namespace
 
+size_t linattn_sm100_d128_workspace_bytes(int B, int H, int L) { return kWsHeader + split_plan(B, H, L).part_bytes; }
+
 chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                                          chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
-                                         void *workspace, cudaStream_t stream)
+                                         void *workspace, cudaStream_t stream, const float *state_in, float *state_out)
 {
-    int *status = (int *)workspace;
     if (in_dtype == CHELA_BF16_PAIR) {
-        if (out_dtype == CHELA_F32) return launch_t<float, true>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
-        return launch_t<__nv_bfloat16, true>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+        if (out_dtype == CHELA_F32) return launch_t<float, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+        return launch_t<__nv_bfloat16, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
     }
-    if (out_dtype == CHELA_F32) return launch_t<float, false>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
-    return launch_t<__nv_bfloat16, false>(q, k, v, o, B, H, L, norm, eps, scale, status, stream);
+    if (out_dtype == CHELA_F32) return launch_t<float, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+    return launch_t<__nv_bfloat16, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
 }
 
 }  // namespace chela

@@ -95,6 +95,14 @@ def test_sweep_shapes_sampled(B, L):
     assert bool(torch.isfinite(o).all())
 
 
+@pytest.mark.parametrize("B,L,H", [(1, 8192, 2), (1, 5000, 3), (1, 2100, 1)])
+def test_sequences_split_along_length_head_dim_128(B, L, H):
+    q, k, v = inputs.qkv(45 + L, B, L, H, 128, 128, "bf16")
+    assert chela.linattn_workspace_bytes(B, H, L, 128, 128, 64) >= 512 + 128 * 128 * 4
+    got = run(q, k, v, "bf16", 128)
+    assert rel_err(got, oracle.linattn_recurrent(q, k, v)) <= TOL["bf16"]
+
+
 @pytest.mark.parametrize("B,L,H", [(1, 8192, 2), (1, 5000, 3), (1, 2100, 1), (2, 4096, 1)])
 def test_sequences_split_along_length(B, L, H):
     """Few (batch, head) pairs: the tensor-core path splits each sequence into groups of chunks whose
