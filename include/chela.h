@@ -70,6 +70,18 @@ chela_status_t chela_shortconv_fwd(const void *x, const float *w, const float *b
                                    chela_dtype_t io_dtype, cudaStream_t stream);
 
 /*
+ * Structural re-parameterisation of parallel short kernels (Sec. 4.2): two depthwise causal kernels applied
+ * to the same input and summed before the activation are one kernel whose taps are the zero-padded sum,
+ *   conv(x; w1) + conv(x; w2) = conv(x; merged),  merged[c][j] = w1[c][j] (j < width1) + w2[c][j] (j < width2),
+ * aligned at lag 0.  w1 : [D, width1], w2 : [D, width2], merged : [D, max(width1, width2)], all fp32 device
+ * pointers.  chela_second_short_width gives the paper's length-dependent width 2 log10(L) + 1, rounded to the
+ * nearest odd integer (the paper's value is not an integer in general) and clamped to [1, 15].
+ */
+int chela_second_short_width(int L);
+chela_status_t chela_shortconv_reparam(const float *w1, int width1, const float *w2, int width2, float *merged, int D,
+                                       cudaStream_t stream);
+
+/*
  * Long convolution (Eq. 6, Sec. 2.2), optionally preceded by the short convolution + SiLU so
  * that the whole of Eq. 7 is one call:
  *   a = (w_short ? silu(shortconv(x; w_short)) : x) ;  z[b,t,c] = sum_{s=0}^{t} k_long[c,s] * a[b,t-s,c].

@@ -30,6 +30,8 @@ _SIGNATURES = {
     "chela_version": (_c_int, []),
     "chela_linattn_kernel_kind": (_c_int, [_c_int] * 6 + [_c_int, _c_int]),
     "chela_shortconv_fwd": (_c_int, [_vp, _vp, _vp, _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _vp]),
+    "chela_second_short_width": (_c_int, [_c_int]),
+    "chela_shortconv_reparam": (_c_int, [_vp, _c_int, _vp, _c_int, _vp, _c_int, _vp]),
     "chela_longconv_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int, _c_int, _c_int]),
     "chela_longconv_fwd": (_c_int, [_vp, _vp, _vp, _c_int, _vp, _c_int, _c_int, _c_int, _c_int, _c_int,
                                     _vp, _c_size_t, _vp]),
@@ -125,6 +127,20 @@ def shortconv_fwd(x, w, bias=None, act=True, out=None):
     _check(lib().chela_shortconv_fwd(_ptr(x), _ptr(w), _ptr(bias), _ptr(y), B, L, D, w.shape[1], int(bool(act)),
                                      _dt(x), _stream()), "chela_shortconv_fwd")
     return y
+
+
+def second_short_width(L: int) -> int:
+    """Width of the length-dependent short kernel, 2 log10(L) + 1 rounded to the nearest odd integer."""
+    return int(lib().chela_second_short_width(int(L)))
+
+
+def shortconv_reparam(w1, w2):
+    """Merge two parallel short kernels [D,width1], [D,width2] (fp32) into one [D,max(width)] kernel."""
+    D = w1.shape[0]
+    merged = torch.empty((D, max(w1.shape[1], w2.shape[1])), dtype=torch.float32, device=w1.device)
+    _check(lib().chela_shortconv_reparam(_ptr(w1), w1.shape[1], _ptr(w2), w2.shape[1], _ptr(merged), D, _stream()),
+           "chela_shortconv_reparam")
+    return merged
 
 
 def longconv_workspace_bytes(B, L, D, in_dtype=BF16, out_dtype=F32) -> int:

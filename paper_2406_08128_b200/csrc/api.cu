@@ -1,4 +1,6 @@
 // C ABI entry points: argument validation, workspace carving and dispatch.  No kernel code here.
+#include <cmath>
+
 #include "common.cuh"
 
 using namespace chela;
@@ -66,6 +68,24 @@ chela_status_t chela_shortconv_fwd(const void *x, const float *w, const float *b
     if (!aligned16(x) || !aligned16(y)) return CHELA_ERR_INVALID_ARG;
     if (width < 1 || width > 16 || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
     return launch_shortconv(x, w, bias, y, B, L, D, width, act, io_dtype, stream);
+}
+
+int chela_second_short_width(int L)
+{
+    if (L < 1) return 1;
+    const double w = 2.0 * log10((double)L) + 1.0;
+    int odd = 2 * (int)floor(w / 2.0) + 1;   // odd integers around w: odd <= w < odd + 2 (or odd - 2 < w)
+    if (w - odd > odd + 2 - w) odd += 2;
+    if (odd - w > w - (odd - 2)) odd -= 2;
+    return odd < 1 ? 1 : (odd > 15 ? 15 : odd);
+}
+
+chela_status_t chela_shortconv_reparam(const float *w1, int width1, const float *w2, int width2, float *merged, int D,
+                                       cudaStream_t stream)
+{
+    if (!w1 || !w2 || !merged || D < 1 || width1 < 1 || width2 < 1) return CHELA_ERR_INVALID_ARG;
+    if (width1 > 16 || width2 > 16) return CHELA_ERR_UNSUPPORTED;
+    return launch_shortconv_reparam(w1, width1, w2, width2, merged, D, stream);
 }
 
 size_t chela_longconv_workspace_bytes(int B, int L, int D, chela_dtype_t, chela_dtype_t)

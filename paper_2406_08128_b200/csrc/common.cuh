@@ -71,6 +71,9 @@ chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const voi
 chela_status_t launch_shortconv(const void *x, const float *w, const float *bias, void *y, int B, int L,
                                 int D, int width, int act, chela_dtype_t io_dtype, cudaStream_t stream);
 
+chela_status_t launch_shortconv_reparam(const float *w1, int width1, const float *w2, int width2, float *merged, int D,
+                                        cudaStream_t stream);
+
 size_t longconv_workspace_bytes(int B, int L, int D);
 chela_status_t launch_longconv(const void *x, const float *k_long, const float *w_short, int short_width,
                                void *z, int B, int L, int D, chela_dtype_t in_dtype,

@@ -619,6 +619,26 @@ chela_status_t launch_shortconv(const void *x, const float *w, const float *bias
 }
 
 namespace {
+__global__ void reparam_kernel(const float *__restrict__ w1, int width1, const float *__restrict__ w2, int width2,
+                               float *__restrict__ merged, int D)
+{
+    const int wm = max(width1, width2);
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= D * wm) return;
+    const int c = i / wm, j = i % wm;
+    merged[i] = (j < width1 ? w1[c * width1 + j] : 0.f) + (j < width2 ? w2[c * width2 + j] : 0.f);
+}
+}  // namespace
+
+chela_status_t launch_shortconv_reparam(const float *w1, int width1, const float *w2, int width2, float *merged, int D,
+                                        cudaStream_t stream)
+{
+    const int n = D * (width1 > width2 ? width1 : width2);
+    reparam_kernel<<<(n + 255) / 256, 256, 0, stream>>>(w1, width1, w2, width2, merged, D);
+    return last_launch_status();
+}
+
+namespace {
 struct LongconvPlan {
     int M, logM, Ls;
     size_t off_at, off_tw, off_spec, total;

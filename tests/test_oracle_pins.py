@@ -330,3 +330,13 @@ def test_gated_mixer_limits_and_numpy_composition():
     # zero gate weights and biases: G_a = silu(0) = 0 and G_o = 1/2, so U = X / 2
     half = oracle.mixer_gated(x, ws, kl, wq, wk, wv, zero, zero, H)
     assert np.allclose(half, 0.5 * x, atol=1e-15)
+
+
+def test_parallel_short_kernels_equal_one_merged_kernel():
+    """Structural re-parameterisation (Sec. 4.2) is linear in the taps: pinned on the oracle's short conv."""
+    B, L, D = 2, 50, 4
+    x, w3, w9 = rnd(80, B, L, D), rnd(81, D, 3), rnd(82, D, 9)
+    merged = w9.copy()
+    merged[:, :3] += w3
+    both = oracle.shortconv(x, w3, act=False) + oracle.shortconv(x, w9, act=False)
+    assert np.allclose(oracle.shortconv(x, merged, act=False), both, atol=1e-13)
