@@ -170,3 +170,13 @@ def mixer_gated(x, w_short, k_long, w_q, w_k, w_v, w_a, w_o, H, b_q=None, b_k=No
                                int(bool(v_silu)), _p(u), B, L, D, H, int(bool(norm)), ctypes.c_double(eps),
                                int(bool(use_fft)))
     return u
+
+
+def linattn_backward(q, k, v, d_o, scale=1.0, norm=True, eps=1e-6):
+    """Gradients (dq, dk, dv) of causal linear attention for the output gradient d_o, by the O(L^2) definition."""
+    q, k, v, B, L, H, dk, dv = _shape_qkv(q, k, v)
+    d_o = _f64(d_o)
+    dq, dk_, dv_ = np.empty_like(q), np.empty_like(k), np.empty_like(v)
+    _load().oracle_linattn_backward(_p(q), _p(k), _p(v), _p(d_o), _p(dq), _p(dk_), _p(dv_), B, H, L, dk, dv,
+                                    ctypes.c_double(scale), int(bool(norm)), ctypes.c_double(eps))
+    return dq, dk_, dv_

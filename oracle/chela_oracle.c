@@ -351,3 +351,75 @@ void oracle_mixer_gated(const double *x, const double *w_short, int width, const
     }
     free(o); free(z); free(ga); free(go);
 }
+
+/* Backward of causal linear attention, written from the definition (Eq. 2 with the causal mask and the
+ * row normaliser): for a loss with gradient d_o[t] with respect to o_t,
+ *   r_t = scale * sum_{s<=t} <q_t,k_s> v_s,  n_t = sqrt(mean_j r_tj^2 + eps),  o_t = r_t / n_t
+ *   g_t = dLoss/dr_t = (d_o[t] - o_t * <o_t, d_o[t]> / d_v) / n_t          (g_t = d_o[t] without the normaliser)
+ *   dq_t = scale * sum_{s<=t} <g_t,v_s> k_s
+ *   dk_s = scale * sum_{t>=s} <g_t,v_s> q_t
+ *   dv_s = scale * sum_{t>=s} <q_t,k_s> g_t
+ * Plain O(L^2) loops per (batch, head). */
+void oracle_linattn_backward(const double *q, const double *k, const double *v, const double *d_o,
+                             double *dq, double *dk_out, double *dv_out,
+                             int B, int H, int L, int dk, int dv, double scale, int norm, double eps)
+{
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            double *g = (double *)malloc(sizeof(double) * (size_t)L * dv);
+            double *r = (double *)malloc(sizeof(double) * dv);
+            for (int t = 0; t < L; ++t) {
+                for (int j = 0; j < dv; ++j) r[j] = 0.0;
+                const double *qt = q + IDX_QK(b, t, h);
+                for (int s = 0; s <= t; ++s) {
+                    const double *ks = k + IDX_QK(b, s, h);
+                    double a = 0.0;
+                    for (int i = 0; i < dk; ++i) a += qt[i] * ks[i];
+                    const double *vs = v + IDX_V(b, s, h);
+                    for (int j = 0; j < dv; ++j) r[j] += scale * a * vs[j];
+                }
+                const double *dot = d_o + IDX_V(b, t, h);
+                double *gt = g + (size_t)t * dv;
+                if (norm) {
+                    double ss = 0.0, od = 0.0;
+                    for (int j = 0; j < dv; ++j) ss += r[j] * r[j];
+                    double n = sqrt(ss / (double)dv + eps);
+                    for (int j = 0; j < dv; ++j) od += (r[j] / n) * dot[j];
+                    for (int j = 0; j < dv; ++j) gt[j] = (dot[j] - (r[j] / n) * od / (double)dv) / n;
+                } else {
+                    for (int j = 0; j < dv; ++j) gt[j] = dot[j];
+                }
+            }
+            for (int t = 0; t < L; ++t) {
+                double *dqt = dq + IDX_QK(b, t, h);
+                for (int i = 0; i < dk; ++i) dqt[i] = 0.0;
+                for (int s = 0; s <= t; ++s) {
+                    const double *vs = v + IDX_V(b, s, h);
+                    const double *ks = k + IDX_QK(b, s, h);
+                    double c = 0.0;
+                    for (int j = 0; j < dv; ++j) c += g[(size_t)t * dv + j] * vs[j];
+                    for (int i = 0; i < dk; ++i) dqt[i] += scale * c * ks[i];
+                }
+            }
+            for (int s = 0; s < L; ++s) {
+                double *dks = dk_out + IDX_QK(b, s, h);
+                double *dvs = dv_out + IDX_V(b, s, h);
+                for (int i = 0; i < dk; ++i) dks[i] = 0.0;
+                for (int j = 0; j < dv; ++j) dvs[j] = 0.0;
+                const double *vs = v + IDX_V(b, s, h);
+                const double *ks = k + IDX_QK(b, s, h);
+                for (int t = s; t < L; ++t) {
+                    const double *qt = q + IDX_QK(b, t, h);
+                    const double *gt = g + (size_t)t * dv;
+                    double c = 0.0, a = 0.0;
+                    for (int j = 0; j < dv; ++j) c += gt[j] * vs[j];
+                    for (int i = 0; i < dk; ++i) a += qt[i] * ks[i];
+                    for (int i = 0; i < dk; ++i) dks[i] += scale * c * qt[i];
+                    for (int j = 0; j < dv; ++j) dvs[j] += scale * a * gt[j];
+                }
+            }
+            free(g);
+            free(r);
+        }
+}

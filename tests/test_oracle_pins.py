@@ -340,3 +340,38 @@ def test_parallel_short_kernels_equal_one_merged_kernel():
     merged[:, :3] += w3
     both = oracle.shortconv(x, w3, act=False) + oracle.shortconv(x, w9, act=False)
     assert np.allclose(oracle.shortconv(x, merged, act=False), both, atol=1e-13)
+
+
+# ---------------------------------------------------------------- backward (finite differences)
+
+@pytest.mark.parametrize("norm", [False, True])
+def test_backward_matches_central_finite_differences(norm):
+    B, L, H, dk, dv = 1, 7, 2, 3, 4
+    q, k, v, w = rnd(90, B, L, H, dk), rnd(91, B, L, H, dk), rnd(92, B, L, H, dv), rnd(93, B, L, H, dv)
+    loss = lambda q_, k_, v_: float((oracle.linattn_quadratic(q_, k_, v_, scale=0.7, norm=norm, eps=1e-3) * w).sum())
+    dq, dk_, dv_ = oracle.linattn_backward(q, k, v, w, scale=0.7, norm=norm, eps=1e-3)
+    h = 1e-6
+    for arr, grad, which in ((q, dq, 0), (k, dk_, 1), (v, dv_, 2)):
+        fd = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            args_p, args_m = [q.copy(), k.copy(), v.copy()], [q.copy(), k.copy(), v.copy()]
+            args_p[which][idx] += h
+            args_m[which][idx] -= h
+            fd[idx] = (loss(*args_p) - loss(*args_m)) / (2 * h)
+        assert np.abs(fd - grad).max() <= 1e-6 * max(1.0, np.abs(grad).max())
+
+
+def test_backward_is_causal_and_linear_in_the_output_gradient():
+    B, L, H, d = 1, 20, 1, 4
+    q, k, v, g1, g2 = (rnd(s, B, L, H, d) for s in (94, 95, 96, 97, 98))
+    a = oracle.linattn_backward(q, k, v, g1, norm=False)
+    b = oracle.linattn_backward(q, k, v, g2, norm=False)
+    c = oracle.linattn_backward(q, k, v, 2 * g1 - g2, norm=False)
+    for x, y, z in zip(a, b, c):
+        assert np.allclose(z, 2 * x - y, atol=1e-12)
+    # an output gradient that is non-zero only at token t0 reaches keys/values at s <= t0 and the query at t0 only
+    t0 = 8
+    g = np.zeros((B, L, H, d)); g[:, t0] = 1.0
+    dq, dk_, dv_ = oracle.linattn_backward(q, k, v, g, norm=True)
+    assert np.all(dq[:, :t0] == 0) and np.all(dq[:, t0 + 1:] == 0) and np.any(dq[:, t0] != 0)
+    assert np.all(dk_[:, t0 + 1:] == 0) and np.all(dv_[:, t0 + 1:] == 0) and np.any(dk_[:, :t0 + 1] != 0)
