@@ -132,6 +132,21 @@ chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void 
                                        void *workspace, size_t workspace_bytes, cudaStream_t stream);
 
 /*
+ * Backward of chela_linattn_fwd (gradients of Eq. 2 with the causal mask and the row normaliser; the
+ * chunked evaluation of Sec. 4.1 run in both directions): given d_o = dLoss/do,
+ *   dq_t = scale sum_{s<=t} <g_t,v_s> k_s,  dk_s = scale sum_{t>=s} <g_t,v_s> q_t,  dv_s = scale sum_{t>=s} <q_t,k_s> g_t,
+ * with g_t = d_o[t] pulled back through the normaliser (g_t = d_o[t] for CHELA_NORM_NONE).  Nothing saved by the
+ * forward pass is needed: the pre-normaliser output is recomputed.
+ * q, k, v, d_o : [B, L, H, d] in_dtype (F32 or BF16).  dq, dk, dv : [B, L, H, d] fp32.
+ * Supported: d_k = d_v in {64, 128}.  fp32 SIMT kernel (a tensor-core version is future work).
+ */
+size_t chela_linattn_bwd_workspace_bytes(int B, int H, int L, int d_k, int d_v);
+chela_status_t chela_linattn_bwd(const void *q, const void *k, const void *v, const void *d_o,
+                                 float *dq, float *dk, float *dv, int B, int H, int L, int d_k, int d_v,
+                                 chela_dtype_t in_dtype, chela_norm_t norm, float norm_eps, float scale,
+                                 void *workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/*
  * Dense projection with optional SiLU, the building block of the Q/K/V formation (Eq. 12; Eqs. 10-11 in
  * their dense form): y = act(a w + bias), fp32 accumulation.
  * a : [M, K], a_dtype in {F32, BF16, BF16_PAIR}.  w : [K, N] row-major, w_dtype in {F32, BF16}.

@@ -40,6 +40,8 @@ _SIGNATURES = {
                                    _c_float, _vp, _c_size_t, _vp]),
     "chela_linattn_carry_fwd": (_c_int, [_vp, _vp, _vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                          _c_float, _vp, _c_size_t, _vp]),
+    "chela_linattn_bwd_workspace_bytes": (_c_size_t, [_c_int] * 5),
+    "chela_linattn_bwd": (_c_int, [_vp] * 7 + [_c_int] * 5 + [_c_int, _c_int, _c_float, _c_float, _vp, _c_size_t, _vp]),
     "chela_dense_workspace_bytes": (_c_size_t, []),
     "chela_dense_fwd": (_c_int, [_vp, _vp, _vp, _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _vp,
                                  _c_size_t, _vp]),
@@ -195,6 +197,19 @@ def linattn_carry_fwd(q, k, v, state_in=None, chunk=64, out_dtype=F32, norm=NORM
                                          d_k, d_v, chunk, in_dtype, _dt(o), int(norm), float(eps), float(scale),
                                          _ptr(workspace), workspace.numel(), _stream()), "chela_linattn_carry_fwd")
     return o, state_out
+
+
+def linattn_bwd(q, k, v, d_o, norm=NORM_RMS, eps=1e-6, scale=1.0, workspace=None):
+    """Gradients (dq, dk, dv), fp32, of linattn_fwd for the output gradient d_o (same dtype as q)."""
+    B, L, H, d_k = q.shape
+    d_v = v.shape[3]
+    dq, dk, dv = (torch.empty(t.shape, dtype=torch.float32, device=q.device) for t in (q, k, v))
+    if workspace is None:
+        workspace = _workspace(int(lib().chela_linattn_bwd_workspace_bytes(B, H, L, d_k, d_v)), q.device)
+    _check(lib().chela_linattn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, L, d_k, d_v,
+                                   _dt(q), int(norm), float(eps), float(scale), _ptr(workspace), workspace.numel(),
+                                   _stream()), "chela_linattn_bwd")
+    return dq, dk, dv
 
 
 def linattn_fwd_static_ws(q, k, v, chunk=64, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale=1.0, out=None):

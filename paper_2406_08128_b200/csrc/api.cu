@@ -149,6 +149,29 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
                                    norm_eps, scale, workspace, workspace_bytes, stream);
 }
 
+size_t chela_linattn_bwd_workspace_bytes(int B, int H, int L, int d_k, int d_v)
+{
+    if (B < 1 || H < 1 || L < 1 || d_k != d_v || (d_k != 64 && d_k != 128)) return 0;
+    return linattn_bwd_workspace_bytes(B, H, L, d_k);
+}
+
+chela_status_t chela_linattn_bwd(const void *q, const void *k, const void *v, const void *d_o, float *dq, float *dk,
+                                 float *dv, int B, int H, int L, int d_k, int d_v, chela_dtype_t in_dtype,
+                                 chela_norm_t norm, float norm_eps, float scale, void *workspace, size_t workspace_bytes,
+                                 cudaStream_t stream)
+{
+    if (!q || !k || !v || !d_o || !dq || !dk || !dv || B < 1 || H < 1 || L < 1 || !dtype_ok(in_dtype) ||
+        (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) || !(norm_eps >= 0.f))
+        return CHELA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) ||
+        !aligned16(dv) || !aligned16(workspace))
+        return CHELA_ERR_INVALID_ARG;
+    if (d_k != d_v || (d_k != 64 && d_k != 128)) return CHELA_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < linattn_bwd_workspace_bytes(B, H, L, d_k)) return CHELA_ERR_WORKSPACE;
+    return launch_linattn_bwd_simt(q, k, v, d_o, dq, dk, dv, B, H, L, d_k, in_dtype, (int)norm, norm_eps, scale, workspace,
+                                   stream);
+}
+
 size_t chela_dense_workspace_bytes(void) { return 256; }
 
 chela_status_t chela_dense_fwd(const void *a, const void *w, const float *bias, void *y, int M, int K, int N, int act,

@@ -68,6 +68,12 @@ chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const voi
                                          void *workspace, cudaStream_t stream, const float *state_in = nullptr,
                                          float *state_out = nullptr);
 
+// backward of causal linear attention (fp32 SIMT); gradients fp32; workspace = one [B,L,H,d] fp32 buffer
+size_t linattn_bwd_workspace_bytes(int B, int H, int L, int d);
+chela_status_t launch_linattn_bwd_simt(const void *q, const void *k, const void *v, const void *d_o, float *dq, float *dk,
+                                       float *dv, int B, int H, int L, int d, chela_dtype_t in_dtype, int norm, float eps,
+                                       float scale, void *workspace, cudaStream_t stream);
+
 chela_status_t launch_shortconv(const void *x, const float *w, const float *bias, void *y, int B, int L,
                                 int D, int width, int act, chela_dtype_t io_dtype, cudaStream_t stream);
 
