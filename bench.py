@@ -431,6 +431,16 @@ def main():
                                                                               chela.BF16_PAIR)})
             del x, k_l, mws, mo
         line["mixer"] = mixers
+        # ---- backward of the timed workload (gradients w.r.t. Q, K, V; normaliser on) ----------------------------
+        (q_, k_, v_), _ = views(L_MAIN)
+        d_o = (torch.randn(q_.shape, device=dev, generator=gen)).to(torch.bfloat16)
+        bws = torch.zeros(int(chela.lib().chela_linattn_bwd_workspace_bytes(q_.shape[0], H, L_MAIN, D, D)), dtype=torch.uint8, device=dev)
+        ms = timed(lambda: chela.linattn_bwd(q_, k_, v_, d_o, workspace=bws), 3, warm=1)
+        if chela.async_status(bws) != chela.OK:
+            raise RuntimeError("device-side wait timed out in the backward pass")
+        line["backward"] = {"ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
+                            "note": "chela_linattn_bwd, bf16 in, fp32 gradients, same workload as the timed step"}
+        del d_o, bws
         # ---- CPU oracle on the host cores, bounded sample -----------------------------------------------
         import oracle
         oracle.build()
