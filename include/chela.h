@@ -138,7 +138,7 @@ chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void 
  * with g_t = d_o[t] pulled back through the normaliser (g_t = d_o[t] for CHELA_NORM_NONE).  Nothing saved by the
  * forward pass is needed: the pre-normaliser output is recomputed.
  * q, k, v, d_o : [B, L, H, d] in_dtype (F32 or BF16).  dq, dk, dv : [B, L, H, d] fp32.
- * Supported: d_k = d_v in {64, 128}.  bf16 inputs with d = 64 run on the tensor cores: the three gradients are
+ * Supported: d_k = d_v in {64, 128}.  bf16 inputs run on the tensor cores: the three gradients are
  * linear attentions with the operands' roles exchanged, evaluated by the forward kernel (two of them in its
  * anti-causal mode) on g rounded to bf16; everything else runs on an fp32 SIMT kernel.  The workspace word 0 is
  * the asynchronous status of the tensor-core launches (chela_async_status).

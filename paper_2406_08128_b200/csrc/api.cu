@@ -153,7 +153,7 @@ size_t chela_linattn_bwd_workspace_bytes(int B, int H, int L, int d_k, int d_v)
 {
     if (B < 1 || H < 1 || L < 1 || d_k != d_v || (d_k != 64 && d_k != 128)) return 0;
     const size_t simt = linattn_bwd_workspace_bytes(B, H, L, d_k);
-    const size_t tensor = d_k == 64 ? linattn_bwd_sm100_workspace_bytes(B, H, L) : 0;   // the query does not know the dtype
+    const size_t tensor = linattn_bwd_sm100_workspace_bytes(B, H, L, d_k);   // the query does not know the dtype
     return simt > tensor ? simt : tensor;
 }
 
@@ -171,7 +171,7 @@ chela_status_t chela_linattn_bwd(const void *q, const void *k, const void *v, co
     if (d_k != d_v || (d_k != 64 && d_k != 128)) return CHELA_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < chela_linattn_bwd_workspace_bytes(B, H, L, d_k, d_v)) return CHELA_ERR_WORKSPACE;
     if (linattn_bwd_sm100_supported(d_k, in_dtype))
-        return launch_linattn_bwd_sm100(q, k, v, d_o, dq, dk, dv, B, H, L, (int)norm, norm_eps, scale, workspace, stream);
+        return launch_linattn_bwd_sm100(q, k, v, d_o, dq, dk, dv, B, H, L, d_k, (int)norm, norm_eps, scale, workspace, stream);
     return launch_linattn_bwd_simt(q, k, v, d_o, dq, dk, dv, B, H, L, d_k, in_dtype, (int)norm, norm_eps, scale, workspace,
                                    stream);
 }

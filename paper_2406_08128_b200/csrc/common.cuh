@@ -66,7 +66,7 @@ size_t linattn_sm100_d128_workspace_bytes(int B, int H, int L);
 chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                                          chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
                                          void *workspace, cudaStream_t stream, const float *state_in = nullptr,
-                                         float *state_out = nullptr);
+                                         float *state_out = nullptr, bool reverse = false, int pair_mask = 7);
 
 // backward of causal linear attention (fp32 SIMT); gradients fp32; workspace = one [B,L,H,d] fp32 buffer
 size_t linattn_bwd_workspace_bytes(int B, int H, int L, int d);
@@ -76,10 +76,10 @@ chela_status_t launch_linattn_bwd_simt(const void *q, const void *k, const void 
 
 // tensor-core backward (bf16, d = 64): four launches of the forward kernel plus an elementwise kernel
 bool linattn_bwd_sm100_supported(int d, chela_dtype_t in_dtype);
-size_t linattn_bwd_sm100_workspace_bytes(int B, int H, int L);
+size_t linattn_bwd_sm100_workspace_bytes(int B, int H, int L, int d);
 chela_status_t launch_linattn_bwd_sm100(const void *q, const void *k, const void *v, const void *d_o, float *dq, float *dk,
-                                        float *dv, int B, int H, int L, int norm, float eps, float scale, void *workspace,
-                                        cudaStream_t stream);
+                                        float *dv, int B, int H, int L, int d, int norm, float eps, float scale,
+                                        void *workspace, cudaStream_t stream);
 
 chela_status_t launch_shortconv(const void *x, const float *w, const float *bias, void *y, int B, int L,
                                 int D, int width, int act, chela_dtype_t io_dtype, cudaStream_t stream);

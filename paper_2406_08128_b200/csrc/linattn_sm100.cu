@@ -658,10 +658,9 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
                                     float scale, void *workspace, cudaStream_t stream, const float *state_in,
                                     float *state_out, bool reverse, int pair_mask)
 {
-    if (d == 128 && reverse) return CHELA_ERR_UNSUPPORTED;
     if (d == 128)
         return launch_linattn_sm100_d128(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, workspace, stream, state_in,
-                                         state_out);
+                                         state_out, reverse, pair_mask);
     // The result does not depend on the chunk size: both supported values run on 64-token tiles.
     (void)chunk;
     if (reverse) {   // anti-causal mirror: fp32 output, no state carry (the backward pass)

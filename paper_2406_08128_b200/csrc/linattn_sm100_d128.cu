@@ -43,7 +43,8 @@ struct Smem {
 constexpr int kTmemCols = 512;
 constexpr int kColOS = 0, kColSb = 128, kColPT = 256;
 
-template <typename TOut, bool kPair>
+// kReverse: the anti-causal mirror used by the backward pass (chunks walked from the end, upper-triangular mask).
+template <typename TOut, bool kPair, bool kReverse>
 __global__ void __launch_bounds__(kThreads)
 linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
@@ -64,8 +65,10 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const int bh = blockIdx.x / G, g = blockIdx.x % G;
     const int b = bh / H, h = bh % H;
     const int c0 = g * cpg;
-    const int nchunks = min(cpg, (L + kC - 1) / kC - c0);
+    const int nch_total = (L + kC - 1) / kC;
+    const int nchunks = min(cpg, nch_total - c0);
     const bool has_init = g > 0 || state_in != nullptr;
+    auto tok = [&](int chunk) { return (kReverse ? nch_total - 1 - (c0 + chunk) : c0 + chunk) * kC; };
 
     const uint32_t bar_full0 = sbase + SM::offBar;
     const uint32_t bar_p = bar_full0 + 8 * kStages, bar_o = bar_p + 8, bar_pt = bar_o + 8, bar_s = bar_pt + 8;
@@ -107,9 +110,9 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 for (int pl = 0; pl < kPlanes; ++pl)
 #pragma unroll
                     for (int x = 0; x < 2; ++x) {
-                        tma_load_5d(tile(chunk, pl, 2 * x), &tm_q, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
-                        tma_load_5d(tile(chunk, pl, 2 * x + 1), &tm_k, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
-                        tma_load_5d(tile(chunk, pl, 4 + x), &tm_v, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
+                        tma_load_5d(tile(chunk, pl, 2 * x), &tm_q, bar, 64 * x, h, tok(chunk), b, pl);
+                        tma_load_5d(tile(chunk, pl, 2 * x + 1), &tm_k, bar, 64 * x, h, tok(chunk), b, pl);
+                        tma_load_5d(tile(chunk, pl, 4 + x), &tm_v, bar, 64 * x, h, tok(chunk), b, pl);
                     }
             };
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);
@@ -278,21 +281,22 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 if (!ok) break;
                 tc_fence_after();
                 float p[2][32];
-                if (warp == 2) tmem_ld32(tmem_warp + kColPT, p[0]);
-                tmem_ld32(tmem_warp + kColPT + 32, p[1]);
+                const bool live0 = kReverse || warp == 2, live1 = !kReverse || warp == 3;
+                if (live0) tmem_ld32(tmem_warp + kColPT, p[0]);
+                if (live1) tmem_ld32(tmem_warp + kColPT + 32, p[1]);
                 tmem_ld_wait();
                 uint8_t *sP = smem + SM::offPT;
 #pragma unroll
                 for (int cb = 0; cb < 2; ++cb) {
-                    const bool live = cb == 1 || warp == 2;
+                    const bool live = cb == 0 ? live0 : live1;
 #pragma unroll
                     for (int c8 = 0; c8 < 4; ++c8) {
                         uint32_t w[4], w2[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int t = cb * 32 + c8 * 8 + e * 2;
-                            const float x0 = (live && t >= r) ? p[cb][c8 * 8 + e * 2] : 0.f;
-                            const float x1 = (live && t + 1 >= r) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
+                            const float x0 = (live && (kReverse ? t <= r : t >= r)) ? p[cb][c8 * 8 + e * 2] : 0.f;
+                            const float x1 = (live && (kReverse ? t + 1 <= r : t + 1 >= r)) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
                             const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
                             w[e] = *reinterpret_cast<const uint32_t *>(&hh);
                             if (kPair) {
@@ -351,7 +355,7 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
 #pragma unroll
                     for (int bx = 0; bx < SM::kOBoxes; ++bx)
                         tma_store_5d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
-                                     (c0 + i) * kC + warp * 32, b, 0);
+                                     tok(i) + warp * 32, b, 0);
                     bulk_commit();
                 }
             } else if (i + 1 < nchunks) {
@@ -413,10 +417,10 @@ struct SmemState {
     static constexpr int bytes = offAbort + 8;
 };
 
-template <bool kPair>
+template <bool kPair, bool kReverse>
 __global__ void __launch_bounds__(kThreads)
 linattn_state_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                          float *__restrict__ s_part, int H, int G, int cpg, int *__restrict__ status)
+                          float *__restrict__ s_part, int H, int L, int G, int cpg, int *__restrict__ status)
 {
     using SM = SmemState<kPair>;
     constexpr int kStages = SM::kStages, kPlanes = SM::kPlanes;
@@ -463,8 +467,9 @@ linattn_state_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid
                 for (int pl = 0; pl < kPlanes; ++pl)
 #pragma unroll
                     for (int x = 0; x < 2; ++x) {
-                        tma_load_5d(tile(chunk, pl, x), &tm_k, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
-                        tma_load_5d(tile(chunk, pl, 2 + x), &tm_v, bar, 64 * x, h, (c0 + chunk) * kC, b, pl);
+                        const int t0 = (kReverse ? (L + kC - 1) / kC - 1 - (c0 + chunk) : c0 + chunk) * kC;
+                        tma_load_5d(tile(chunk, pl, x), &tm_k, bar, 64 * x, h, t0, b, pl);
+                        tma_load_5d(tile(chunk, pl, 2 + x), &tm_v, bar, 64 * x, h, t0, b, pl);
                     }
             };
             constexpr uint32_t idesc = make_idesc(128, 128, 1, 1);
@@ -563,27 +568,30 @@ SplitPlan split_plan(int B, int H, int L)
 }
 constexpr size_t kWsHeader = 512;
 
-template <typename TOut, bool kPair>
+template <typename TOut, bool kPair, bool kReverse>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
-                        float scale, void *workspace, const float *state_in, float *state_out, cudaStream_t stream)
+                        float scale, void *workspace, const float *state_in, float *state_out, cudaStream_t stream,
+                        int pair_mask = 7)
 {
+    // pair_mask: which of q, k, v really are pairs; a single bf16 operand of a pair kernel gets a one-plane map
+    // and its low plane arrives as zeros (out of bounds for the copy engine)
     CUtensorMap mq, mk, mv, mo;
-    const int planes = kPair ? 2 : 1;
-    if (!make_map(&mq, q, B, H, L, kC, false, planes) || !make_map(&mk, k, B, H, L, kC, false, planes) ||
-        !make_map(&mv, v, B, H, L, kC, false, planes) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4, 1))
+    const int pq = (kPair && (pair_mask & 1)) ? 2 : 1, pk = (kPair && (pair_mask & 2)) ? 2 : 1, pv = (kPair && (pair_mask & 4)) ? 2 : 1;
+    if (!make_map(&mq, q, B, H, L, kC, false, pq) || !make_map(&mk, k, B, H, L, kC, false, pk) ||
+        !make_map(&mv, v, B, H, L, kC, false, pv) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4, 1))
         return CHELA_ERR_CUDA;
     int *status = (int *)workspace;
     float *s_part = (float *)((char *)workspace + kWsHeader);
     const SplitPlan plan = split_plan(B, H, L);
     if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
     if (plan.G > 1) {
-        auto skern = linattn_state_d128_kernel<kPair>;
+        auto skern = linattn_state_d128_kernel<kPair, kReverse>;
         if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemState<kPair>::bytes) != cudaSuccess)
             return CHELA_ERR_CUDA;
-        skern<<<B * H * (plan.G - 1), kThreads, SmemState<kPair>::bytes, stream>>>(mk, mv, s_part, H, plan.G, plan.cpg, status);
+        skern<<<B * H * (plan.G - 1), kThreads, SmemState<kPair>::bytes, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cpg, status);
         if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
     }
-    auto kern = linattn_sm100_d128_kernel<TOut, kPair>;
+    auto kern = linattn_sm100_d128_kernel<TOut, kPair, kReverse>;
     const int smem = Smem<TOut, kPair>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
     kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg,
@@ -597,14 +605,22 @@ size_t linattn_sm100_d128_workspace_bytes(int B, int H, int L) { return kWsHeade
 
 chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                                          chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
-                                         void *workspace, cudaStream_t stream, const float *state_in, float *state_out)
+                                         void *workspace, cudaStream_t stream, const float *state_in, float *state_out, bool reverse,
+                                         int pair_mask)
 {
-    if (in_dtype == CHELA_BF16_PAIR) {
-        if (out_dtype == CHELA_F32) return launch_t<float, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
-        return launch_t<__nv_bfloat16, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+    if (reverse) {
+        if (out_dtype != CHELA_F32 || state_in || state_out) return CHELA_ERR_UNSUPPORTED;
+        if (in_dtype == CHELA_BF16_PAIR)
+            return launch_t<float, true, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pair_mask);
+        return launch_t<float, false, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream);
     }
-    if (out_dtype == CHELA_F32) return launch_t<float, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
-    return launch_t<__nv_bfloat16, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+    if (in_dtype == CHELA_BF16_PAIR) {
+        if (out_dtype == CHELA_F32)
+            return launch_t<float, true, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pair_mask);
+        return launch_t<__nv_bfloat16, true, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+    }
+    if (out_dtype == CHELA_F32) return launch_t<float, false, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+    return launch_t<__nv_bfloat16, false, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
 }
 
 }  // namespace chela

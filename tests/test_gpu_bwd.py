@@ -25,8 +25,10 @@ def test_gradients_match_the_oracle(dtype, B, L, H, d, norm):
     # With a single token the normaliser makes g orthogonal to r up to eps / n^2, so dq and dk are a small
     # residual of a cancellation: that one case gets an order of magnitude more.
     tol = 1e-3 if (L == 1 and norm) else TOLB
-    if dtype == "bf16" and d == 64:
-        tol = 2e-2   # tensor-core path: bf16 operands (scores, G) like the forward pass
+    if dtype == "bf16":
+        # tensor-core path.  Without the normaliser the scores and G are single bf16 values like the forward
+        # pass; with it every rounded intermediate (scores, state, G) is carried as a bf16 pair.
+        tol = 1e-3 if norm else 2e-2
     for got, ref in ((dq, rq), (dk, rk), (dv, rv)):
         assert rel_err(to_numpy(got), ref) <= tol, rel_err(to_numpy(got), ref)
 
