@@ -88,6 +88,8 @@ chela_status_t launch_shortconv_reparam(const float *w1, int width1, const float
                                         cudaStream_t stream);
 
 size_t longconv_workspace_bytes(int B, int L, int D);
+bool launch_fft_conv_fast(int mode, float *rows, int row_stride, int L, int D, int nrows, int logM, const float2 *tw,
+                          float2 *spec, int spec_stride, cudaStream_t stream);
 chela_status_t launch_longconv(const void *x, const float *k_long, const float *w_short, int short_width,
                                void *z, int B, int L, int D, chela_dtype_t in_dtype,
                                chela_dtype_t out_dtype, void *workspace, cudaStream_t stream);

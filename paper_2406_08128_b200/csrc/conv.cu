@@ -498,7 +498,7 @@ __device__ __forceinline__ int bitrev(int f, int logM) { return (int)(__brev((un
 //         convolution back over the row.
 template <int MODE>
 __global__ void __launch_bounds__(1024) fft_conv_kernel(float *__restrict__ rows, int row_stride, int L, int D, int M, int logM,
-                                const float2 *__restrict__ tw_global, float2 *__restrict__ spec)
+                                const float2 *__restrict__ tw_global, float2 *__restrict__ spec, int spec_stride)
 {
     extern __shared__ __align__(16) float2 s[];   // M data points (swizzled), then the two twiddle tables
     float2 *t1 = s + M, *t2 = t1 + 128;
@@ -532,7 +532,7 @@ __global__ void __launch_bounds__(1024) fft_conv_kernel(float *__restrict__ rows
     // The kernel spectrum is kept in the same bit-reversed order as the data (entry p holds K[bitrev(p)];
     // entry M holds the Nyquist term), and the loop runs over positions p rather than frequencies: lanes
     // then touch consecutive shared-memory and global addresses instead of one bank.
-    float2 *kspec = spec + (size_t)(MODE == 1 ? row % D : row) * (M + 1);
+    float2 *kspec = spec + (size_t)(MODE == 1 ? row % D : row) * spec_stride;
     for (int pf = threadIdx.x; pf < M; pf += blockDim.x) {
         const int f = bitrev(pf, logM);
         if (f > (M >> 1)) continue;   // the pair (f, M-f) is handled by its smaller member
@@ -653,12 +653,26 @@ LongconvPlan longconv_plan(int B, int L, int D)
     p.off_at = 0;
     p.off_tw = align_up(p.off_at + (size_t)B * D * p.Ls * sizeof(float), 256);
     p.off_spec = align_up(p.off_tw + (size_t)p.M * sizeof(float2), 256);
-    p.total = align_up(p.off_spec + (size_t)D * (p.M + 1) * sizeof(float2), 256);
+    p.total = align_up(p.off_spec + (size_t)D * (p.M + 2) * sizeof(float2), 256);   // rows of M + 1 entries, 16-byte aligned
     return p;
 }
 }  // namespace
 
 size_t longconv_workspace_bytes(int B, int L, int D) { return longconv_plan(B, L, D).total; }
+
+// rows [B*D][Ls] back to token-major [B, L, D] in the output dtype
+static chela_status_t finish_longconv(const float *at, void *z, int B, int L, int D, int Ls, chela_dtype_t out_dtype,
+                                      cudaStream_t stream)
+{
+    dim3 g2((L + 31) / 32, (D + 63) / 64, B);
+    if (out_dtype == CHELA_BF16 || out_dtype == CHELA_BF16_PAIR) {
+        dim3 gf((L + 63) / 64, (D + 63) / 64, B);
+        transpose_out_bf16_kernel<<<gf, 256, 0, stream>>>(at, (__nv_bfloat16 *)z, L, D, Ls,
+                                                          out_dtype == CHELA_BF16_PAIR ? (size_t)B * L * D : 0);
+    } else
+        transpose_out_kernel<float><<<g2, 256, 0, stream>>>(at, (float *)z, L, D, Ls, 0);
+    return last_launch_status();
+}
 
 chela_status_t launch_longconv(const void *x, const float *k_long, const float *w_short, int short_width,
                                void *z, int B, int L, int D, chela_dtype_t in_dtype,
@@ -689,6 +703,12 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
         conv_transpose_kernel<float><<<g1, 256, 0, stream>>>((const float *)x, w_short, short_width, at, L, D, p.Ls);
     twiddle_kernel<<<(p.M + 255) / 256, 256, 0, stream>>>(tw, p.M);
 
+    // sizes 2^10 .. 2^14: the kernels with compile-time strides; other sizes: the generic kernel below
+    const int spec_stride = p.M + 2;
+    if (launch_fft_conv_fast(0, const_cast<float *>(k_long), L, L, D, D, p.logM, tw, spec, spec_stride, stream) &&
+        launch_fft_conv_fast(1, at, p.Ls, L, D, B * D, p.logM, tw, spec, spec_stride, stream)) {
+        return finish_longconv(at, z, B, L, D, p.Ls, out_dtype, stream);
+    }
     const size_t smem = (size_t)(p.M + 256) * sizeof(float2);
     int threads = p.M / 16;
     threads = threads < 32 ? 32 : (threads > 1024 ? 1024 : threads);
@@ -696,17 +716,9 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(fft_conv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return CHELA_ERR_CUDA;
-    fft_conv_kernel<0><<<D, threads, smem, stream>>>(const_cast<float *>(k_long), L, L, D, p.M, p.logM, tw, spec);
-    fft_conv_kernel<1><<<B * D, threads, smem, stream>>>(at, p.Ls, L, D, p.M, p.logM, tw, spec);
-
-    dim3 g2((L + 31) / 32, (D + 63) / 64, B);
-    if (out_dtype == CHELA_BF16 || out_dtype == CHELA_BF16_PAIR) {
-        dim3 gf((L + 63) / 64, (D + 63) / 64, B);
-        transpose_out_bf16_kernel<<<gf, 256, 0, stream>>>(at, (__nv_bfloat16 *)z, L, D, p.Ls,
-                                                          out_dtype == CHELA_BF16_PAIR ? (size_t)B * L * D : 0);
-    } else
-        transpose_out_kernel<float><<<g2, 256, 0, stream>>>(at, (float *)z, L, D, p.Ls, 0);
-    return last_launch_status();
+    fft_conv_kernel<0><<<D, threads, smem, stream>>>(const_cast<float *>(k_long), L, L, D, p.M, p.logM, tw, spec, spec_stride);
+    fft_conv_kernel<1><<<B * D, threads, smem, stream>>>(at, p.Ls, L, D, p.M, p.logM, tw, spec, spec_stride);
+    return finish_longconv(at, z, B, L, D, p.Ls, out_dtype, stream);
 }
 
 }  // namespace chela

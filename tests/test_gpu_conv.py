@@ -32,7 +32,8 @@ def test_shortconv(dtype, tol, B, L, D, width, act):
 
 
 @pytest.mark.parametrize("B,L,D", [(1, 1, 8), (2, 3, 8), (2, 5, 16), (1, 16, 8), (2, 17, 24), (1, 64, 8),
-                                   (2, 1000, 40), (1, 4096, 16), (2, 5000, 8), (1, 16384, 8)])
+                                   (2, 1000, 40), (1, 1025, 8), (3, 2047, 8), (1, 4096, 16), (2, 5000, 8), (1, 8192, 8),
+                                   (1, 16384, 8), (1, 16383, 8)])
 @pytest.mark.parametrize("fused_short", [False, True])
 def test_longconv_against_direct_and_fft_oracle(B, L, D, fused_short):
     m = inputs.mixer(300 + L, B, L, D, dtype="bf16", decay=0.001)
