@@ -6,13 +6,13 @@
 // leading digits to cancellation in Q K^T.  W [K, N] is bf16.  Y [M, N] is written as bf16 or as a
 // bf16 pair (hi = round(y), lo = round(y - hi)).
 //
-// Persistent kernel, one CTA per SM, 128 x 128 output tiles, K blocks of 64:
-//   warp 4 lane 0 : TMA producer (A_hi, A_lo: [128 rows] x 128 B K-major tiles; W: two [64 k-rows] x 128 B
-//                   atoms, MN-major), 3-stage ring
-//   warp 5 lane 0 : tcgen05.mma issuer, M = 128, N = 128 (64 cycles per instruction: full rate);
-//                   accumulators double-buffered in TMEM (2 x 128 columns)
+// Persistent kernel, one CTA per SM, 128 x BN output tiles (BN = 256 when N allows, else 128), K blocks of 64:
+//   warp 4 lane 0 : TMA producer (A_hi, A_lo: [128 rows] x 128 B K-major tiles; W: BN / 64 atoms of
+//                   [64 k-rows] x 128 B, MN-major), 3- or 4-stage ring (192 KB in flight at BN = 256)
+//   warp 5 lane 0 : tcgen05.mma issuer, M = 128, N = BN (BN / 2 cycles per instruction: full rate);
+//                   accumulators double-buffered in TMEM (2 x BN columns)
 //   warps 0-3     : epilogue: TMEM -> bias, activation, hi/lo split -> swizzled staging -> TMA store,
-//                   32 rows x 64 columns per warp and box, ping-pong staging
+//                   32 rows x 64 columns per warp and box (ping-pong staging at BN = 128)
 // Every wait is bounded; a timeout records CHELA_ERR_TIMEOUT in the status word and ends the CTA cleanly.
 #include "sm100_ptx.cuh"
 
@@ -21,30 +21,39 @@ namespace {
 
 using namespace sm100;
 
-constexpr int BM = 128, BN = 128, BK = 64;
-constexpr int kStages = 3;
+constexpr int BM = 128, BK = 64;
 constexpr int kThreads = 192;
 constexpr int kATile = BM * 128;        // 16 KB
-constexpr int kBTile = BK * 128 * 2;    // two 64-column atoms, 16 KB
-constexpr int kStageBytes = 2 * kATile + kBTile;
-constexpr int kStagingWarp = 4 * 32 * 128;   // per warp: 2 buffers x (hi, lo) x [32 rows x 128 B]
+constexpr int kMaxStages = 4;
 
+// BN = 256 where N allows: the SM takes its operands from L2 at about 45 bytes per clock, which a 128 x 128
+// tile with a pair A operand exceeds; a 128 x 256 tile needs two thirds of the bytes per flop.
+template <int BN, bool kAPair>
 struct Smem {
+    static constexpr int kBTile = BK * 128 * (BN / 64);             // BN / 64 atoms of 64 columns
+    static constexpr int kStageBytes = (kAPair ? 2 : 1) * kATile + kBTile;
+    static constexpr int kStages = (BN == 256 && !kAPair) ? 4 : 3;  // 192 KB of operands in flight at BN = 256
+    static constexpr int kStagingBufs = BN == 256 ? 1 : 2;          // per warp: buffers of (hi, lo) x [32 rows x 128 B]
+    static constexpr int kStagingWarp = kStagingBufs * 2 * 32 * 128;
     static constexpr int offStage = 0;
     static constexpr int offStaging = kStages * kStageBytes;
-    static constexpr int offBar = offStaging + 4 * kStagingWarp;   // full[3], empty[3], tfull[2], tempty[2]
-    static constexpr int offTmem = offBar + 8 * (2 * kStages + 4);
+    static constexpr int offBar = offStaging + 4 * kStagingWarp;   // full[kStages], empty[kStages], tfull[2], tempty[2]
+    static constexpr int offTmem = offBar + 8 * (2 * kMaxStages + 4);
     static constexpr int offAbort = offTmem + 8;
     static constexpr int bytes = offAbort + 8;
+    static_assert(bytes <= 232448, "shared memory per CTA");
 };
 
-template <bool kAPair, bool kYPair>
+template <int BN, bool kAPair, bool kYPair>
 __global__ void __launch_bounds__(kThreads)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_constant__ CUtensorMap tm_a_lo,
                   const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y_hi,
                   const __grid_constant__ CUtensorMap tm_y_lo, const float *__restrict__ bias, int M, int N, int K,
                   int act, int *__restrict__ status)
 {
+    using Smem = Smem<BN, kAPair>;
+    constexpr int kStages = Smem::kStages, kStageBytes = Smem::kStageBytes, kStagingWarp = Smem::kStagingWarp;
+    constexpr int kAOff = (kAPair ? 2 : 1) * kATile;   // W atoms follow the A tile(s) of a stage
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     if (sbase & 1023u) {
@@ -73,7 +82,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
         tma_prefetch_desc(&tm_y_hi);
     }
     if (warp == 0) {
-        tmem_alloc(sbase + Smem::offTmem, 256);
+        tmem_alloc(sbase + Smem::offTmem, 2 * BN);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -95,11 +104,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                     ok = mbar_wait(bar_empty0 + 8 * s, ((it / kStages) & 1) ^ 1, abort_flag);
                     if (!ok) break;
                     const uint32_t bar = bar_full0 + 8 * s, dst = sbase + Smem::offStage + s * kStageBytes;
-                    mbar_expect_tx(bar, (kAPair ? 2 : 1) * kATile + kBTile);
+                    mbar_expect_tx(bar, kStageBytes);
                     tma_load_2d(dst, &tm_a_hi, bar, kb * BK, m0);
                     if (kAPair) tma_load_2d(dst + kATile, &tm_a_lo, bar, kb * BK, m0);
-                    tma_load_2d(dst + 2 * kATile, &tm_w, bar, n0, kb * BK);
-                    tma_load_2d(dst + 2 * kATile + BK * 128, &tm_w, bar, n0 + 64, kb * BK);
+#pragma unroll
+                    for (int a = 0; a < BN / 64; ++a) tma_load_2d(dst + kAOff + a * BK * 128, &tm_w, bar, n0 + 64 * a, kb * BK);
                     issued = it + 1;
                 }
             }
@@ -128,7 +137,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t st = sbase + Smem::offStage + s * kStageBytes;
-                    const uint32_t a_hi = desc_lo(st), a_lo = desc_lo(st + kATile), w_lo = desc_lo(st + 2 * kATile, BK * 128);
+                    const uint32_t a_hi = desc_lo(st), a_lo = desc_lo(st + kATile), w_lo = desc_lo(st + kAOff, BK * 128);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
                         umma_bf16(d, a_hi + 2 * k, w_lo + 128 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
@@ -168,10 +177,15 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_tempty0 + 8 * buf);
                 }
-                // staging buffer (nbox & 1) is free once the store issued two boxes ago has been read
-                if (lane == 0) bulk_wait_read1();
+                // the staging buffer is free once the store that last used it has been read (two boxes ago with
+                // ping-pong buffers, the previous box with one)
+                if (lane == 0) {
+                    if (Smem::kStagingBufs == 2) bulk_wait_read1();
+                    else bulk_wait_read0();
+                }
                 __syncwarp();
-                uint8_t *hi = stg + (nbox & 1) * (2 * 32 * 128), *lo = hi + 32 * 128;
+                const int sb = Smem::kStagingBufs == 2 ? (nbox & 1) : 0;
+                uint8_t *hi = stg + sb * (2 * 32 * 128), *lo = hi + 32 * 128;
 #pragma unroll
                 for (int j8 = 0; j8 < 8; ++j8) {
                     uint32_t wh[4], wl[4];
@@ -201,7 +215,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) {   // rows past M are clipped by the copy engine
-                    const uint32_t src = stg_u32 + (nbox & 1) * (2 * 32 * 128);
+                    const uint32_t src = stg_u32 + sb * (2 * 32 * 128);
                     tma_store_2d(&tm_y_hi, src, n0 + c * 64, m0 + warp * 32);
                     if (kYPair) tma_store_2d(&tm_y_lo, src + 32 * 128, n0 + c * 64, m0 + warp * 32);
                     bulk_commit();
@@ -216,7 +230,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 256);
+    if (warp == 0) tmem_dealloc(tmem, 2 * BN);
 }
 
 bool map_2d(CUtensorMap *map, const void *ptr, size_t rows, int cols, int box_cols, int box_rows)
@@ -231,7 +245,7 @@ bool map_2d(CUtensorMap *map, const void *ptr, size_t rows, int cols, int box_co
 
 bool gemm_sm100_supported(size_t M, int K, int N, chela_dtype_t a_dtype, chela_dtype_t w_dtype, chela_dtype_t y_dtype)
 {
-    return M >= 1 && M < (1ull << 31) && K % BK == 0 && N % BN == 0 && w_dtype == CHELA_BF16 &&
+    return M >= 1 && M < (1ull << 31) && K % BK == 0 && N % 128 == 0 && w_dtype == CHELA_BF16 &&
            (a_dtype == CHELA_BF16 || a_dtype == CHELA_BF16_PAIR) && (y_dtype == CHELA_BF16 || y_dtype == CHELA_BF16_PAIR);
 }
 
@@ -249,13 +263,23 @@ chela_status_t launch_gemm_sm100(const void *a, const void *w, const float *bias
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         sms = 148;
-    const long long tiles = (long long)((M + BM - 1) / BM) * (N / BN);
+    const int bn = (N % 256 == 0) ? 256 : 128;
+    const long long tiles = (long long)((M + BM - 1) / BM) * (N / bn);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float *, int, int, int, int, int *) =
-        a_pair ? (y_pair ? gemm_sm100_kernel<true, true> : gemm_sm100_kernel<true, false>)
-               : (y_pair ? gemm_sm100_kernel<false, true> : gemm_sm100_kernel<false, false>);
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::bytes) != cudaSuccess) return CHELA_ERR_CUDA;
-    kern<<<grid, kThreads, Smem::bytes, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status);
+    typedef void (*Kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float *, int, int, int, int, int *);
+    Kern kern;
+    int smem;
+    if (bn == 256) {
+        kern = a_pair ? (y_pair ? gemm_sm100_kernel<256, true, true> : gemm_sm100_kernel<256, true, false>)
+                      : (y_pair ? gemm_sm100_kernel<256, false, true> : gemm_sm100_kernel<256, false, false>);
+        smem = a_pair ? Smem<256, true>::bytes : Smem<256, false>::bytes;
+    } else {
+        kern = a_pair ? (y_pair ? gemm_sm100_kernel<128, true, true> : gemm_sm100_kernel<128, true, false>)
+                      : (y_pair ? gemm_sm100_kernel<128, false, true> : gemm_sm100_kernel<128, false, false>);
+        smem = a_pair ? Smem<128, true>::bytes : Smem<128, false>::bytes;
+    }
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
+    kern<<<grid, kThreads, smem, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status);
     return last_launch_status();
 }
 

@@ -21,7 +21,7 @@ def pair_to_device(a):
     return torch.stack([to_device(hi, "bf16"), to_device(lo, "bf16")]).contiguous(), hi.astype(np.float64) + lo
 
 
-@pytest.mark.parametrize("M,K,N", [(128, 64, 128), (256, 512, 256), (1000, 128, 384), (4096, 512, 1024), (100, 1024, 128),
+@pytest.mark.parametrize("M,K,N", [(128, 64, 128), (256, 512, 256), (1000, 128, 384), (4096, 512, 1024), (100, 1024, 128), (300, 192, 512),
                                    (1, 64, 128)])
 @pytest.mark.parametrize("a_pair,y_pair", [(False, False), (True, True), (False, True), (True, False)])
 def test_tensor_core_path(M, K, N, a_pair, y_pair):
