@@ -441,6 +441,22 @@ def main():
         line["backward"] = {"ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
                             "note": "chela_linattn_bwd, bf16 in, fp32 gradients, same workload as the timed step"}
         del d_o, bws
+        # ---- decode step: one token per sequence against the carried state (bound by the state's bytes) --------
+        db, dh = 256, H
+        qs, ks, vs = ((torch.randn((db, dh, D), device=dev, generator=gen) * 0.125).to(torch.bfloat16) for _ in range(3))
+        states = [torch.zeros((db, dh, D, D), device=dev) for _ in range(3)]   # 3 x 67 MB: rotated, larger than L2
+        o_step = torch.empty((db, dh, D), device=dev)
+        it = [0]
+
+        def step_once():
+            chela.linattn_step(qs, ks, vs, states[it[0] % 3], out=o_step)
+            it[0] += 1
+        ms = timed(step_once, 30, warm=6)
+        line["decode_step"] = {"ms": ms, "sequences": db * dh, "tokens_per_s": db / (ms * 1e-3),
+                               "state_GBps": 2 * db * dh * D * D * 4 / (ms * 1e-3) / 1e9,
+                               "hbm_frac": 2 * db * dh * D * D * 4 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                               "note": "chela_linattn_step, B=256 H=16 d=64, fp32 state read and written once per token"}
+        del qs, ks, vs, states, o_step
         # ---- CPU oracle on the host cores, bounded sample -----------------------------------------------
         import oracle
         oracle.build()

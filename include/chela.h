@@ -132,6 +132,21 @@ chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void 
                                        void *workspace, size_t workspace_bytes, cudaStream_t stream);
 
 /*
+ * Decoding step: one new token per sequence against the carried state (recurrent form of Eq. 2; Sec. 5's
+ * sequential evaluation taken to segments of one token):
+ *   S <- S + k v^T  (in place),   r = scale * S^T q,   o = Norm(r) as in chela_linattn_fwd.
+ * Equals chela_linattn_carry_fwd with L = 1 and state_in = state_out = state, without its per-call tile
+ * machinery: the state is read and written once.
+ * q, k : [B, H, d_k];  v, o : [B, H, d_v];  state : [B, H, d_k, d_v] fp32, updated in place; device pointers,
+ * 16-byte aligned, owned by the caller.  Supported: d_k = d_v in {64, 128}; in_dtype F32 or BF16; out_dtype
+ * F32 or BF16.  No workspace.  Errors: CHELA_ERR_INVALID_ARG (null pointer, B, H < 1), CHELA_ERR_UNSUPPORTED.
+ */
+chela_status_t chela_linattn_step(const void *q, const void *k, const void *v, void *o, float *state,
+                                  int B, int H, int d_k, int d_v,
+                                  chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                                  chela_norm_t norm, float norm_eps, float scale, cudaStream_t stream);
+
+/*
  * Backward of chela_linattn_fwd (gradients of Eq. 2 with the causal mask and the row normaliser; the
  * chunked evaluation of Sec. 4.1 run in both directions): given d_o = dLoss/do,
  *   dq_t = scale sum_{s<=t} <g_t,v_s> k_s,  dk_s = scale sum_{t>=s} <g_t,v_s> q_t,  dv_s = scale sum_{t>=s} <q_t,k_s> g_t,

@@ -40,6 +40,7 @@ _SIGNATURES = {
                                    _c_float, _vp, _c_size_t, _vp]),
     "chela_linattn_carry_fwd": (_c_int, [_vp, _vp, _vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                          _c_float, _vp, _c_size_t, _vp]),
+    "chela_linattn_step": (_c_int, [_vp] * 5 + [_c_int] * 4 + [_c_int, _c_int, _c_int, _c_float, _c_float, _vp]),
     "chela_linattn_bwd_workspace_bytes": (_c_size_t, [_c_int] * 5),
     "chela_linattn_bwd": (_c_int, [_vp] * 7 + [_c_int] * 5 + [_c_int, _c_int, _c_float, _c_float, _vp, _c_size_t, _vp]),
     "chela_dense_workspace_bytes": (_c_size_t, []),
@@ -197,6 +198,16 @@ def linattn_carry_fwd(q, k, v, state_in=None, chunk=64, out_dtype=F32, norm=NORM
                                          d_k, d_v, chunk, in_dtype, _dt(o), int(norm), float(eps), float(scale),
                                          _ptr(workspace), workspace.numel(), _stream()), "chela_linattn_carry_fwd")
     return o, state_out
+
+
+def linattn_step(q, k, v, state, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale=1.0, out=None):
+    """chela_linattn_step: one token per sequence; q, k, v [B,H,d]; state [B,H,d,d] fp32 is updated in place."""
+    B, H, d_k = q.shape
+    d_v = v.shape[2]
+    o = torch.empty((B, H, d_v), dtype=_tdtype(out_dtype), device=q.device) if out is None else out
+    _check(lib().chela_linattn_step(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(state), B, H, d_k, d_v, _dt(q), _dt(o),
+                                    int(norm), float(eps), float(scale), _stream()), "chela_linattn_step")
+    return o
 
 
 def linattn_bwd(q, k, v, d_o, norm=NORM_RMS, eps=1e-6, scale=1.0, workspace=None):

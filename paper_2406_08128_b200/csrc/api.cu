@@ -149,6 +149,18 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
                                    norm_eps, scale, workspace, workspace_bytes, stream);
 }
 
+chela_status_t chela_linattn_step(const void *q, const void *k, const void *v, void *o, float *state, int B, int H,
+                                  int d_k, int d_v, chela_dtype_t in_dtype, chela_dtype_t out_dtype, chela_norm_t norm,
+                                  float norm_eps, float scale, cudaStream_t stream)
+{
+    if (!q || !k || !v || !o || !state || B < 1 || H < 1 || d_k < 1 || d_v < 1 || !dtype_ok(in_dtype) || !dtype_ok(out_dtype) ||
+        (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) || !(norm_eps >= 0.f))
+        return CHELA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(state)) return CHELA_ERR_INVALID_ARG;
+    if (d_k != d_v || (d_k != 64 && d_k != 128)) return CHELA_ERR_UNSUPPORTED;
+    return launch_linattn_step(q, k, v, o, state, B, H, d_k, in_dtype, out_dtype, (int)norm, norm_eps, scale, stream);
+}
+
 size_t chela_linattn_bwd_workspace_bytes(int B, int H, int L, int d_k, int d_v)
 {
     if (B < 1 || H < 1 || L < 1 || d_k != d_v || (d_k != 64 && d_k != 128)) return 0;

@@ -180,7 +180,88 @@ chela_status_t launch_d(const void *q, const void *k, const void *v, void *o, in
     return launch_t<D, C, float, __nv_bfloat16>(q, k, v, o, B, H, L, norm, eps, scale, stream, state_in, state_out);
 }
 
+// ------------------------------------------------------------------------------- decode step
+//
+// One token per sequence with the state carried in place (recurrent form of Eq. 2):
+//   S <- S + k v^T,   r = scale * S^T q,   o = Norm(r).
+// One CTA of 256 threads per (batch, head).  The state is read and written exactly once (float4): the step is
+// bound by those 2 * d * d * 4 bytes.  Thread t owns the four columns 4 * (t % (D/4)) of the rows
+// t / (D/4) + j * (1024 / D); column sums are finished through shared memory.
+template <int D, typename TIn, typename TOut>
+__global__ void __launch_bounds__(256)
+linattn_step_kernel(const TIn *__restrict__ q, const TIn *__restrict__ k, const TIn *__restrict__ v, TOut *__restrict__ o,
+                    float *__restrict__ state, float scale, int norm, float eps)
+{
+    constexpr int CG = D / 4, RG = 256 / CG;   // column groups, row groups
+    __shared__ float sq[D], sk[D];
+    __shared__ float4 part[RG][CG];
+    __shared__ float sr[D];
+    const int tid = threadIdx.x, cg = tid % CG, rg = tid / CG;
+    const size_t bh = blockIdx.x;
+    if (tid < D) {
+        sq[tid] = load1(q + bh * D + tid);
+        sk[tid] = load1(k + bh * D + tid);
+    }
+    const float4 vv = load4(v + bh * D + 4 * cg);
+    __syncthreads();
+    float4 *S = reinterpret_cast<float4 *>(state + bh * D * D);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int i = rg; i < D; i += RG) {
+        float4 sv = S[i * CG + cg];
+        const float ki = sk[i], qi = sq[i];
+        sv.x = fmaf(ki, vv.x, sv.x); sv.y = fmaf(ki, vv.y, sv.y); sv.z = fmaf(ki, vv.z, sv.z); sv.w = fmaf(ki, vv.w, sv.w);
+        S[i * CG + cg] = sv;
+        acc.x = fmaf(qi, sv.x, acc.x); acc.y = fmaf(qi, sv.y, acc.y); acc.z = fmaf(qi, sv.z, acc.z); acc.w = fmaf(qi, sv.w, acc.w);
+    }
+    part[rg][cg] = acc;
+    __syncthreads();
+    if (tid < CG) {
+        float4 r = part[0][tid];
+        for (int g = 1; g < RG; ++g) {
+            const float4 p = part[g][tid];
+            r.x += p.x; r.y += p.y; r.z += p.z; r.w += p.w;
+        }
+        r.x *= scale; r.y *= scale; r.z *= scale; r.w *= scale;
+        *reinterpret_cast<float4 *>(sr + 4 * tid) = r;
+    }
+    __syncthreads();
+    if (tid < 32) {
+        float ss = 0.f;
+        for (int j = tid; j < D; j += 32) ss = fmaf(sr[j], sr[j], ss);
+#pragma unroll
+        for (int m = 16; m >= 1; m >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, m);
+        const float inv = norm ? rsqrtf(ss * (1.0f / D) + eps) : 1.0f;
+        for (int j = tid; j < D; j += 32) store1(o + bh * D + j, sr[j] * inv);
+    }
+}
+
+template <int D>
+chela_status_t launch_step_d(const void *q, const void *k, const void *v, void *o, float *state, int B, int H,
+                             chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale, cudaStream_t stream)
+{
+    const int grid = B * H;
+    if (in_dtype == CHELA_F32 && out_dtype == CHELA_F32)
+        linattn_step_kernel<D, float, float><<<grid, 256, 0, stream>>>((const float *)q, (const float *)k, (const float *)v, (float *)o, state, scale, norm, eps);
+    else if (in_dtype == CHELA_F32)
+        linattn_step_kernel<D, float, __nv_bfloat16><<<grid, 256, 0, stream>>>((const float *)q, (const float *)k, (const float *)v, (__nv_bfloat16 *)o, state, scale, norm, eps);
+    else if (out_dtype == CHELA_F32)
+        linattn_step_kernel<D, __nv_bfloat16, float><<<grid, 256, 0, stream>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, (float *)o, state, scale, norm, eps);
+    else
+        linattn_step_kernel<D, __nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, stream>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, (__nv_bfloat16 *)o, state, scale, norm, eps);
+    return last_launch_status();
+}
+
 }  // namespace
+
+chela_status_t launch_linattn_step(const void *q, const void *k, const void *v, void *o, float *state, int B, int H, int d,
+                                   chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
+                                   cudaStream_t stream)
+{
+    if (d == 64) return launch_step_d<64>(q, k, v, o, state, B, H, in_dtype, out_dtype, norm, eps, scale, stream);
+    if (d == 128) return launch_step_d<128>(q, k, v, o, state, B, H, in_dtype, out_dtype, norm, eps, scale, stream);
+    return CHELA_ERR_UNSUPPORTED;
+}
 
 // The result does not depend on the chunk size; with d = 128 the shared-memory budget holds
 // 64-token chunks only, so chunk = 128 is evaluated as two 64-token chunks there.

@@ -39,3 +39,35 @@ def test_state_out_without_state_in_and_oracle_state_in():
                                     state_in=torch.from_numpy(s0).cuda())
     assert rel_err(to_numpy(o), ref) <= 2e-2
     assert np.abs(to_numpy(s1) - ref_state).max() <= 2e-3 * np.abs(ref_state).max()
+
+
+@pytest.mark.parametrize("dtype,tol", [("bf16", 1e-4), ("f32", 1e-4)])
+@pytest.mark.parametrize("B,H,d,T,norm", [(2, 3, 64, 40, True), (1, 2, 128, 25, True), (3, 1, 64, 10, False), (1, 1, 128, 5, False)])
+def test_decode_steps_equal_the_sequence(dtype, tol, B, H, d, T, norm):
+    """Token-by-token chela_linattn_step from a prefix state reproduces the oracle's outputs over the whole
+    sequence (fp32 state and arithmetic on inputs exact in the storage dtype: the fp32 bound)."""
+    import torch
+    P = 70   # prefix evaluated by the chunked kernel, then T decode steps
+    q, k, v = inputs.qkv(80 + d + T, B, P + T, H, d, d, dtype)
+    ref, ref_state = oracle.linattn_recurrent(q, k, v, norm=norm, scale=0.5, return_state=True)
+    nrm = chela.NORM_RMS if norm else chela.NORM_NONE
+    qd, kd, vd = (to_device(x, dtype) for x in (q, k, v))
+    _, state = chela.linattn_carry_fwd(qd[:, :P].contiguous(), kd[:, :P].contiguous(), vd[:, :P].contiguous(), norm=nrm, scale=0.5)
+    if dtype == "bf16":   # the prefix state of the tensor kernel carries bf16-score rounding; take the oracle's
+        state = torch.from_numpy(oracle.linattn_recurrent(q[:, :P], k[:, :P], v[:, :P], return_state=True)[1].astype(np.float32)).cuda()
+    outs = []
+    for t in range(P, P + T):
+        outs.append(to_numpy(chela.linattn_step(qd[:, t].contiguous(), kd[:, t].contiguous(), vd[:, t].contiguous(), state,
+                                                norm=nrm, scale=0.5)))
+    got = np.stack(outs, axis=1)
+    assert rel_err(got, ref[:, P:]) <= tol
+    assert np.abs(to_numpy(state) - ref_state).max() <= 1e-5 * np.abs(ref_state).max()
+
+
+def test_decode_step_argument_checks():
+    import torch
+    q = torch.zeros(1, 1, 32, device="cuda")
+    s = torch.zeros(1, 1, 32, 32, device="cuda")
+    with pytest.raises(chela.ChelaError) as e:
+        chela.linattn_step(q, q, q, s)
+    assert e.value.status == chela.ERR_UNSUPPORTED
