@@ -35,19 +35,26 @@ constexpr int kThreads = 160;            // 4 compute warps + 1 issuer warp
 constexpr int kC = 64;       // tokens per tile
 constexpr int kTile = kC * 128;   // one 64-row x 128-byte tile
 
-// kPair: Q, K, V arrive as bf16 pairs (hi + lo planes); every product then takes three tensor-core
-// terms (hi*hi + hi*lo + lo*hi) and the score tile is kept as a pair too.
-template <typename TOut, bool kPair>
+// kMask says which operands are bf16 pairs (hi + lo planes): bit 0 = Q, bit 1 = K, bit 2 = V, bit 3 = the score
+// tile P (an internal operand: rounded once to bf16, or kept as hi + lo).  A product with a pair operand takes one
+// more tensor-core term per pair side (hi*hi + hi*lo + lo*hi; lo*lo is dropped).  0 = the plain bf16 kernel, 15 = the
+// mixer's attention; the backward pass uses 8 (recomputed forward), 9, 10 and 12 (one gradient operand is a pair).
+__host__ __device__ constexpr int popc3(int m) { return (m & 1) + ((m >> 1) & 1) + ((m >> 2) & 1); }
+template <typename TOut, int kMask>
 struct Smem {
-    static constexpr int kStages = kPair ? 2 : 3;
-    static constexpr int kTilesPerStage = kPair ? 6 : 3;  // Q, K, V (hi), then Q, K, V (lo); adjacent
+    static constexpr int kIn = kMask & 7;
+    static constexpr bool kPPair = (kMask & 8) != 0;
+    static constexpr int kTilesPerStage = 3 + popc3(kIn);   // Q, K, V (hi), then the low planes that exist, in that order
+    static constexpr int iQlo = 3, iKlo = 3 + (kIn & 1), iVlo = 3 + popc3(kIn & 3);
+    static constexpr int kStages = (kMask == 0) ? 3 : 2;
     static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as 128-byte wide boxes
     static constexpr int offPT = 0;                       // masked scores, transposed: rows = s, 64 t per row (hi, lo)
-    static constexpr int offShi = offPT + (kPair ? 2 : 1) * kTile;   // state, bf16 high part: rows = d_k
+    static constexpr int offShi = offPT + (kPPair ? 2 : 1) * kTile;   // state, bf16 high part: rows = d_k
     static constexpr int offSlo = offShi + kTile;         // state, bf16 low part
-    static constexpr int offO = offSlo + kTile;           // output staging
-    static constexpr int offStage = offO + kOBoxes * kTile;
-    static constexpr int offBar = offStage + kStages * kTilesPerStage * kTile;   // full[kStages], p, o, pt, s
+    static constexpr int offStage = offSlo + kTile;       // after the score tile: the G3 descriptor reaches K from P forwards
+    // output staging; also what a 128-row operand that starts in the last tile of the last stage reads past it
+    static constexpr int offO = offStage + kStages * kTilesPerStage * kTile;
+    static constexpr int offBar = offO + (kOBoxes > 1 ? kOBoxes : 1) * kTile;   // full[kStages], p, o, pt, s
     static constexpr int offTmem = offBar + 8 * (kStages + 4);
     static constexpr int offAbort = offTmem + 8;
     static constexpr int bytes = offAbort + 8;
@@ -69,7 +76,7 @@ constexpr int kColPT = 64;   // rows 64..127: transposed scores; 64 columns
 // kReverse: the anti-causal mirror (token t attends keys s >= t; the state accumulates from the end of the
 // sequence).  Chunks are walked from the last to the first and the mask is the upper triangle; everything
 // else, including the split into groups, works on the mirrored chunk index.  Used by the backward pass.
-template <typename TOut, bool kPair, bool kReverse>
+template <typename TOut, int kMask, bool kReverse>
 __global__ void __launch_bounds__(kThreads)
 linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
@@ -79,9 +86,11 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     // Grid: one CTA per (batch*head, group).  Group g covers chunks [g*cpg, (g+1)*cpg) of its sequence and
     // starts from the state sum_{g' < g} s_part[bh][g'] (per-group K^T V sums written by the state kernel),
     // plus the caller's initial state state_in[bh] if given; the last group writes the final state.
-    using SM = Smem<TOut, kPair>;
+    using SM = Smem<TOut, kMask>;
     constexpr int kStages = SM::kStages;
     constexpr int kTPS = SM::kTilesPerStage;
+    constexpr int kIn = SM::kIn;
+    constexpr bool kPPair = SM::kPPair;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     if (sbase & 1023u) {  // swizzled tiles need a 1024-byte aligned base: report instead of corrupting
@@ -136,12 +145,12 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             auto issue_load = [&](int chunk) {
                 const uint32_t bar = bar_full0 + 8 * (chunk % kStages), dst = stage_base(chunk);
                 mbar_expect_tx(bar, kTPS * kTile);
-#pragma unroll
-                for (int pl = 0; pl < (kPair ? 2 : 1); ++pl) {
-                    tma_load_5d(dst + (3 * pl) * kTile, &tm_q, bar, 0, h, tok(chunk), b, pl);
-                    tma_load_5d(dst + (3 * pl + 1) * kTile, &tm_k, bar, 0, h, tok(chunk), b, pl);
-                    tma_load_5d(dst + (3 * pl + 2) * kTile, &tm_v, bar, 0, h, tok(chunk), b, pl);
-                }
+                tma_load_5d(dst, &tm_q, bar, 0, h, tok(chunk), b, 0);
+                tma_load_5d(dst + kTile, &tm_k, bar, 0, h, tok(chunk), b, 0);
+                tma_load_5d(dst + 2 * kTile, &tm_v, bar, 0, h, tok(chunk), b, 0);
+                if (kIn & 1) tma_load_5d(dst + SM::iQlo * kTile, &tm_q, bar, 0, h, tok(chunk), b, 1);
+                if (kIn & 2) tma_load_5d(dst + SM::iKlo * kTile, &tm_k, bar, 0, h, tok(chunk), b, 1);
+                if (kIn & 4) tma_load_5d(dst + SM::iVlo * kTile, &tm_v, bar, 0, h, tok(chunk), b, 1);
             };
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [Q;K] (K-major) x Q^T (K-major)
             constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;K] (K-major) x S (MN-major)
@@ -153,12 +162,15 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const uint32_t qk_lo = desc_lo(stage_base(chunk));
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk_lo + 2 * k, qk_lo + 2 * k, idescG1, k > 0);
-                if (kPair) {   // + K_hi Q_lo^T + K_lo Q_hi^T
-                    const uint32_t qk2_lo = desc_lo(stage_base(chunk) + 3 * kTile);
+                if (kIn & 1) {   // + K_hi Q_lo^T
+                    const uint32_t q2_lo = desc_lo(stage_base(chunk) + SM::iQlo * kTile);
 #pragma unroll
-                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk_lo + 2 * k, qk2_lo + 2 * k, idescG1, 1);
+                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk_lo + 2 * k, q2_lo + 2 * k, idescG1, 1);
+                }
+                if (kIn & 2) {   // + K_lo Q_hi^T: the 128-row operand starts one tile before K_lo (rows 0..63 are not used)
+                    const uint32_t xk2_lo = desc_lo(stage_base(chunk) + (SM::iKlo - 1) * kTile);
 #pragma unroll
-                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, qk2_lo + 2 * k, qk_lo + 2 * k, idescG1, 1);
+                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT, xk2_lo + 2 * k, qk_lo + 2 * k, idescG1, 1);
                 }
                 umma_commit(bar_p);
                 return true;
@@ -183,8 +195,8 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, shi_lo + 128 * k, idescG2, k > 0, 1);
 #pragma unroll
                     for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, slo_lo + 128 * k, idescG2, 1, 1);
-                    if (kPair) {   // + Q_lo S_hi
-                        const uint32_t qk2_lo = desc_lo(st + 3 * kTile);
+                    if (kIn & 1) {   // + Q_lo S_hi (rows 64..127 of the operand: whatever follows Q_lo; their lanes are write-disabled)
+                        const uint32_t qk2_lo = desc_lo(st + SM::iQlo * kTile);
 #pragma unroll
                         for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk2_lo + 2 * k, shi_lo + 128 * k, idescG2, 1, 1);
                     }
@@ -199,13 +211,18 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k)
                     umma_bf16(tmem + kColOS, a_lo + 128 * k, v_lo + 128 * k, idescG3, (i > 0 || has_init || k > 0) ? 1u : 0u);
-                if (kPair) {   // + [P_hi^T | K_hi]^T V_lo + [P_lo^T | K_lo]^T V_hi
-                    const uint32_t v2_lo = desc_lo(st + 5 * kTile);
-                    const uint32_t a2_lo = desc_lo(sbase + SM::offPT + kTile, st + 4 * kTile - (sbase + SM::offPT + kTile));
+                if (kIn & 4) {   // + [P_hi^T | K_hi]^T V_lo
+                    const uint32_t v2_lo = desc_lo(st + SM::iVlo * kTile);
 #pragma unroll
                     for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS, a_lo + 128 * k, v2_lo + 128 * k, idescG3, 1);
+                }
+                if (kPPair || (kIn & 2)) {   // + [P_lo^T | K_lo]^T V_hi; a half that does not exist is write-disabled
+                    const uint32_t atom0 = sbase + SM::offPT + (kPPair ? kTile : 0);
+                    const uint32_t atom1 = st + ((kIn & 2) ? SM::iKlo : 1) * kTile;
+                    const uint32_t a2_lo = desc_lo(atom0, atom1 - atom0);
+                    const uint32_t lanes = (kPPair && (kIn & 2)) ? 0u : (kPPair ? 1u : 2u);
 #pragma unroll
-                    for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS, a2_lo + 128 * k, v_lo + 128 * k, idescG3, 1);
+                    for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS, a2_lo + 128 * k, v_lo + 128 * k, idescG3, 1, lanes);
                 }
                 umma_commit(bar_o);
                 if (i + 1 < nchunks) {
@@ -323,13 +340,13 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             const float x1 = (live && (kReverse ? t + 1 <= r : t + 1 >= r)) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
                             const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
                             w[e] = *reinterpret_cast<const uint32_t *>(&hh);
-                            if (kPair) {
+                            if (kPPair) {
                                 const float2 hf = __bfloat1622float2(hh);
                                 w2[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
                             }
                         }
                         *reinterpret_cast<uint4 *>(sP + sw128(r, cb * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
-                        if (kPair) *reinterpret_cast<uint4 *>(sP + kTile + sw128(r, cb * 4 + c8)) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+                        if (kPPair) *reinterpret_cast<uint4 *>(sP + kTile + sw128(r, cb * 4 + c8)) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
                     }
                 }
                 fence_proxy_async();
@@ -430,22 +447,26 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 // One tcgen05.mma group per chunk: A = [K_i | V_i] (MN-major, two atoms), B = V_i; rows 0..63 of the
 // accumulator are K^T V, rows 64..127 (V^T V) are ignored.
 constexpr int kStStages = 4;
-template <bool kPair>
+template <int kMask>
 struct SmemState {
-    static constexpr int kTilesPerStage = kPair ? 4 : 2;           // K, V (hi) then K, V (lo); adjacent
+    static constexpr int kKV = kMask & 6;                          // bit 1: K is a pair, bit 2: V is a pair
+    static constexpr int kTilesPerStage = 2 + popc3(kKV);          // K, V (hi), then the low planes that exist
+    static constexpr int iKlo = 2, iVlo = 2 + ((kKV >> 1) & 1);
     static constexpr int offStage = 0;
-    static constexpr int offBar = kStStages * kTilesPerStage * kTile;   // full[kStStages], empty[kStStages], done
+    // one spare tile after the ring: a two-atom operand that starts in the ring's last tile reads it
+    static constexpr int offBar = (kStStages * kTilesPerStage + 1) * kTile;   // full[kStStages], empty[kStStages], done
     static constexpr int offTmem = offBar + 8 * (2 * kStStages + 1);
     static constexpr int offAbort = offTmem + 8;
     static constexpr int bytes = offAbort + 8;
 };
 
-template <bool kPair, bool kReverse>
+template <int kMask, bool kReverse>
 __global__ void __launch_bounds__(kThreads)
 linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                      float *__restrict__ s_part, int H, int L, int G, int cpg, int *__restrict__ status)
 {
-    using SM = SmemState<kPair>;
+    using SM = SmemState<kMask>;
+    constexpr int kKV = SM::kKV;
     constexpr int kTPS = SM::kTilesPerStage;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
@@ -487,12 +508,11 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             auto issue_load = [&](int chunk) {
                 const uint32_t bar = bar_full0 + 8 * (chunk % kStStages), dst = sbase + SM::offStage + (chunk % kStStages) * kTPS * kTile;
                 mbar_expect_tx(bar, kTPS * kTile);
-#pragma unroll
-                for (int pl = 0; pl < (kPair ? 2 : 1); ++pl) {
-                    const int t0 = (kReverse ? (L + kC - 1) / kC - 1 - (c0 + chunk) : c0 + chunk) * kC;
-                    tma_load_5d(dst + 2 * pl * kTile, &tm_k, bar, 0, h, t0, b, pl);
-                    tma_load_5d(dst + (2 * pl + 1) * kTile, &tm_v, bar, 0, h, t0, b, pl);
-                }
+                const int t0 = (kReverse ? (L + kC - 1) / kC - 1 - (c0 + chunk) : c0 + chunk) * kC;
+                tma_load_5d(dst, &tm_k, bar, 0, h, t0, b, 0);
+                tma_load_5d(dst + kTile, &tm_v, bar, 0, h, t0, b, 0);
+                if (kKV & 2) tma_load_5d(dst + SM::iKlo * kTile, &tm_k, bar, 0, h, t0, b, 1);
+                if (kKV & 4) tma_load_5d(dst + SM::iVlo * kTile, &tm_v, bar, 0, h, t0, b, 1);
             };
             constexpr uint32_t idesc = make_idesc(128, kD, 1, 1);
             int loads_issued = 0, consumed = 0;
@@ -507,10 +527,13 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 const uint32_t a_lo = desc_lo(st, kTile), v_lo = desc_lo(st + kTile);
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem, a_lo + 128 * k, v_lo + 128 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-                if (kPair) {   // + K_hi^T V_lo + K_lo^T V_hi
-                    const uint32_t a2_lo = desc_lo(st + 2 * kTile, kTile), v2_lo = desc_lo(st + 3 * kTile);
+                if (kKV & 4) {   // + K_hi^T V_lo
+                    const uint32_t v2_lo = desc_lo(st + SM::iVlo * kTile);
 #pragma unroll
                     for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem, a_lo + 128 * k, v2_lo + 128 * k, idesc, 1);
+                }
+                if (kKV & 2) {   // + K_lo^T V_hi (second atom: whatever tile follows; its rows are the ignored ones)
+                    const uint32_t a2_lo = desc_lo(st + SM::iKlo * kTile, kTile);
 #pragma unroll
                     for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem, a2_lo + 128 * k, v_lo + 128 * k, idesc, 1);
                 }
@@ -575,7 +598,7 @@ struct SplitPlan {
     int G, cpg;
     size_t part_bytes;
 };
-SplitPlan split_plan(int B, int H, int L, bool pair)
+SplitPlan split_plan(int B, int H, int L, bool pair)   // pair: the kernel's shared memory allows one CTA per SM only
 {
     int sms = 0;
     int dev = 0;
@@ -601,32 +624,32 @@ SplitPlan split_plan(int B, int H, int L, bool pair)
 }
 constexpr size_t kWsHeader = 512;   // word 0: asynchronous status; the rest: diagnostics
 
-template <typename TOut, bool kPair, bool kReverse>
+template <typename TOut, int kMask, bool kReverse>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
                         float scale, void *workspace, const float *state_in, float *state_out, cudaStream_t stream,
-                        int pair_mask = 7)
+                        int planes_mask)
 {
-    // pair_mask (pair kernels only): bit 0/1/2 set = q/k/v really is a pair.  An operand given as a single bf16
-    // tensor gets a one-plane map; its "low plane" is then out of bounds for the copy engine and arrives as zeros
-    // without touching memory.
+    // planes_mask: which of q, k, v are given with two planes.  An operand that the kernel treats as a pair but
+    // that has one plane gets a one-plane map: its "low plane" is then out of bounds for the copy engine and
+    // arrives as zeros without touching memory (only the full-pair kernel, kMask = 15, is used that way).
     CUtensorMap mq, mk, mv, mo;
-    const int pq = (kPair && (pair_mask & 1)) ? 2 : 1, pk = (kPair && (pair_mask & 2)) ? 2 : 1, pv = (kPair && (pair_mask & 4)) ? 2 : 1;
+    const int pq = (planes_mask & 1) ? 2 : 1, pk = (planes_mask & 2) ? 2 : 1, pv = (planes_mask & 4) ? 2 : 1;
     if (!make_map(&mq, q, B, H, L, kC, false, pq) || !make_map(&mk, k, B, H, L, kC, false, pk) ||
         !make_map(&mv, v, B, H, L, kC, false, pv) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4, 1))
         return CHELA_ERR_CUDA;
-    const SplitPlan plan = split_plan(B, H, L, kPair);
+    const SplitPlan plan = split_plan(B, H, L, Smem<TOut, kMask>::bytes > 113 * 1024);
     int *status = (int *)workspace;
     float *s_part = (float *)((char *)workspace + kWsHeader);
     if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
     if (plan.G > 1) {
-        auto skern = linattn_state_kernel<kPair, kReverse>;
-        if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemState<kPair>::bytes) != cudaSuccess)
-            return CHELA_ERR_CUDA;
-        skern<<<B * H * (plan.G - 1), kThreads, SmemState<kPair>::bytes, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cpg, status);
+        auto skern = linattn_state_kernel<(kMask & 6), kReverse>;
+        constexpr int ssmem = SmemState<(kMask & 6)>::bytes;
+        if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, ssmem) != cudaSuccess) return CHELA_ERR_CUDA;
+        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cpg, status);
         if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
     }
-    auto kern = linattn_sm100_kernel<TOut, kPair, kReverse>;
-    const int smem = Smem<TOut, kPair>::bytes;
+    auto kern = linattn_sm100_kernel<TOut, kMask, kReverse>;
+    const int smem = Smem<TOut, kMask>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return CHELA_ERR_CUDA;
     kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg,
@@ -663,19 +686,28 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
                                          state_out, reverse, pair_mask);
     // The result does not depend on the chunk size: both supported values run on 64-token tiles.
     (void)chunk;
+    const bool pair = in_dtype == CHELA_BF16_PAIR;
+    const int pm = pair ? (pair_mask & 7) : 0;
     if (reverse) {   // anti-causal mirror: fp32 output, no state carry (the backward pass)
         if (out_dtype != CHELA_F32 || state_in || state_out) return CHELA_ERR_UNSUPPORTED;
-        if (in_dtype == CHELA_BF16_PAIR)
-            return launch_t<float, true, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pair_mask);
-        return launch_t<float, false, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream);
+        if (!pair) return launch_t<float, 0, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, 0);
+        if (pm == 2) return launch_t<float, 10, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm);
+        if (pm == 4) return launch_t<float, 12, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm);
+        return CHELA_ERR_UNSUPPORTED;
     }
-    if (in_dtype == CHELA_BF16_PAIR) {
+    if (pair) {
+        // One gradient operand of the backward pass is a pair (or none: scores and state kept as pairs only):
+        // kernels without the absent low planes; fp32 output, no state carry.
+        if (pm != 7 && out_dtype == CHELA_F32 && !state_in && !state_out) {
+            if (pm == 0) return launch_t<float, 8, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm);
+            if (pm == 1) return launch_t<float, 9, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm);
+        }
         if (out_dtype == CHELA_F32)
-            return launch_t<float, true, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pair_mask);
-        return launch_t<__nv_bfloat16, true, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+            return launch_t<float, 15, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pm);
+        return launch_t<__nv_bfloat16, 15, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pm);
     }
-    if (out_dtype == CHELA_F32) return launch_t<float, false, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
-    return launch_t<__nv_bfloat16, false, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+    if (out_dtype == CHELA_F32) return launch_t<float, 0, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 0);
+    return launch_t<__nv_bfloat16, 0, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 0);
 }
 
 }  // namespace chela
