@@ -78,6 +78,8 @@ chela_status_t launch_linattn_bwd_simt(const void *q, const void *k, const void 
 chela_status_t launch_linattn_step(const void *q, const void *k, const void *v, void *o, float *state, int B, int H, int d,
                                    chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
                                    cudaStream_t stream);
+chela_status_t launch_linattn_sm100_grad(const void *q, const void *k, const void *v, const void *d_o, void *g, int B, int H, int L,
+                                         float eps, float scale, void *workspace, cudaStream_t stream);
 bool linattn_bwd_sm100_supported(int d, chela_dtype_t in_dtype);
 size_t linattn_bwd_sm100_workspace_bytes(int B, int H, int L, int d);
 chela_status_t launch_linattn_bwd_sm100(const void *q, const void *k, const void *v, const void *d_o, float *dq, float *dk,

@@ -90,22 +90,32 @@ chela_status_t launch_linattn_bwd_sm100(const void *q, const void *k, const void
     float *r = (float *)(ws + align_up(linattn_sm100_workspace_bytes(B, H, L, d, 64), 256));
     __nv_bfloat16 *g = (__nv_bfloat16 *)(r + n);
     chela_status_t st = CHELA_OK;
-    if (norm)   // r_t = scale * sum_{s<=t} <q_t,k_s> v_s
-        // as a pair kernel whose low input planes are all absent: scores and state keep their low halves, so that
-        // r, which the normaliser differentiates through, is good to fp32 rather than to bf16 scores
+    const void *gp = g;
+    float gscale = 1.0f;
+    if (!norm) {
+        // G = scale * d_o: the gradient launches take d_o itself and the factor
+        gp = d_o;
+        gscale = scale;
+    } else if (d == 64) {
+        // one launch recomputes r (scores and state kept as bf16 pairs: the normaliser differentiates through r,
+        // which therefore has to be good to fp32 rather than to bf16 scores) and writes G from its epilogue
+        st = launch_linattn_sm100_grad(q, k, v, d_o, g, B, H, L, eps, scale, attn_ws, stream);
+        if (st != CHELA_OK) return st;
+    } else {
+        // d = 128: r from the pair kernel with every low input plane absent, then G by an elementwise kernel
         st = launch_linattn_sm100(q, k, v, r, B, H, L, d, 64, CHELA_BF16_PAIR, CHELA_F32, 0, eps, scale, attn_ws, stream,
                                   nullptr, nullptr, false, 0);
-    if (st != CHELA_OK) return st;
-    const int blocks = (int)((rows + 7) / 8 < (size_t)148 * 16 ? (rows + 7) / 8 : (size_t)148 * 16);
-    if (d == 64) bwd_prep_kernel<64><<<blocks, 256, 0, stream>>>(r, (const __nv_bfloat16 *)d_o, g, rows, scale, norm, eps);
-    else bwd_prep_kernel<128><<<blocks, 256, 0, stream>>>(r, (const __nv_bfloat16 *)d_o, g, rows, scale, norm, eps);
-    if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
+        if (st != CHELA_OK) return st;
+        const int blocks = (int)((rows + 7) / 8 < (size_t)148 * 16 ? (rows + 7) / 8 : (size_t)148 * 16);
+        bwd_prep_kernel<128><<<blocks, 256, 0, stream>>>(r, (const __nv_bfloat16 *)d_o, g, rows, scale, norm, eps);
+        if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
+    }
     const chela_dtype_t dt = norm ? CHELA_BF16_PAIR : CHELA_BF16;   // the pair is G, in a different role each time
-    st = launch_linattn_sm100(g, v, k, dq, B, H, L, d, 64, dt, CHELA_F32, 0, eps, 1.0f, attn_ws, stream, nullptr, nullptr, false, 1);
+    st = launch_linattn_sm100(gp, v, k, dq, B, H, L, d, 64, dt, CHELA_F32, 0, eps, gscale, attn_ws, stream, nullptr, nullptr, false, 1);
     if (st != CHELA_OK) return st;
-    st = launch_linattn_sm100(v, g, q, dk, B, H, L, d, 64, dt, CHELA_F32, 0, eps, 1.0f, attn_ws, stream, nullptr, nullptr, true, 2);
+    st = launch_linattn_sm100(v, gp, q, dk, B, H, L, d, 64, dt, CHELA_F32, 0, eps, gscale, attn_ws, stream, nullptr, nullptr, true, 2);
     if (st != CHELA_OK) return st;
-    return launch_linattn_sm100(k, q, g, dv, B, H, L, d, 64, dt, CHELA_F32, 0, eps, 1.0f, attn_ws, stream, nullptr, nullptr, true, 4);
+    return launch_linattn_sm100(k, q, gp, dv, B, H, L, d, 64, dt, CHELA_F32, 0, eps, gscale, attn_ws, stream, nullptr, nullptr, true, 4);
 }
 
 }  // namespace chela

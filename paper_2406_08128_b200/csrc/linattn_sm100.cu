@@ -40,22 +40,26 @@ constexpr int kTile = kC * 128;   // one 64-row x 128-byte tile
 // more tensor-core term per pair side (hi*hi + hi*lo + lo*hi; lo*lo is dropped).  0 = the plain bf16 kernel, 15 = the
 // mixer's attention; the backward pass uses 8 (recomputed forward), 9, 10 and 12 (one gradient operand is a pair).
 __host__ __device__ constexpr int popc3(int m) { return (m & 1) + ((m >> 1) & 1) + ((m >> 2) & 1); }
-template <typename TOut, int kMask>
+// kGrad (backward pass, with kMask = 8): the epilogue does not store the output row but pulls the output gradient
+// d_o back through the normaliser, G = scale (d_o - o <o, d_o> / d) / n, and stores G as a bf16 pair; the d_o tiles
+// are one more tile of every stage.
+template <typename TOut, int kMask, bool kGrad = false>
 struct Smem {
     static constexpr int kIn = kMask & 7;
     static constexpr bool kPPair = (kMask & 8) != 0;
-    static constexpr int kTilesPerStage = 3 + popc3(kIn);   // Q, K, V (hi), then the low planes that exist, in that order
+    static constexpr int kTilesPerStage = 3 + popc3(kIn) + (kGrad ? 1 : 0);   // Q, K, V (hi), the low planes that exist, d_o (kGrad)
+    static constexpr int iD = 3 + popc3(kIn);
     static constexpr int iQlo = 3, iKlo = 3 + (kIn & 1), iVlo = 3 + popc3(kIn & 3);
     static constexpr int kStages = (kMask == 0) ? 3 : 2;
-    static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as 128-byte wide boxes
+    static constexpr int kOBoxes = kGrad ? 2 : (int)sizeof(TOut) * kD / 128;   // output staged as 128-byte wide boxes (kGrad: hi, lo)
     static constexpr int offPT = 0;                       // masked scores, transposed: rows = s, 64 t per row (hi, lo)
     static constexpr int offShi = offPT + (kPPair ? 2 : 1) * kTile;   // state, bf16 high part: rows = d_k
     static constexpr int offSlo = offShi + kTile;         // state, bf16 low part
     static constexpr int offStage = offSlo + kTile;       // after the score tile: the G3 descriptor reaches K from P forwards
     // output staging; also what a 128-row operand that starts in the last tile of the last stage reads past it
     static constexpr int offO = offStage + kStages * kTilesPerStage * kTile;
-    static constexpr int offBar = offO + (kOBoxes > 1 ? kOBoxes : 1) * kTile;   // full[kStages], p, o, pt, s
-    static constexpr int offTmem = offBar + 8 * (kStages + 4);
+    static constexpr int offBar = offO + (kOBoxes > 1 ? kOBoxes : 1) * kTile;   // full[kStages], p, o, pt, s, dr
+    static constexpr int offTmem = offBar + 8 * (kStages + 5);
     static constexpr int offAbort = offTmem + 8;
     static constexpr int bytes = offAbort + 8;
 };
@@ -76,17 +80,20 @@ constexpr int kColPT = 64;   // rows 64..127: transposed scores; 64 columns
 // kReverse: the anti-causal mirror (token t attends keys s >= t; the state accumulates from the end of the
 // sequence).  Chunks are walked from the last to the first and the mask is the upper triangle; everything
 // else, including the split into groups, works on the mirrored chunk index.  Used by the backward pass.
-template <typename TOut, int kMask, bool kReverse>
-__global__ void __launch_bounds__(kThreads)
+template <typename TOut, int kMask, bool kReverse, bool kGrad = false>
+// Two CTAs per SM wherever shared memory allows (every mask but 15): 10 warps over the four register files put
+// three on one of them, which caps a thread at 168 registers.
+__global__ void __launch_bounds__(kThreads, kMask == 15 ? 1 : 2)
 linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
+                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                     const __grid_constant__ CUtensorMap tm_d, int H, int L,
                      float scale, int norm, float eps, int *__restrict__ status, const float *__restrict__ s_part,
                      int G, int cpg, const float *__restrict__ state_in, float *__restrict__ state_out)
 {
     // Grid: one CTA per (batch*head, group).  Group g covers chunks [g*cpg, (g+1)*cpg) of its sequence and
     // starts from the state sum_{g' < g} s_part[bh][g'] (per-group K^T V sums written by the state kernel),
     // plus the caller's initial state state_in[bh] if given; the last group writes the final state.
-    using SM = Smem<TOut, kMask>;
+    using SM = Smem<TOut, kMask, kGrad>;
     constexpr int kStages = SM::kStages;
     constexpr int kTPS = SM::kTilesPerStage;
     constexpr int kIn = SM::kIn;
@@ -112,6 +119,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const uint32_t bar_o = bar_p + 8;                 // G2 + G3 of a chunk have completed (-> all roles)
     const uint32_t bar_pt = bar_o + 8;                // score tile of a chunk is in shared memory (warps 2,3 -> issuer)
     const uint32_t bar_s = bar_pt + 8;                // output/state rows read, state tiles written (4 warps -> issuer)
+    const uint32_t bar_dr = bar_s + 8;                // kGrad: both epilogue warps hold their d_o rows of a chunk (-> issuer)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
 
@@ -121,6 +129,10 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         mbar_init(bar_o, 1);
         mbar_init(bar_pt, 2);
         mbar_init(bar_s, 4);
+        if (kGrad) {
+            mbar_init(bar_dr, 2);
+            tma_prefetch_desc(&tm_d);
+        }
         *abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tm_q);
@@ -151,6 +163,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (kIn & 1) tma_load_5d(dst + SM::iQlo * kTile, &tm_q, bar, 0, h, tok(chunk), b, 1);
                 if (kIn & 2) tma_load_5d(dst + SM::iKlo * kTile, &tm_k, bar, 0, h, tok(chunk), b, 1);
                 if (kIn & 4) tma_load_5d(dst + SM::iVlo * kTile, &tm_v, bar, 0, h, tok(chunk), b, 1);
+                if (kGrad) tma_load_5d(dst + SM::iD * kTile, &tm_d, bar, 0, h, tok(chunk), b, 0);
             };
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [Q;K] (K-major) x Q^T (K-major)
             constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;K] (K-major) x S (MN-major)
@@ -233,6 +246,10 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 // the stage is free once G3 has completed: prefetch the chunk that will use it next
                 ok = mbar_wait(bar_o, i & 1, abort_flag);
                 if (!ok) break;
+                if (kGrad) {   // the stage also holds the d_o tile: wait until the epilogue warps have copied their rows
+                    ok = mbar_wait(bar_dr, i & 1, abort_flag);
+                    if (!ok) break;
+                }
                 consumed = i + 1;
                 if (i + kStages < nchunks) {
                     issue_load(i + kStages);
@@ -355,6 +372,16 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (lane == 0) mbar_arrive(bar_pt);
                 TMARK(1);
             }
+            uint4 dq4[kGrad ? 8 : 1];   // kGrad: row t of d_o (64 bf16), copied out of the stage before the stage can be reloaded
+            if (kGrad && !upper) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_full0 + 8 * (i % kStages), (i / kStages) & 1, abort_flag));
+                if (!ok) break;
+                const uint8_t *sD = smem + SM::offStage + ((i % kStages) * kTPS + SM::iD) * kTile;
+#pragma unroll
+                for (int c8 = 0; c8 < 8; ++c8) dq4[c8] = *reinterpret_cast<const uint4 *>(sD + sw128(r, c8));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_dr);
+            }
             ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
@@ -380,7 +407,34 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 }
                 const float inv = norm ? rsqrtf(ss * (1.0f / kD) + eps) : 1.0f;
                 uint8_t *sO = smem + SM::offO;
-                if (sizeof(TOut) == 4) {
+                if (kGrad) {
+                    // acc = r (scaled); o = r inv; G = scale (d_o - o <o, d_o> / d) inv, stored as hi and lo planes
+                    float od = 0.f;
+                    const __nv_bfloat162 *dh = reinterpret_cast<const __nv_bfloat162 *>(dq4);
+#pragma unroll
+                    for (int j = 0; j < kD / 2; ++j) {
+                        const float2 d2 = __bfloat1622float2(dh[j]);
+                        od = fmaf(acc[2 * j] * inv, d2.x, od);
+                        od = fmaf(acc[2 * j + 1] * inv, d2.y, od);
+                    }
+                    od *= 1.0f / kD;
+#pragma unroll
+                    for (int c8 = 0; c8 < 8; ++c8) {
+                        uint32_t wh[4], wl[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int j = c8 * 4 + e;
+                            const float2 d2 = __bfloat1622float2(dh[j]);
+                            const float g0 = scale * (d2.x - acc[2 * j] * inv * od) * inv, g1 = scale * (d2.y - acc[2 * j + 1] * inv * od) * inv;
+                            const __nv_bfloat162 hh = __floats2bfloat162_rn(g0, g1);
+                            const float2 hf = __bfloat1622float2(hh);
+                            wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                            wl[e] = pack_bf16(g0 - hf.x, g1 - hf.y);
+                        }
+                        *reinterpret_cast<uint4 *>(sO + sw128(r, c8)) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                        *reinterpret_cast<uint4 *>(sO + kTile + sw128(r, c8)) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                    }
+                } else if (sizeof(TOut) == 4) {
 #pragma unroll
                     for (int j = 0; j < kD; j += 4)
                         *reinterpret_cast<float4 *>(sO + (j / 32) * kTile + sw128(r, (j % 32) / 4)) =
@@ -398,8 +452,11 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (lane == 0) {
 #pragma unroll
                     for (int bx = 0; bx < SM::kOBoxes; ++bx)
-                        tma_store_5d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
-                                     tok(i) + warp * 32, b, 0);   // the map's rank is 5 (plane = 0)
+                        if (kGrad)   // box = plane (hi, lo)
+                            tma_store_5d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, 0, h, tok(i) + warp * 32, b, bx);
+                        else
+                            tma_store_5d(&tm_o, sbase + SM::offO + bx * kTile + warp * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
+                                         tok(i) + warp * 32, b, 0);   // the map's rank is 5 (plane = 0)
                     bulk_commit();
                 }
                 TMARK(3);
@@ -652,12 +709,46 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
     const int smem = Smem<TOut, kMask>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return CHELA_ERR_CUDA;
-    kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg,
+    kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg,
                                                      state_in, state_out);
     return last_launch_status();
 }
 
+// Backward pass, first launch: recomputes the forward rows (scores and state kept as bf16 pairs) and writes
+// G = d_o pulled back through the normaliser, as a bf16 pair (two planes at g).
+chela_status_t launch_grad(const void *q, const void *k, const void *v, const void *d_o, void *g, int B, int H, int L, float eps,
+                           float scale, void *workspace, cudaStream_t stream)
+{
+    CUtensorMap mq, mk, mv, mg, md;
+    if (!make_map(&mq, q, B, H, L, kC, false, 1) || !make_map(&mk, k, B, H, L, kC, false, 1) || !make_map(&mv, v, B, H, L, kC, false, 1) ||
+        !make_map(&md, d_o, B, H, L, kC, false, 1) || !make_map(&mg, g, B, H, L, 32, false, 2))
+        return CHELA_ERR_CUDA;
+    using SM = Smem<__nv_bfloat16, 8, true>;
+    const SplitPlan plan = split_plan(B, H, L, SM::bytes > 113 * 1024);
+    int *status = (int *)workspace;
+    float *s_part = (float *)((char *)workspace + kWsHeader);
+    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+    if (plan.G > 1) {
+        auto skern = linattn_state_kernel<0, false>;
+        constexpr int ssmem = SmemState<0>::bytes;
+        if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, ssmem) != cudaSuccess) return CHELA_ERR_CUDA;
+        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cpg, status);
+        if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
+    }
+    auto kern = linattn_sm100_kernel<__nv_bfloat16, 8, false, true>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::bytes) != cudaSuccess) return CHELA_ERR_CUDA;
+    kern<<<B * H * plan.G, kThreads, SM::bytes, stream>>>(mq, mk, mv, mg, md, H, L, scale, 1, eps, status, s_part, plan.G, plan.cpg,
+                                                          nullptr, nullptr);
+    return last_launch_status();
+}
+
 }  // namespace
+
+chela_status_t launch_linattn_sm100_grad(const void *q, const void *k, const void *v, const void *d_o, void *g, int B, int H, int L,
+                                         float eps, float scale, void *workspace, cudaStream_t stream)
+{
+    return launch_grad(q, k, v, d_o, g, B, H, L, eps, scale, workspace, stream);
+}
 
 bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype)
 {
