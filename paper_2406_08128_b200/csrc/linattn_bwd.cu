@@ -4,14 +4,16 @@
 //   dQ = causal(q <- G, k <- V, v <- K)            dq_t = sum_{s<=t} <g_t,v_s> k_s
 //   dK = anti-causal(q <- V, k <- G, v <- Q)       dk_s = sum_{t>=s} <v_s,g_t> q_t
 //   dV = anti-causal(q <- K, k <- Q, v <- G)       dv_s = sum_{t>=s} <k_s,q_t> g_t
-// so the pass is: the forward kernel without normaliser (recomputes r; nothing is saved by the forward pass),
-// one elementwise kernel (r, d_o -> G), and three more launches of the forward kernel, two of them in its
-// mirrored (anti-causal) mode.
+// so the pass is four launches of the forward kernel (nothing is saved by the forward pass): one that recomputes
+// r and writes G from its epilogue (d = 64; for d = 128 the forward kernel writes r and an elementwise kernel
+// makes G), and three that evaluate the gradients, two of them in the mirrored (anti-causal) mode.
 // With the normaliser G is a bf16 pair (hi + lo): g_t is orthogonal to r_t up to eps / n_t^2, so dq, dk are
 // residuals of a cancellation wherever n_t is small, and a G rounded to 8 bits loses them (measured 0.04-0.35
-// of RMS).  The three launches then run the pair kernel with one real pair operand; the other two are single
-// bf16 tensors whose absent low planes the copy engine zero-fills.  Without the normaliser G = scale * d_o is
-// rounded to bf16 like every other operand and the single-bf16 kernel is used.
+// of RMS); r itself, which the normaliser differentiates through, is recomputed with scores and state kept as
+// pairs, and so are the scores of the gradient launches (single-bf16 scores there: 1-3e-2 of RMS).  Each
+// gradient launch has one pair operand (G, in a different role each time) and runs the kernel variant that
+// carries exactly that low plane.  Without the normaliser G = scale * d_o: the launches take d_o itself, the
+// factor goes into their scale argument, and the plain bf16 kernel is used.
 #include "common.cuh"
 
 namespace chela {
