@@ -34,7 +34,7 @@ METRIC = "linattn_fwd_tokens_per_s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture
 # summarised in profiles/linattn_sm100_L2048_B16_ncu_full.md: 294.8 MB for 32768 tokens (B=16, L=2048, same
 # grid), scaled by tokens to the timed workload (traffic is proportional to tokens: every tile is read once)
-NCU_TRAFFIC_BYTES_PER_TOKEN = 294.8e6 / 32768
+NCU_TRAFFIC_BYTES_PER_TOKEN = 293.9e6 / 32768
 FALLBACK_HBM_GBS = 6650.0
 
 
