@@ -13,7 +13,8 @@ TOLB = 1e-4
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("B,L,H,d", [(1, 1, 1, 64), (2, 63, 2, 64), (1, 300, 3, 64), (2, 1000, 2, 64), (1, 200, 2, 128),
-                                     (1, 777, 1, 128)])
+                                     (1, 777, 1, 128),
+                                     (1, 2100, 1, 64), (1, 2100, 1, 128)])   # the last two: split along L (state kernel)
 @pytest.mark.parametrize("norm", [True, False])
 def test_gradients_match_the_oracle(dtype, B, L, H, d, norm):
     q, k, v = inputs.qkv(70 + L + d, B, L, H, d, d, dtype)
