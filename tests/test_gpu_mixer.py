@@ -68,6 +68,18 @@ def test_mixer_config3_shape_one_batch():
     assert rel_err(got, ref) <= TOL
 
 
+@pytest.mark.parametrize("seed,B,L,D,H,chunk", [(2, 4, 16384, 512, 8, 64), (3, 8, 8192, 1024, 8, 128)])
+def test_mixer_configs_3_and_4_full_size_sampled_rows(seed, B, L, D, H, chunk):
+    """Configs 3 and 4 at their full sizes, i.e. the launch configuration the benchmark times; the oracle checks
+    the first and the last batch row (rows are independent: a row's oracle takes its slice of x alone)."""
+    m = inputs.mixer(seed, B, L, D)
+    got = run_mixer(m, H, chunk)
+    assert np.isfinite(got).all()
+    for b in (0, B - 1):
+        ref = oracle.mixer(m["x"][b:b + 1], m["w_short"], m["k_long"], m["w_q"], m["w_k"], m["w_v"], H)
+        assert rel_err(got[b:b + 1], ref) <= TOL, b
+
+
 @pytest.mark.parametrize("B,L,D,H,chunk,dtype", [(2, 300, 128, 2, 64, "bf16"), (1, 1000, 256, 2, 128, "bf16"),
                                                  (1, 2048, 512, 8, 64, "bf16"), (1, 200, 64, 1, 64, "f32")])
 def test_gated_mixer(B, L, D, H, chunk, dtype):
