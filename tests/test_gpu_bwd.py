@@ -44,3 +44,42 @@ def test_backward_argument_checks():
     with pytest.raises(chela.ChelaError) as e:
         chela.linattn_bwd(q32, q32, q32, q32, workspace=torch.zeros(1 << 20, dtype=torch.uint8, device="cuda"))
     assert e.value.status == chela.ERR_UNSUPPORTED
+
+
+def test_backward_at_the_benchmark_size_by_directional_derivatives():
+    """B16 L16384 H16 d64 bf16, the launch configuration the benchmark times.  The O(L^2) gradient oracle takes most
+    of a minute per head there, so the check uses a property that holds at any size: for sampled (batch, head)
+    pairs, the gradients' inner product with a direction equals the central difference of the float64 oracle's
+    forward pass along that direction.  Directions: the computed gradient itself (overall scale), and random
+    directions confined to one token row of q, k or v (64 numbers, so that the inner product is a sizeable
+    fraction of |g_row| |direction| and a wrong row shows)."""
+    import torch
+    B, L, H, d = 16, 16384, 16, 64
+    q, k, v = inputs.qkv(90, B, L, H, d, d, "bf16")
+    d_o = inputs.qkv(91, B, L, H, d, d, "bf16", std=1.0)[0]
+    dq, dk, dv = chela.linattn_bwd(*(to_device(a, "bf16") for a in (q, k, v, d_o)), norm=chela.NORM_RMS, scale=1.0)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(92)
+
+    def central_difference(x, go, dirs, eps):
+        f = [float((go * oracle.linattn_recurrent(*[a + s * eps * dd for a, dd in zip(x, dirs)])).sum()) for s in (1.0, -1.0)]
+        return (f[0] - f[1]) / (2 * eps)
+
+    for b, h in ((0, 0), (B - 1, H - 1), (int(rng.integers(B)), int(rng.integers(H)))):
+        sl = (slice(b, b + 1), slice(None), slice(h, h + 1))
+        x = [np.asarray(a[sl], dtype=np.float64) for a in (q, k, v)]
+        go = np.asarray(d_o[sl], dtype=np.float64)
+        grads = [to_numpy(g[b:b + 1, :, h:h + 1]).astype(np.float64) for g in (dq, dk, dv)]
+        # along the gradient: num = <g_true, g>, ana = |g|^2
+        gnorm2 = sum(float((g * g).sum()) for g in grads)
+        num = central_difference(x, go, grads, 1e-4 / np.sqrt(gnorm2 / (3 * L * d)))
+        assert abs(num - gnorm2) <= 2e-3 * gnorm2, (b, h, num, gnorm2)
+        # one token row of one operand at a time (early, late and random tokens)
+        for which in range(3):
+            for t in (0, L - 1, int(rng.integers(L)), int(rng.integers(L))):
+                dirs = [np.zeros_like(a) for a in x]
+                dirs[which][0, t, 0, :] = rng.standard_normal(d)
+                grow, drow = grads[which][0, t, 0, :], dirs[which][0, t, 0, :]
+                ana = float((grow * drow).sum())
+                num = central_difference(x, go, dirs, 1e-3)
+                assert abs(num - ana) <= 1e-2 * np.linalg.norm(grow) * np.linalg.norm(drow), (b, h, which, t, num, ana)
