@@ -88,11 +88,14 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                      const __grid_constant__ CUtensorMap tm_d, int H, int L,
                      float scale, int norm, float eps, int *__restrict__ status, const float *__restrict__ s_part,
-                     int G, int cpg, const float *__restrict__ state_in, float *__restrict__ state_out)
+                     int G, int cg0, int cg, const float *__restrict__ state_in, float *__restrict__ state_out)
 {
-    // Grid: one CTA per (batch*head, group).  Group g covers chunks [g*cpg, (g+1)*cpg) of its sequence and
-    // starts from the state sum_{g' < g} s_part[bh][g'] (per-group K^T V sums written by the state kernel),
-    // plus the caller's initial state state_in[bh] if given; the last group writes the final state.
+    // Grid: one CTA per (group, batch*head), group-major.  Group 0 covers the first cg0 chunks of its sequence, group
+    // g >= 1 the next cg chunks each (the last one what is left).  Group g starts from the state
+    // sum_{g' < g} s_part[bh][g'] (per-group K^T V sums written by the state kernel), plus the caller's initial state
+    // state_in[bh] if given; the last group writes the final state.  When G > 1 this kernel is launched as a
+    // programmatic dependent of the state kernel: group 0 needs nothing from it and runs beside it (hence the longer
+    // first group), the other groups wait for it before they read s_part.
     using SM = Smem<TOut, kMask, kGrad>;
     constexpr int kStages = SM::kStages;
     constexpr int kTPS = SM::kTilesPerStage;
@@ -105,11 +108,12 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         return;
     }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x / G, g = blockIdx.x % G;
+    const int nbh = gridDim.x / G;
+    const int bh = blockIdx.x % nbh, g = blockIdx.x / nbh;
     const int b = bh / H, h = bh % H;
-    const int c0 = g * cpg;                                        // first (mirrored) chunk of this group
+    const int c0 = g == 0 ? 0 : cg0 + (g - 1) * cg;                // first (mirrored) chunk of this group
     const int nch_total = (L + kC - 1) / kC;
-    const int nchunks = min(cpg, nch_total - c0);                  // chunks of this group
+    const int nchunks = min(g == 0 ? cg0 : cg, nch_total - c0);    // chunks of this group
     // token offset of the group's chunk number `chunk`
     auto tok = [&](int chunk) { return (kReverse ? nch_total - 1 - (c0 + chunk) : c0 + chunk) * kC; };
     const bool has_init = g > 0 || state_in != nullptr;
@@ -311,6 +315,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         sv[4 * j] = x.x; sv[4 * j + 1] = x.y; sv[4 * j + 2] = x.z; sv[4 * j + 3] = x.w;
                     }
                 }
+                if (g > 0) griddep_wait();   // the state kernel has completed
                 for (int gp = 0; gp < g; ++gp) {
                     const float4 *src = reinterpret_cast<const float4 *>(s_part + (((size_t)bh * (G - 1) + gp) * kD + r) * kD);
 #pragma unroll
@@ -520,7 +525,7 @@ struct SmemState {
 template <int kMask, bool kReverse>
 __global__ void __launch_bounds__(kThreads)
 linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                     float *__restrict__ s_part, int H, int L, int G, int cpg, int *__restrict__ status)
+                     float *__restrict__ s_part, int H, int L, int G, int cg0, int cg, int *__restrict__ status)
 {
     using SM = SmemState<kMask>;
     constexpr int kKV = SM::kKV;
@@ -532,9 +537,12 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         return;
     }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x / (G - 1), g = blockIdx.x % (G - 1);
+    griddep_launch_dependents();   // the main kernel's first groups may be scheduled beside this kernel
+    // group-major like the main kernel, longest group (0) first
+    const int nbh = gridDim.x / (G - 1);
+    const int bh = blockIdx.x % nbh, g = blockIdx.x / nbh;
     const int b = bh / H, h = bh % H;
-    const int c0 = g * cpg, nchunks = cpg;    // every group but the last is full
+    const int c0 = g == 0 ? 0 : cg0 + (g - 1) * cg, nchunks = g == 0 ? cg0 : cg;    // every group but the last is full
 
     const uint32_t bar_full0 = sbase + SM::offBar, bar_empty0 = bar_full0 + 8 * kStStages,
                    bar_done = bar_empty0 + 8 * kStStages;
@@ -650,9 +658,11 @@ bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int C, boo
 }
 
 // How a call is split along L.  The grid holds B*H*G CTAs, no more than are resident at once (two per SM,
-// one per SM for bf16-pair inputs); a group never has fewer than 16 chunks.
+// one per SM for the full-pair kernel); a group never has fewer than 16 chunks.  Group 0 is longer than the
+// others when there are two: it runs beside the state kernel, the second starts when that has finished, and both
+// should end together.
 struct SplitPlan {
-    int G, cpg;
+    int G, cg0, cg;
     size_t part_bytes;
 };
 SplitPlan split_plan(int B, int H, int L, bool pair)   // pair: the kernel's shared memory allows one CTA per SM only
@@ -674,10 +684,39 @@ SplitPlan split_plan(int B, int H, int L, bool pair)   // pair: the kernel's sha
         if (G < 1) G = 1;
     }
     SplitPlan p;
-    p.cpg = (nchunks + G - 1) / G;
-    p.G = (nchunks + p.cpg - 1) / p.cpg;
+    if (G == 1) {
+        p.G = 1;
+        p.cg0 = p.cg = nchunks;
+    } else {
+        // cg / cg0, measured on B200 (L = 32K...128K, B*H = 32...128): with two groups everything is resident at once and
+        // the first group should be twice the second; with more groups the later ones queue for CTA slots behind the
+        // state kernel anyway and equal groups are best
+        const double rho = G == 2 ? 0.5 : 1.0;
+        p.cg0 = (int)((double)nchunks / (1.0 + (G - 1) * rho) + 0.999);
+        if (p.cg0 > nchunks - (G - 1)) p.cg0 = nchunks - (G - 1);
+        p.cg = (nchunks - p.cg0 + G - 2) / (G - 1);
+        p.G = 1 + (nchunks - p.cg0 + p.cg - 1) / p.cg;
+    }
     p.part_bytes = (size_t)bh * (p.G - 1) * kD * kD * sizeof(float);
     return p;
+}
+
+// The main kernel after the state kernel of the same call, allowed to start while that still runs.
+template <typename Kern, typename... Args>
+chela_status_t launch_dependent(Kern kern, int grid, int smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, args...) != cudaSuccess) return CHELA_ERR_CUDA;
+    return last_launch_status();
 }
 constexpr size_t kWsHeader = 512;   // word 0: asynchronous status; the rest: diagnostics
 
@@ -702,15 +741,18 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
         auto skern = linattn_state_kernel<(kMask & 6), kReverse>;
         constexpr int ssmem = SmemState<(kMask & 6)>::bytes;
         if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, ssmem) != cudaSuccess) return CHELA_ERR_CUDA;
-        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cpg, status);
+        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cg0, plan.cg, status);
         if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
     }
     auto kern = linattn_sm100_kernel<TOut, kMask, kReverse>;
     const int smem = Smem<TOut, kMask>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return CHELA_ERR_CUDA;
-    kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg,
-                                                     state_in, state_out);
+    if (plan.G > 1)
+        return launch_dependent(kern, B * H * plan.G, smem, stream, mq, mk, mv, mo, mo, H, L, scale, norm, eps, status,
+                                (const float *)s_part, plan.G, plan.cg0, plan.cg, state_in, state_out);
+    kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, mo, mo, H, L, scale, norm, eps, status, s_part, 1, plan.cg0, plan.cg,
+                                            state_in, state_out);
     return last_launch_status();
 }
 
@@ -732,13 +774,16 @@ chela_status_t launch_grad(const void *q, const void *k, const void *v, const vo
         auto skern = linattn_state_kernel<0, false>;
         constexpr int ssmem = SmemState<0>::bytes;
         if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, ssmem) != cudaSuccess) return CHELA_ERR_CUDA;
-        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cpg, status);
+        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cg0, plan.cg, status);
         if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
     }
     auto kern = linattn_sm100_kernel<__nv_bfloat16, 8, false, true>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::bytes) != cudaSuccess) return CHELA_ERR_CUDA;
-    kern<<<B * H * plan.G, kThreads, SM::bytes, stream>>>(mq, mk, mv, mg, md, H, L, scale, 1, eps, status, s_part, plan.G, plan.cpg,
-                                                          nullptr, nullptr);
+    if (plan.G > 1)
+        return launch_dependent(kern, B * H * plan.G, SM::bytes, stream, mq, mk, mv, mg, md, H, L, scale, 1, eps, status,
+                                (const float *)s_part, plan.G, plan.cg0, plan.cg, (const float *)nullptr, (float *)nullptr);
+    kern<<<B * H, kThreads, SM::bytes, stream>>>(mq, mk, mv, mg, md, H, L, scale, 1, eps, status, s_part, 1, plan.cg0, plan.cg,
+                                                 nullptr, nullptr);
     return last_launch_status();
 }
 
