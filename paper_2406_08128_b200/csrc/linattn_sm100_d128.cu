@@ -49,10 +49,12 @@ __global__ void __launch_bounds__(kThreads)
 linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
                           float scale, int norm, float eps, int *__restrict__ status, const float *__restrict__ s_part, int G,
-                          int cpg, const float *__restrict__ state_in, float *__restrict__ state_out)
+                          int cg0, int cg, const float *__restrict__ state_in, float *__restrict__ state_out)
 {
-    // Grid: one CTA per (batch*head, group); group g covers chunks [g*cpg, (g+1)*cpg) and starts from
-    // state_in[bh] + sum_{g' < g} s_part[bh][g'] (128 x 128 fp32 each); the last group writes state_out[bh].
+    // Grid: one CTA per (group, batch*head), group-major; group 0 covers the first cg0 chunks, group g >= 1 the next
+    // cg each, and starts from state_in[bh] + sum_{g' < g} s_part[bh][g'] (128 x 128 fp32 each); the last group
+    // writes state_out[bh].  With G > 1 the kernel is a programmatic dependent of the state kernel: group 0 runs
+    // beside it, the others wait for it before reading s_part.
     using SM = Smem<TOut, kPair>;
     constexpr int kStages = SM::kStages, kPlanes = SM::kPlanes;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -62,11 +64,12 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         return;
     }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x / G, g = blockIdx.x % G;
+    const int nbh = gridDim.x / G;
+    const int bh = blockIdx.x % nbh, g = blockIdx.x / nbh;
     const int b = bh / H, h = bh % H;
-    const int c0 = g * cpg;
+    const int c0 = g == 0 ? 0 : cg0 + (g - 1) * cg;
     const int nch_total = (L + kC - 1) / kC;
-    const int nchunks = min(cpg, nch_total - c0);
+    const int nchunks = min(g == 0 ? cg0 : cg, nch_total - c0);
     const bool has_init = g > 0 || state_in != nullptr;
     auto tok = [&](int chunk) { return (kReverse ? nch_total - 1 - (c0 + chunk) : c0 + chunk) * kC; };
 
@@ -261,6 +264,7 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                             }
                         };
                         if (state_in) add_row(state_in + (size_t)bh * kD * kD);
+                        if (g > 0) griddep_wait();   // the state kernel has completed
                         for (int gp = 0; gp < g; ++gp) add_row(s_part + ((size_t)bh * (G - 1) + gp) * kD * kD);
                         const uint32_t col = (x == 0 ? kColOS : kColSb) + 64 * half;
                         tmem_st32(tmem_warp + col, *reinterpret_cast<const float(*)[32]>(&sv[0]));
@@ -420,7 +424,7 @@ struct SmemState {
 template <bool kPair, bool kReverse>
 __global__ void __launch_bounds__(kThreads)
 linattn_state_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                          float *__restrict__ s_part, int H, int L, int G, int cpg, int *__restrict__ status)
+                          float *__restrict__ s_part, int H, int L, int G, int cg0, int cg, int *__restrict__ status)
 {
     using SM = SmemState<kPair>;
     constexpr int kStages = SM::kStages, kPlanes = SM::kPlanes;
@@ -431,9 +435,11 @@ linattn_state_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid
         return;
     }
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x / (G - 1), g = blockIdx.x % (G - 1);
+    griddep_launch_dependents();   // the main kernel's first groups may be scheduled beside this kernel
+    const int nbh = gridDim.x / (G - 1);
+    const int bh = blockIdx.x % nbh, g = blockIdx.x / nbh;
     const int b = bh / H, h = bh % H;
-    const int c0 = g * cpg, nchunks = cpg;
+    const int c0 = g == 0 ? 0 : cg0 + (g - 1) * cg, nchunks = g == 0 ? cg0 : cg;
     const uint32_t bar_full0 = sbase + SM::offBar, bar_empty0 = bar_full0 + 8 * kStages, bar_done = bar_empty0 + 8 * kStages;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
@@ -544,7 +550,7 @@ bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int box_ro
 
 // Split along L: one CTA per SM is resident (shared memory), at least 16 chunks per group.
 struct SplitPlan {
-    int G, cpg;
+    int G, cg0, cg;   // group 0: cg0 chunks, the others cg (two groups: the first a quarter longer, it runs beside the state kernel)
     size_t part_bytes;
 };
 SplitPlan split_plan(int B, int H, int L)
@@ -561,8 +567,16 @@ SplitPlan split_plan(int B, int H, int L)
         if (G < 1) G = 1;
     }
     SplitPlan p;
-    p.cpg = (nchunks + G - 1) / G;
-    p.G = (nchunks + p.cpg - 1) / p.cpg;
+    if (G == 1) {
+        p.G = 1;
+        p.cg0 = p.cg = nchunks;
+    } else {
+        const double rho = G == 2 ? 0.8 : 1.0;   // measured: one CTA per SM, the state pass costs 0.23 of the main pass per chunk
+        p.cg0 = (int)((double)nchunks / (1.0 + (G - 1) * rho) + 0.999);
+        if (p.cg0 > nchunks - (G - 1)) p.cg0 = nchunks - (G - 1);
+        p.cg = (nchunks - p.cg0 + G - 2) / (G - 1);
+        p.G = 1 + (nchunks - p.cg0 + p.cg - 1) / p.cg;
+    }
     p.part_bytes = (size_t)bh * (p.G - 1) * kD * kD * sizeof(float);
     return p;
 }
@@ -588,14 +602,30 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
         auto skern = linattn_state_d128_kernel<kPair, kReverse>;
         if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemState<kPair>::bytes) != cudaSuccess)
             return CHELA_ERR_CUDA;
-        skern<<<B * H * (plan.G - 1), kThreads, SmemState<kPair>::bytes, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cpg, status);
+        skern<<<B * H * (plan.G - 1), kThreads, SmemState<kPair>::bytes, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cg0, plan.cg, status);
         if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
     }
     auto kern = linattn_sm100_d128_kernel<TOut, kPair, kReverse>;
     const int smem = Smem<TOut, kPair>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
-    kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cpg,
-                                                     state_in, state_out);
+    if (plan.G > 1) {   // may start while the state kernel still runs
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(B * H * plan.G);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, kern, mq, mk, mv, mo, H, L, scale, norm, eps, status, (const float *)s_part, plan.G, plan.cg0,
+                               plan.cg, state_in, state_out) != cudaSuccess)
+            return CHELA_ERR_CUDA;
+        return last_launch_status();
+    }
+    kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, 1, plan.cg0, plan.cg, state_in,
+                                            state_out);
     return last_launch_status();
 }
 
