@@ -209,6 +209,43 @@ def run_mixer_mode(args):
                                            "the long convolution (fp32 FFT on the plain ALUs) is inside the time"}}))
 
 
+def run_backward_mode(args):
+    """--backward: one step = one chela_linattn_bwd call at the timed workload (normaliser on); one JSON line."""
+    import torch
+    from paper_2406_08128_b200 import build as _build, chela
+    _build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device=dev).manual_seed(3)
+    B, L = args.tokens // args.L, args.L
+    q, k, v, d_o = ((torch.randn((B, L, H, D), device=dev, generator=gen) * s).to(torch.bfloat16) for s in (0.125, 0.125, 0.125, 1.0))
+    ws = torch.zeros(int(chela.lib().chela_linattn_bwd_workspace_bytes(B, H, L, D, D)), dtype=torch.uint8, device=dev)
+    step = lambda: chela.linattn_bwd(q, k, v, d_o, workspace=ws)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    if chela.async_status(ws) != chela.OK:
+        raise RuntimeError("device-side wait timed out")
+    ms = e0.elapsed_time(e1) / args.steps
+    peaks, peak_kind = measured_peaks()
+    # minimum traffic of a backward pass: read q, k, v, d_o (bf16), write dq, dk, dv (fp32)
+    alg = B * L * H * D * (4 * 2 + 3 * 4)
+    print(json.dumps({"metric": "linattn_bwd_tokens_per_s", "value": B * L / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "linattn backward B=%d L=%d H=%d d=%d, bf16 in, fp32 gradients, normaliser on" % (B, L, H, D)},
+                      "roofline": {"bound": "hbm", "achieved": alg / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_kind,
+                                   "note": "algorithmic bytes of a one-pass backward (20 B per element) over the time of the "
+                                           "four-launch pass, which itself moves 2.4 times as much"}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -218,10 +255,14 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the sweep / config-2 / mixer / CPU-oracle extras")
     ap.add_argument("--tokens", type=int, default=TOTAL_TOKENS, help="B*L of the timed step (profiling captures use a smaller case)")
     ap.add_argument("--L", type=int, default=L_MAIN, help="sequence length of the timed step")
+    ap.add_argument("--backward", action="store_true", help="time chela_linattn_bwd at the timed workload instead")
     ap.add_argument("--mixer", default=None, metavar="B,L,D,H,chunk",
                     help="time the whole token mixer (short conv, long conv, Q/K/V, attention) on this shape instead, "
                          "e.g. 4,16384,512,8,64 (config 3) or 8,8192,1024,8,128 (config 4); single GPU")
     args = ap.parse_args()
+    if args.backward:
+        run_backward_mode(args)
+        return
     if args.mixer:
         return run_mixer_mode(args)
     if (args.tokens, args.L) != (TOTAL_TOKENS, L_MAIN):
