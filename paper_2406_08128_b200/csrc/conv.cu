@@ -5,13 +5,15 @@
 //   1. conv_transpose_kernel : x[B,L,D] -> a^T[B,D,Ls] fp32, applying the short convolution and
 //      SiLU on the way when short taps are given (Eq. 7); rows become contiguous sequences.
 //   2. twiddle_kernel        : w[j] = exp(-2 pi i j / N), j < M, N = 2M, M = nextpow2(L) (>= 16).
-//   3. fft_conv_kernel (mode 0) : half spectrum K[c][0..M] of each zero-padded long kernel.
-//   4. fft_conv_kernel (mode 1) : per (b,c) row, a real sequence of N = 2M samples (zero padded, so the
+//   3. FFT kernel, mode 0   : half spectrum K[c][0..M] of each zero-padded long kernel.
+//   4. FFT kernel, mode 1   : per (b,c) row, a real sequence of N = 2M samples (zero padded, so the
 //      circular product is the causal linear convolution) is packed into M complex points,
 //      transformed in shared memory (forward decimation-in-frequency, no reordering pass),
 //      multiplied with the kernel spectrum, transformed back (decimation-in-time from
 //      bit-reversed order) and written over its own row.
 //   5. transpose_out_kernel  : z^T[B,D,Ls] -> z[B,L,D] in the output dtype.
+// Steps 3 and 4 run fft_conv_fast_kernel (longconv_fft.cu: compile-time strides) for M = 2^10 .. 2^14 and the
+// generic fft_conv_kernel of this file for every other size.
 #include "common.cuh"
 
 namespace chela {

@@ -17,6 +17,8 @@
 //   warps 2,3: state rows (fp32, never leave the SM) -> bf16 hi + lo -> shared (B operand of the next G2)
 // The state is fed back to the tensor core as S_hi + S_lo (two bf16 terms, ~16 mantissa bits) so the
 // inter-chunk term keeps fp32-like accuracy; P is rounded to bf16 once.
+// Variants by template: operands given as bf16 pairs (kMask), the anti-causal mirror (kReverse) and the backward
+// pass's gradient epilogue (kGrad); sequences of few (batch, head) pairs are split along L (linattn_state_kernel).
 //
 // Every wait is bounded: on a timeout the CTA records CHELA_ERR_TIMEOUT in the status word, drains its
 // outstanding TMA loads (bounded), frees its TMEM and returns.
