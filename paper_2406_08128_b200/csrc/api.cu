@@ -273,10 +273,17 @@ chela_status_t mixer_impl(const void *x, const float *w_short, int short_width, 
     if (tensor_path) {
         __nv_bfloat16 *zp = (__nv_bfloat16 *)z, *qp = (__nv_bfloat16 *)qq, *kp = (__nv_bfloat16 *)kk, *vp = (__nv_bfloat16 *)vv;
         int *status = (int *)ws + 1;   // word 1 of the header: the GEMMs; word 0: the attention kernels
-        st = launch_longconv(x, k_long, w_short, short_width, zp, B, L, D, in_dtype, CHELA_BF16_PAIR, ws + p.off_conv, stream);
+        // Z stays in the FFT kernel's row layout [B][D][L] when the projections can read it as a transposed operand:
+        // saves the transpose back to token-major
+        const int Ls = longconv_row_stride(L);
+        const bool zt = !qk_diag && longconv_transposed_pair_supported(L) && gemm_sm100_at_supported(B, L, Ls, D, D);
+        st = launch_longconv(x, k_long, w_short, short_width, zp, B, L, D, in_dtype, CHELA_BF16_PAIR, ws + p.off_conv, stream, zt);
         if (st != CHELA_OK) return st;
         if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
-        if (qk_diag) {
+        if (zt) {
+            st = launch_gemm_sm100_at(zp, B, L, Ls, w_q, b_q, qp, D, D, 0, status, stream);
+            if (st == CHELA_OK) st = launch_gemm_sm100_at(zp, B, L, Ls, w_k, b_k, kp, D, D, 0, status, stream);
+        } else if (qk_diag) {
             st = launch_affine_pair(zp, w_q, b_q, qp, M, D, in_dtype, stream);
             if (st == CHELA_OK) st = launch_affine_pair(zp, w_k, b_k, kp, M, D, in_dtype, stream);
         } else {
@@ -287,8 +294,13 @@ chela_status_t mixer_impl(const void *x, const float *w_short, int short_width, 
         st = launch_gemm_sm100(x, w_v, b_v, vp, M, D, D, v_silu ? 1 : 0, CHELA_BF16, CHELA_BF16_PAIR, status, stream);
         if (st != CHELA_OK) return st;
         if (gated) {   // G_a = silu(Z W_a + b_a), G_o = sigmoid(Z W_o + b_o), as bf16 pairs
-            st = launch_gemm_sm100(zp, w_a, b_a, ws + p.off_ga, M, D, D, 1, CHELA_BF16_PAIR, CHELA_BF16_PAIR, status, stream);
-            if (st == CHELA_OK) st = launch_gemm_sm100(zp, w_o, b_o, ws + p.off_go, M, D, D, 2, CHELA_BF16_PAIR, CHELA_BF16_PAIR, status, stream);
+            if (zt) {
+                st = launch_gemm_sm100_at(zp, B, L, Ls, w_a, b_a, ws + p.off_ga, D, D, 1, status, stream);
+                if (st == CHELA_OK) st = launch_gemm_sm100_at(zp, B, L, Ls, w_o, b_o, ws + p.off_go, D, D, 2, status, stream);
+            } else {
+                st = launch_gemm_sm100(zp, w_a, b_a, ws + p.off_ga, M, D, D, 1, CHELA_BF16_PAIR, CHELA_BF16_PAIR, status, stream);
+                if (st == CHELA_OK) st = launch_gemm_sm100(zp, w_o, b_o, ws + p.off_go, M, D, D, 2, CHELA_BF16_PAIR, CHELA_BF16_PAIR, status, stream);
+            }
             if (st != CHELA_OK) return st;
         }
         st = launch_linattn_sm100(qp, kp, vp, attn_out, B, H, L, d, chunk, CHELA_BF16_PAIR, attn_dtype, (int)norm, norm_eps, 1.0f,

@@ -94,10 +94,13 @@ chela_status_t launch_shortconv_reparam(const float *w1, int width1, const float
 
 size_t longconv_workspace_bytes(int B, int L, int D);
 bool launch_fft_conv_fast(int mode, float *rows, int row_stride, int L, int D, int nrows, int logM, const float2 *tw,
-                          float2 *spec, int spec_stride, cudaStream_t stream);
+                          float2 *spec, int spec_stride, cudaStream_t stream, __nv_bfloat16 *zt = nullptr,
+                          size_t zt_lo_offset = 0);
+bool longconv_transposed_pair_supported(int L);
+int longconv_row_stride(int L);
 chela_status_t launch_longconv(const void *x, const float *k_long, const float *w_short, int short_width,
                                void *z, int B, int L, int D, chela_dtype_t in_dtype,
-                               chela_dtype_t out_dtype, void *workspace, cudaStream_t stream);
+                               chela_dtype_t out_dtype, void *workspace, cudaStream_t stream, bool transposed_pair = false);
 
 // y[M,N] = act(a[M,K] w[K,N] + bias[N]); a: a_dtype, w: w_dtype, y: y_dtype.
 chela_status_t launch_gemm_simt(const void *a, const void *w, const float *bias, void *y, size_t M, int K,
@@ -105,6 +108,9 @@ chela_status_t launch_gemm_simt(const void *a, const void *w, const float *bias,
                                 chela_dtype_t y_dtype, cudaStream_t stream);
 // tcgen05 GEMM: a bf16 or bf16 pair, w bf16, y bf16 or bf16 pair
 bool gemm_sm100_supported(size_t M, int K, int N, chela_dtype_t a_dtype, chela_dtype_t w_dtype, chela_dtype_t y_dtype);
+bool gemm_sm100_at_supported(int B, int L, int Ls, int K, int N);
+chela_status_t launch_gemm_sm100_at(const void *at, int B, int L, int Ls, const void *w, const float *bias, void *y, int K, int N,
+                                    int act, int *status, cudaStream_t stream);
 chela_status_t launch_gemm_sm100(const void *a, const void *w, const float *bias, void *y, size_t M, int K, int N,
                                  int act, chela_dtype_t a_dtype, chela_dtype_t y_dtype, int *status, cudaStream_t stream);
 // y[m,c] = alpha[c] * z[m,c] + beta[c]

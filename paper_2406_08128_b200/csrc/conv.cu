@@ -661,6 +661,9 @@ LongconvPlan longconv_plan(int B, int L, int D)
 }  // namespace
 
 size_t longconv_workspace_bytes(int B, int L, int D) { return longconv_plan(B, L, D).total; }
+int longconv_row_stride(int L) { return (int)align_up((size_t)L, 8); }
+// the FFT kernels that can write bf16 pair rows cover 2^10 .. 2^14 points
+bool longconv_transposed_pair_supported(int L) { return L > 512 && L <= 16384; }
 
 // rows [B*D][Ls] back to token-major [B, L, D] in the output dtype
 static chela_status_t finish_longconv(const float *at, void *z, int B, int L, int D, int Ls, chela_dtype_t out_dtype,
@@ -678,8 +681,11 @@ static chela_status_t finish_longconv(const float *at, void *z, int B, int L, in
 
 chela_status_t launch_longconv(const void *x, const float *k_long, const float *w_short, int short_width,
                                void *z, int B, int L, int D, chela_dtype_t in_dtype,
-                               chela_dtype_t out_dtype, void *workspace, cudaStream_t stream)
+                               chela_dtype_t out_dtype, void *workspace, cudaStream_t stream, bool transposed_pair)
 {
+    // transposed_pair: z receives the rows as they leave the FFT kernel, [2][B][D][Ls] bf16 (hi plane, lo plane),
+    // and the transpose back to token-major is skipped (the projections read this layout as a transposed operand)
+    if (transposed_pair && !longconv_transposed_pair_supported(L)) return CHELA_ERR_UNSUPPORTED;
     const LongconvPlan p = longconv_plan(B, L, D);
     char *ws = (char *)workspace;
     float *at = (float *)(ws + p.off_at);
@@ -708,9 +714,12 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
     // sizes 2^10 .. 2^14: the kernels with compile-time strides; other sizes: the generic kernel below
     const int spec_stride = p.M + 2;
     if (launch_fft_conv_fast(0, const_cast<float *>(k_long), L, L, D, D, p.logM, tw, spec, spec_stride, stream) &&
-        launch_fft_conv_fast(1, at, p.Ls, L, D, B * D, p.logM, tw, spec, spec_stride, stream)) {
+        launch_fft_conv_fast(1, at, p.Ls, L, D, B * D, p.logM, tw, spec, spec_stride, stream,
+                             transposed_pair ? (__nv_bfloat16 *)z : nullptr, (size_t)B * D * p.Ls)) {
+        if (transposed_pair) return last_launch_status();
         return finish_longconv(at, z, B, L, D, p.Ls, out_dtype, stream);
     }
+    if (transposed_pair) return CHELA_ERR_UNSUPPORTED;
     const size_t smem = (size_t)(p.M + 256) * sizeof(float2);
     int threads = p.M / 16;
     threads = threads < 32 ? 32 : (threads > 1024 ? 1024 : threads);

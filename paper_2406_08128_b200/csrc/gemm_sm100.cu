@@ -44,12 +44,15 @@ struct Smem {
     static_assert(bytes <= 232448, "shared memory per CTA");
 };
 
-template <int BN, bool kAPair, bool kYPair>
+// kATrans: A is given transposed, [B][K][Lt] per plane (the long convolution's row layout: channel-major, tokens
+// contiguous); its tiles are then MN-major like W's, two 64-token atoms per 128-row tile, and row tile m0 lies in
+// batch m0 / Lt at token m0 % Lt (Lt a multiple of 128).
+template <int BN, bool kAPair, bool kYPair, bool kATrans = false>
 __global__ void __launch_bounds__(kThreads)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_constant__ CUtensorMap tm_a_lo,
                   const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y_hi,
                   const __grid_constant__ CUtensorMap tm_y_lo, const float *__restrict__ bias, int M, int N, int K,
-                  int act, int *__restrict__ status)
+                  int act, int *__restrict__ status, int Lt)
 {
     using Smem = Smem<BN, kAPair>;
     constexpr int kStages = Smem::kStages, kStageBytes = Smem::kStageBytes, kStagingWarp = Smem::kStagingWarp;
@@ -105,8 +108,17 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                     if (!ok) break;
                     const uint32_t bar = bar_full0 + 8 * s, dst = sbase + Smem::offStage + s * kStageBytes;
                     mbar_expect_tx(bar, kStageBytes);
-                    tma_load_2d(dst, &tm_a_hi, bar, kb * BK, m0);
-                    if (kAPair) tma_load_2d(dst + kATile, &tm_a_lo, bar, kb * BK, m0);
+                    if (kATrans) {
+                        const int bb = m0 / Lt, t0 = m0 % Lt;
+#pragma unroll
+                        for (int a = 0; a < 2; ++a) {
+                            tma_load_3d(dst + a * (kATile / 2), &tm_a_hi, bar, t0 + 64 * a, kb * BK, bb);
+                            if (kAPair) tma_load_3d(dst + kATile + a * (kATile / 2), &tm_a_lo, bar, t0 + 64 * a, kb * BK, bb);
+                        }
+                    } else {
+                        tma_load_2d(dst, &tm_a_hi, bar, kb * BK, m0);
+                        if (kAPair) tma_load_2d(dst + kATile, &tm_a_lo, bar, kb * BK, m0);
+                    }
 #pragma unroll
                     for (int a = 0; a < BN / 64; ++a) tma_load_2d(dst + kAOff + a * BK * 128, &tm_w, bar, n0 + 64 * a, kb * BK);
                     issued = it + 1;
@@ -122,7 +134,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
     } else if (warp == 5) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BM, BN, 0, 1);
+            constexpr uint32_t idesc = make_idesc(BM, BN, kATrans ? 1 : 0, 1);
             int it = 0, ti = 0;
             bool ok = true;
             for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
@@ -137,11 +149,15 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t st = sbase + Smem::offStage + s * kStageBytes;
-                    const uint32_t a_hi = desc_lo(st), a_lo = desc_lo(st + kATile), w_lo = desc_lo(st + kAOff, BK * 128);
+                    // K-major A: +32 bytes per K step along the row; MN-major A (kATrans): two atoms, +16 rows per K step
+                    const uint32_t a_hi = kATrans ? desc_lo(st, kATile / 2) : desc_lo(st),
+                                   a_lo = kATrans ? desc_lo(st + kATile, kATile / 2) : desc_lo(st + kATile),
+                                   w_lo = desc_lo(st + kAOff, BK * 128);
+                    constexpr uint32_t a_step = kATrans ? 128 : 2;
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
-                        umma_bf16(d, a_hi + 2 * k, w_lo + 128 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                        if (kAPair) umma_bf16(d, a_lo + 2 * k, w_lo + 128 * k, idesc, 1u);
+                        umma_bf16(d, a_hi + a_step * k, w_lo + 128 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        if (kAPair) umma_bf16(d, a_lo + a_step * k, w_lo + 128 * k, idesc, 1u);
                     }
                     umma_commit(bar_empty0 + 8 * s);
                 }
@@ -266,7 +282,7 @@ chela_status_t launch_gemm_sm100(const void *a, const void *w, const float *bias
     const int bn = (N % 256 == 0) ? 256 : 128;
     const long long tiles = (long long)((M + BM - 1) / BM) * (N / bn);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    typedef void (*Kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float *, int, int, int, int, int *);
+    typedef void (*Kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float *, int, int, int, int, int *, int);
     Kern kern;
     int smem;
     if (bn == 256) {
@@ -279,7 +295,39 @@ chela_status_t launch_gemm_sm100(const void *a, const void *w, const float *bias
         smem = a_pair ? Smem<128, true>::bytes : Smem<128, false>::bytes;
     }
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
-    kern<<<grid, kThreads, smem, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status);
+    kern<<<grid, kThreads, smem, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status, 0);
+    return last_launch_status();
+}
+
+bool gemm_sm100_at_supported(int B, int L, int Ls, int K, int N)
+{
+    return B >= 1 && L % BM == 0 && Ls % 8 == 0 && Ls >= L && K % BK == 0 && N % 256 == 0;
+}
+
+// Y [B*L, N] = act(A W + bias) with A given transposed as a bf16 pair: at = [2][B][K][Ls] (hi plane, lo plane),
+// rows of Ls >= L tokens.  Y is written as a bf16 pair.
+chela_status_t launch_gemm_sm100_at(const void *at, int B, int L, int Ls, const void *w, const float *bias, void *y, int K, int N,
+                                    int act, int *status, cudaStream_t stream)
+{
+    const size_t M = (size_t)B * L;
+    const __nv_bfloat16 *a_hi = (const __nv_bfloat16 *)at, *a_lo = a_hi + (size_t)B * K * Ls;
+    __nv_bfloat16 *y_hi = (__nv_bfloat16 *)y, *y_lo = y_hi + M * N;
+    CUtensorMap ma_hi, ma_lo, mw, my_hi, my_lo;
+    const cuuint64_t dims[3] = {(cuuint64_t)L, (cuuint64_t)K, (cuuint64_t)B};
+    const cuuint64_t strides[2] = {(cuuint64_t)Ls * 2, (cuuint64_t)K * Ls * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)BK, 1};
+    if (!make_map_sw128(&ma_hi, a_hi, false, 3, dims, strides, box) || !make_map_sw128(&ma_lo, a_lo, false, 3, dims, strides, box) ||
+        !map_2d(&mw, w, K, N, 64, BK) || !map_2d(&my_hi, y_hi, M, N, 64, 32) || !map_2d(&my_lo, y_lo, M, N, 64, 32))
+        return CHELA_ERR_CUDA;
+    int sms = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+    const long long tiles = (long long)(M / BM) * (N / 256);
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    auto kern = gemm_sm100_kernel<256, true, true, true>;
+    constexpr int smem = Smem<256, true>::bytes;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
+    kern<<<grid, kThreads, smem, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status, L);
     return last_launch_status();
 }
 

@@ -238,7 +238,7 @@ __device__ __forceinline__ void first_pass_fwd(float2 *s, int g, const Tables &t
 // t >= L are written as zeros up to the row stride.
 template <int LOGM, int R0>
 __device__ __forceinline__ void first_pass_inv(const float2 *s, int g, const Tables &tb, float *__restrict__ x, int L, int row_stride,
-                                               float scale)
+                                               float scale, __nv_bfloat16 *__restrict__ zt_hi, __nv_bfloat16 *__restrict__ zt_lo)
 {
     constexpr int M = 1 << LOGM, G0 = 1 << R0, NG = 16 / G0, q0 = M / G0, NT = M / 16;
     constexpr int PQ0 = q0 + q0 / 8, PNT = NT + NT / 8;
@@ -273,7 +273,15 @@ __device__ __forceinline__ void first_pass_inv(const float2 *s, int g, const Tab
             const int t = 2 * (g + u * NT + j * q0);
             if (t < row_stride) {   // row_stride is even
                 const float2 o = v[u * G0 + j];
-                *reinterpret_cast<float2 *>(x + t) = make_float2(t < L ? o.x * scale : 0.f, t + 1 < L ? o.y * scale : 0.f);
+                const float r0 = t < L ? o.x * scale : 0.f, r1 = t + 1 < L ? o.y * scale : 0.f;
+                if (zt_hi) {   // bf16 pair rows (hi plane, lo plane) instead of the fp32 row
+                    const __nv_bfloat162 hh = __floats2bfloat162_rn(r0, r1);
+                    const float2 hf = __bfloat1622float2(hh);
+                    *reinterpret_cast<__nv_bfloat162 *>(zt_hi + t) = hh;
+                    *reinterpret_cast<__nv_bfloat162 *>(zt_lo + t) = __floats2bfloat162_rn(r0 - hf.x, r1 - hf.y);
+                } else {
+                    *reinterpret_cast<float2 *>(x + t) = make_float2(r0, r1);
+                }
             }
         }
 }
@@ -392,7 +400,7 @@ __device__ __forceinline__ void merge_quad(float2 *s, int i, const Tables &tb, f
 template <int LOGM, int MODE, int NTHR>
 __global__ void __launch_bounds__(NTHR) fft_conv_fast_kernel(float *__restrict__ rows, int row_stride, int L, int D,
                                                              const float2 *__restrict__ tw_global, float2 *__restrict__ spec,
-                                                             int spec_stride)
+                                                             int spec_stride, __nv_bfloat16 *__restrict__ zt, size_t zt_lo_offset)
 {
     constexpr int M = 1 << LOGM, NSLOT = M / 16, R0 = ((LOGM - 1) & 3) + 1, LEN1 = M >> R0;
     static_assert(LEN1 == 4096 || LEN1 == 256, "middle passes cover sub-lengths 4096 and 256");
@@ -462,23 +470,26 @@ __global__ void __launch_bounds__(NTHR) fft_conv_fast_kernel(float *__restrict__
     }
     const float scale = 1.0f / (float)M;
 #pragma unroll 1
-    for (int g = threadIdx.x; g < NSLOT; g += NTHR) first_pass_inv<LOGM, R0>(s, g, tb, x, L, row_stride, scale);
+    // zt given: the result leaves as bf16 pair rows [row][row_stride] (the layout the projections read as a transposed
+    // operand) instead of overwriting the fp32 row
+    __nv_bfloat16 *zh = zt ? zt + (size_t)row * row_stride : nullptr;
+    for (int g = threadIdx.x; g < NSLOT; g += NTHR) first_pass_inv<LOGM, R0>(s, g, tb, x, L, row_stride, scale, zh, zh + zt_lo_offset);
 }
 
 template <int LOGM, int NTHR>
 bool launch_fast_t(int mode, float *rows, int row_stride, int L, int D, int nrows, const float2 *tw, float2 *spec, int spec_stride,
-                   cudaStream_t stream)
+                   cudaStream_t stream, __nv_bfloat16 *zt, size_t zt_lo_offset)
 {
     constexpr int M = 1 << LOGM;
     const size_t smem = (size_t)(M + M / 8 + 128 + 128 + M / 16 + 256 + 256) * sizeof(float2);
     if (mode == 0) {
         auto kern = fft_conv_fast_kernel<LOGM, 0, NTHR>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
-        kern<<<nrows, NTHR, smem, stream>>>(rows, row_stride, L, D, tw, spec, spec_stride);
+        kern<<<nrows, NTHR, smem, stream>>>(rows, row_stride, L, D, tw, spec, spec_stride, nullptr, 0);
     } else {
         auto kern = fft_conv_fast_kernel<LOGM, 1, NTHR>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
-        kern<<<nrows, NTHR, smem, stream>>>(rows, row_stride, L, D, tw, spec, spec_stride);
+        kern<<<nrows, NTHR, smem, stream>>>(rows, row_stride, L, D, tw, spec, spec_stride, zt, zt_lo_offset);
     }
     return true;
 }
@@ -486,20 +497,21 @@ bool launch_fast_t(int mode, float *rows, int row_stride, int L, int D, int nrow
 }  // namespace
 
 // True if the size is covered (2^10 <= M <= 2^14) and the kernel was enqueued.  `tw` holds exp(-2 pi i j / 2M),
-// j < M; rows of mode 1 must be 8-byte aligned with an even stride.
+// j < M; rows of mode 1 must be 8-byte aligned with an even stride.  zt (mode 1, optional): write the result as bf16
+// pair rows [nrows][row_stride] at zt and zt + zt_lo_offset instead of over the fp32 rows.
 bool launch_fft_conv_fast(int mode, float *rows, int row_stride, int L, int D, int nrows, int logM, const float2 *tw, float2 *spec,
-                          int spec_stride, cudaStream_t stream)
+                          int spec_stride, cudaStream_t stream, __nv_bfloat16 *zt, size_t zt_lo_offset)
 {
     if (mode == 1 && (row_stride & 1)) return false;
     switch (logM) {
-        case 10: return launch_fast_t<10, 64>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream);
-        case 11: return launch_fast_t<11, 128>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream);
-        case 12: return launch_fast_t<12, 256>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream);
-        case 13: return launch_fast_t<13, 512>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream);
+        case 10: return launch_fast_t<10, 64>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream, zt, zt_lo_offset);
+        case 11: return launch_fast_t<11, 128>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream, zt, zt_lo_offset);
+        case 12: return launch_fast_t<12, 256>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream, zt, zt_lo_offset);
+        case 13: return launch_fast_t<13, 512>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream, zt, zt_lo_offset);
 #ifndef CHELA_FFT14_THREADS
 #define CHELA_FFT14_THREADS 1024
 #endif
-        case 14: return launch_fast_t<14, CHELA_FFT14_THREADS>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream);
+        case 14: return launch_fast_t<14, CHELA_FFT14_THREADS>(mode, rows, row_stride, L, D, nrows, tw, spec, spec_stride, stream, zt, zt_lo_offset);
         default: return false;
     }
 }
