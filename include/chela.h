@@ -59,6 +59,15 @@ int chela_version(void);
 int chela_linattn_kernel_kind(int B, int H, int L, int d_k, int d_v, int chunk,
                               chela_dtype_t in_dtype, chela_dtype_t out_dtype);
 
+/* How the tensor-core kernels split a sequence along L when there are fewer (batch, head) pairs than SMs (host
+ * logic only, no launch; the paper's tiling of Sec. 4.1 has no counterpart: it walks each sequence in one block).
+ * The sequence's 64-token chunks are divided into *groups consecutive groups: the first of *first_chunks chunks, the
+ * others of *other_chunks (the last one what is left); every group but the last is full and none is empty.
+ * sms: SM count to plan for, <= 0 = the current device's.  in_dtype CHELA_BF16_PAIR plans for the full-pair kernel
+ * (one CTA per SM).  Returns 1, or 0 for arguments no tensor-core kernel takes (d not 64 or 128, null pointers). */
+int chela_linattn_split_plan(int B, int H, int L, int d, chela_dtype_t in_dtype, int sms,
+                             int *groups, int *first_chunks, int *other_chunks);
+
 /*
  * Short depthwise causal convolution with optional SiLU (Eq. 7, inner part; Sec. 4.2):
  *   y[b,t,c] = act( bias[c] + sum_{j=0}^{width-1} w[c,j] * x[b,t-j,c] ),   x[b,t<0,c] = 0.

@@ -40,6 +40,7 @@ _SIGNATURES = {
                                    _c_float, _vp, _c_size_t, _vp]),
     "chela_linattn_carry_fwd": (_c_int, [_vp, _vp, _vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                          _c_float, _vp, _c_size_t, _vp]),
+    "chela_linattn_split_plan": (_c_int, [_c_int] * 6 + [_vp, _vp, _vp]),
     "chela_linattn_step": (_c_int, [_vp] * 5 + [_c_int] * 4 + [_c_int, _c_int, _c_int, _c_float, _c_float, _vp]),
     "chela_linattn_bwd_workspace_bytes": (_c_size_t, [_c_int] * 5),
     "chela_linattn_bwd": (_c_int, [_vp] * 7 + [_c_int] * 5 + [_c_int, _c_int, _c_float, _c_float, _vp, _c_size_t, _vp]),
@@ -198,6 +199,13 @@ def linattn_carry_fwd(q, k, v, state_in=None, chunk=64, out_dtype=F32, norm=NORM
                                          d_k, d_v, chunk, in_dtype, _dt(o), int(norm), float(eps), float(scale),
                                          _ptr(workspace), workspace.numel(), _stream()), "chela_linattn_carry_fwd")
     return o, state_out
+
+
+def linattn_split_plan(B, H, L, d=64, in_dtype=BF16, sms=0):
+    """chela_linattn_split_plan: (groups, first_chunks, other_chunks), or None if no tensor-core kernel takes d."""
+    g, c0, c = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0)
+    ok = lib().chela_linattn_split_plan(B, H, L, d, int(in_dtype), int(sms), ctypes.byref(g), ctypes.byref(c0), ctypes.byref(c))
+    return (g.value, c0.value, c.value) if ok else None
 
 
 def linattn_step(q, k, v, state, out_dtype=F32, norm=NORM_RMS, eps=1e-6, scale=1.0, out=None):

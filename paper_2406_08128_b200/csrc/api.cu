@@ -60,6 +60,14 @@ int chela_linattn_kernel_kind(int B, int H, int L, int d_k, int d_v, int chunk, 
     return in_dtype == CHELA_BF16_PAIR ? 0 : 1;
 }
 
+int chela_linattn_split_plan(int B, int H, int L, int d, chela_dtype_t in_dtype, int sms, int *groups, int *first_chunks,
+                             int *other_chunks)
+{
+    if (B < 1 || H < 1 || L < 1 || (d != 64 && d != 128) || !groups || !first_chunks || !other_chunks) return 0;
+    linattn_sm100_split(B, H, L, d, in_dtype == CHELA_BF16_PAIR, sms, groups, first_chunks, other_chunks);
+    return 1;
+}
+
 chela_status_t chela_shortconv_fwd(const void *x, const float *w, const float *bias, void *y, int B, int L,
                                    int D, int width, int act, chela_dtype_t io_dtype, cudaStream_t stream)
 {

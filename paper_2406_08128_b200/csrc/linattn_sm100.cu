@@ -667,12 +667,11 @@ struct SplitPlan {
     int G, cg0, cg;
     size_t part_bytes;
 };
-SplitPlan split_plan(int B, int H, int L, bool pair)   // pair: the kernel's shared memory allows one CTA per SM only
+SplitPlan split_plan(int B, int H, int L, bool pair, int sms = 0)   // pair: shared memory allows one CTA per SM only
 {
-    int sms = 0;
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        sms <= 0)
+    if (sms <= 0 && (cudaGetDevice(&dev) != cudaSuccess ||
+                     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0))
         sms = 148;
     const long long bh = (long long)B * H;
     const int nchunks = (L + kC - 1) / kC;
@@ -795,6 +794,18 @@ chela_status_t launch_linattn_sm100_grad(const void *q, const void *k, const voi
                                          float eps, float scale, void *workspace, cudaStream_t stream)
 {
     return launch_grad(q, k, v, d_o, g, B, H, L, eps, scale, workspace, stream);
+}
+
+void linattn_sm100_split(int B, int H, int L, int d, bool full_pair, int sms, int *G, int *cg0, int *cg)
+{
+    if (d == 128) {
+        linattn_sm100_d128_split(B, H, L, sms, G, cg0, cg);
+        return;
+    }
+    const SplitPlan p = split_plan(B, H, L, full_pair, sms);
+    *G = p.G;
+    *cg0 = p.cg0;
+    *cg = p.cg;
 }
 
 bool linattn_sm100_supported(int B, int H, int L, int d, int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype)

@@ -553,10 +553,11 @@ struct SplitPlan {
     int G, cg0, cg;   // group 0: cg0 chunks, the others cg (two groups: the first a quarter longer, it runs beside the state kernel)
     size_t part_bytes;
 };
-SplitPlan split_plan(int B, int H, int L)
+SplitPlan split_plan(int B, int H, int L, int sms = 0)
 {
-    int sms = 0, dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    int dev = 0;
+    if (sms <= 0 && (cudaGetDevice(&dev) != cudaSuccess ||
+                     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0))
         sms = 148;
     const long long bh = (long long)B * H;
     const int nchunks = (L + kC - 1) / kC;
@@ -632,6 +633,14 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
 }  // namespace
 
 size_t linattn_sm100_d128_workspace_bytes(int B, int H, int L) { return kWsHeader + split_plan(B, H, L).part_bytes; }
+
+void linattn_sm100_d128_split(int B, int H, int L, int sms, int *G, int *cg0, int *cg)
+{
+    const SplitPlan p = split_plan(B, H, L, sms);
+    *G = p.G;
+    *cg0 = p.cg0;
+    *cg = p.cg;
+}
 
 chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                                          chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,

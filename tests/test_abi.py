@@ -92,3 +92,30 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(chela, "LIB_PATH", os.path.join(ROOT, "does_not_exist.so"))
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         chela.lib()
+
+
+def test_split_plan_covers_every_sequence_exactly(lib):
+    """Host logic of the split along L (no GPU: the SM count is passed in).  For every shape: the groups tile the
+    sequence's chunks exactly, none is empty, all but the last are full, no more CTAs than are resident at once,
+    and no split at all once there are as many (batch, head) pairs as SMs."""
+    sms = 148
+    for d, pair in ((64, False), (64, True), (128, False)):
+        dt = chela.BF16_PAIR if pair else chela.BF16
+        for bh in (1, 2, 3, 7, 32, 64, 73, 74, 96, 128, 147, 148, 149, 256):
+            for L in (1, 63, 64, 65, 1000, 1024, 2047, 2048, 2100, 4096, 5000, 8192, 16384, 32768, 65536, 65600, 131072):
+                plan = chela.linattn_split_plan(1, bh, L, d=d, in_dtype=dt, sms=sms)
+                assert plan is not None
+                G, c0, c = plan
+                nch = (L + 63) // 64
+                assert G >= 1 and c0 >= 1 and c >= 1, (d, pair, bh, L, plan)
+                if G == 1:
+                    assert c0 >= nch
+                else:
+                    # groups 0 .. G-2 are full and leave at least one chunk for the last one, which fits in c
+                    assert c0 + (G - 2) * c < nch <= c0 + (G - 1) * c, (d, pair, bh, L, plan)
+                    assert min(c0, c) >= 7, (d, pair, bh, L, plan)          # groups stay long enough to amortise the state pass
+                    per_sm = 1 if (pair or d == 128) else 2
+                    assert bh * G <= per_sm * sms, (d, pair, bh, L, plan)   # every CTA of the call is resident
+                if bh >= sms:
+                    assert G == 1
+    assert chela.linattn_split_plan(1, 1, 100, d=32) is None
