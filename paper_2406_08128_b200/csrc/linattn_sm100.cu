@@ -716,7 +716,11 @@ chela_status_t launch_dependent(Kern kern, int grid, int smem, cudaStream_t stre
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, args...) != cudaSuccess) return CHELA_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, args...) != cudaSuccess) {
+        // without the attribute the launch is an ordinary stream-ordered one and griddepcontrol.wait returns at once
+        (void)cudaGetLastError();
+        kern<<<grid, kThreads, smem, stream>>>(args...);
+    }
     return last_launch_status();
 }
 constexpr size_t kWsHeader = 512;   // word 0: asynchronous status; the rest: diagnostics

@@ -621,8 +621,12 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         if (cudaLaunchKernelEx(&cfg, kern, mq, mk, mv, mo, H, L, scale, norm, eps, status, (const float *)s_part, plan.G, plan.cg0,
-                               plan.cg, state_in, state_out) != cudaSuccess)
-            return CHELA_ERR_CUDA;
+                               plan.cg, state_in, state_out) != cudaSuccess) {
+            // without the attribute: an ordinary stream-ordered launch (griddepcontrol.wait returns at once)
+            (void)cudaGetLastError();
+            kern<<<B * H * plan.G, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, plan.G, plan.cg0,
+                                                             plan.cg, state_in, state_out);
+        }
         return last_launch_status();
     }
     kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, s_part, 1, plan.cg0, plan.cg, state_in,
