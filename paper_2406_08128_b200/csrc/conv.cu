@@ -54,45 +54,48 @@ __global__ void shortconv_kernel(const T *__restrict__ x, const float *__restric
     }
 }
 
-// Fast form for W <= 4 taps: one thread owns 8 consecutive channels (128-bit accesses for bf16) and
-// 16 consecutive tokens, four at a time (four 128-bit loads in flight), with the taps and the previous
-// W-1 inputs in registers: every input is loaded once plus a W-1 token halo per thread.
-template <typename T, int W>
-__global__ void __launch_bounds__(256)
+// Fast form for W <= 4 taps: one thread owns CH consecutive channels (CH = 4: one 8-byte access for bf16) and
+// kTok consecutive tokens, kSub at a time (kSub loads in flight), with the taps and the previous W-1 inputs in
+// registers: every input is loaded once plus a W-1 token halo per thread.  CH = 4 keeps the thread at about 64
+// registers (four CTAs per SM); with 8 channels it needed 121 and the kernel ran at a third of the HBM rate.
+template <typename T, int W, int CH>
+__global__ void __launch_bounds__(256, 4)
 shortconv_fast_kernel(const T *__restrict__ x, const float *__restrict__ w, const float *__restrict__ bias,
                       T *__restrict__ y, int B, int L, int D, int act)
 {
-    constexpr int kTok = 16, kSub = 4;
-    const int nvec = D / 8, nblk = (L + kTok - 1) / kTok;
+    constexpr int kTok = 32, kSub = 4;
+    const int nvec = D / CH, nblk = (L + kTok - 1) / kTok;
     const size_t total = (size_t)B * nblk * nvec;
     for (size_t idx = blockIdx.x * (size_t)blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
         const int cv = (int)(idx % nvec);
         const size_t r = idx / nvec;
         const int tb = (int)(r % nblk), b = (int)(r / nblk);
-        const int c0 = cv * 8, t0 = tb * kTok;
-        float wt[8][W], bs[8];
+        const int c0 = cv * CH, t0 = tb * kTok;
+        float wt[CH][W], bs[CH];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
+        for (int e = 0; e < CH; ++e) {
             bs[e] = bias ? bias[c0 + e] : 0.f;
 #pragma unroll
             for (int j = 0; j < W; ++j) wt[e][j] = w[(c0 + e) * W + j];
         }
         // xin[i] = x[ts - (W-1) + i] for the current sub-block of kSub tokens starting at ts
-        float xin[kSub + W - 1][8];
-        auto load = [&](int t, float (&dst)[8]) {
+        float xin[kSub + W - 1][CH];
+        auto load = [&](int t, float (&dst)[CH]) {
             if (t < 0 || t >= L) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) dst[e] = 0.f;
+                for (int e = 0; e < CH; ++e) dst[e] = 0.f;
                 return;
             }
             const T *px = x + ((size_t)b * L + t) * D + c0;
-            const float4 lo = load4(px), hi = load4(px + 4);
-            dst[0] = lo.x; dst[1] = lo.y; dst[2] = lo.z; dst[3] = lo.w;
-            dst[4] = hi.x; dst[5] = hi.y; dst[6] = hi.z; dst[7] = hi.w;
+#pragma unroll
+            for (int v4 = 0; v4 < CH / 4; ++v4) {
+                const float4 f = load4(px + 4 * v4);
+                dst[4 * v4] = f.x; dst[4 * v4 + 1] = f.y; dst[4 * v4 + 2] = f.z; dst[4 * v4 + 3] = f.w;
+            }
         };
 #pragma unroll
         for (int i = 0; i < W - 1; ++i) load(t0 - (W - 1) + i, xin[i]);
-#pragma unroll
+#pragma unroll 1
         for (int sb = 0; sb < kTok / kSub; ++sb) {
             const int ts = t0 + sb * kSub;
             if (ts >= L) break;
@@ -101,27 +104,27 @@ shortconv_fast_kernel(const T *__restrict__ x, const float *__restrict__ w, cons
 #pragma unroll
             for (int i = 0; i < kSub; ++i) {
                 if (ts + i >= L) break;
-                float acc[8];
+                float acc[CH];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
+                for (int e = 0; e < CH; ++e) {
                     acc[e] = bs[e];
 #pragma unroll
                     for (int j = 0; j < W; ++j) acc[e] = fmaf(wt[e][j], xin[i + W - 1 - j][e], acc[e]);
                     if (act) acc[e] = silu_f(acc[e]);
                 }
                 T *py = y + ((size_t)b * L + ts + i) * D + c0;
-                store4(py, make_float4(acc[0], acc[1], acc[2], acc[3]));
-                store4(py + 4, make_float4(acc[4], acc[5], acc[6], acc[7]));
+#pragma unroll
+                for (int v4 = 0; v4 < CH / 4; ++v4)
+                    store4(py + 4 * v4, make_float4(acc[4 * v4], acc[4 * v4 + 1], acc[4 * v4 + 2], acc[4 * v4 + 3]));
             }
 #pragma unroll
             for (int i = 0; i < W - 1; ++i)
 #pragma unroll
-                for (int e = 0; e < 8; ++e) xin[i][e] = xin[kSub + i][e];
+                for (int e = 0; e < CH; ++e) xin[i][e] = xin[kSub + i][e];
         }
     }
 }
 
-// x[B,L,D] -> at[B,D,Ls] fp32; with taps: at = silu(shortconv(x)).  Tile: 32 channels x 64 tokens.
 template <typename T>
 __global__ void conv_transpose_kernel(const T *__restrict__ x, const float *__restrict__ w, int width,
                                       float *__restrict__ at, int L, int D, int Ls)
@@ -594,15 +597,16 @@ chela_status_t launch_shortconv_t(const void *x, const float *w, const float *bi
 {
     const int threads = 256, max_blocks = 148 * 32;
     if (width <= 4) {
-        const size_t total = (size_t)B * ((L + 15) / 16) * (D / 8);
+        constexpr int CH = 4;
+        const size_t total = (size_t)B * ((L + 31) / 32) * (D / CH);
         const int blocks = (int)((total + threads - 1) / threads < (size_t)max_blocks ? (total + threads - 1) / threads : max_blocks);
         const T *xi = (const T *)x;
         T *yo = (T *)y;
         switch (width) {
-            case 1: shortconv_fast_kernel<T, 1><<<blocks, threads, 0, stream>>>(xi, w, bias, yo, B, L, D, act); break;
-            case 2: shortconv_fast_kernel<T, 2><<<blocks, threads, 0, stream>>>(xi, w, bias, yo, B, L, D, act); break;
-            case 3: shortconv_fast_kernel<T, 3><<<blocks, threads, 0, stream>>>(xi, w, bias, yo, B, L, D, act); break;
-            default: shortconv_fast_kernel<T, 4><<<blocks, threads, 0, stream>>>(xi, w, bias, yo, B, L, D, act); break;
+            case 1: shortconv_fast_kernel<T, 1, CH><<<blocks, threads, 0, stream>>>(xi, w, bias, yo, B, L, D, act); break;
+            case 2: shortconv_fast_kernel<T, 2, CH><<<blocks, threads, 0, stream>>>(xi, w, bias, yo, B, L, D, act); break;
+            case 3: shortconv_fast_kernel<T, 3, CH><<<blocks, threads, 0, stream>>>(xi, w, bias, yo, B, L, D, act); break;
+            default: shortconv_fast_kernel<T, 4, CH><<<blocks, threads, 0, stream>>>(xi, w, bias, yo, B, L, D, act); break;
         }
     } else {
         const size_t nvec = (size_t)B * L * (D / 8);
