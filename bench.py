@@ -441,7 +441,7 @@ def main():
         # ---- every L of the sweep, same kernel and launch path ---------------------------------------
         sweep = []
         for L in SWEEP_L:
-            ms = timed(lambda: step(L), 20)
+            ms = timed(lambda: step(L), 30, warm=5)
             sweep.append({"L": L, "B": TOTAL_TOKENS // L, "ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
                           "hbm_frac": alg_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]})
         line["sweep"] = sweep
@@ -475,7 +475,7 @@ def main():
             w_q, w_k, w_v = [(torch.randn(md, md, device=dev, generator=gen) / md ** 0.5).to(torch.bfloat16) for _ in range(3)]
             mws = torch.zeros(chela.mixer_workspace_bytes(mb, ml, md, mh, mc), dtype=torch.uint8, device=dev)
             mo = torch.empty(mb, ml, md, device=dev)
-            ms = timed(lambda: chela.mixer_fwd(x, w_s, k_l, w_q, w_k, w_v, mh, chunk=mc, out=mo, workspace=mws), 5, warm=2)
+            ms = timed(lambda: chela.mixer_fwd(x, w_s, k_l, w_q, w_k, w_v, mh, chunk=mc, out=mo, workspace=mws), 20, warm=5)
             if chela.async_status(mws) != chela.OK:
                 raise RuntimeError("device-side wait timed out in the mixer")
             d_head = md // mh
@@ -491,7 +491,7 @@ def main():
         (q_, k_, v_), _ = views(L_MAIN)
         d_o = (torch.randn(q_.shape, device=dev, generator=gen)).to(torch.bfloat16)
         bws = torch.zeros(int(chela.lib().chela_linattn_bwd_workspace_bytes(q_.shape[0], H, L_MAIN, D, D)), dtype=torch.uint8, device=dev)
-        ms = timed(lambda: chela.linattn_bwd(q_, k_, v_, d_o, workspace=bws), 3, warm=1)
+        ms = timed(lambda: chela.linattn_bwd(q_, k_, v_, d_o, workspace=bws), 10, warm=3)
         if chela.async_status(bws) != chela.OK:
             raise RuntimeError("device-side wait timed out in the backward pass")
         line["backward"] = {"ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
