@@ -485,7 +485,32 @@ def main():
                            "tensor_frac": flops_tok * mb * ml / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                            "attention_kernel_kind": chela.linattn_kernel_kind(mb, mh, ml, d_head, d_head, mc,
                                                                               chela.BF16_PAIR)})
-            del x, k_l, mws, mo
+            # the prologue stages and one projection of the same shapes on their own (rows a1, a2, a3 of the path)
+            stage = {}
+            y_s = torch.empty_like(x)
+            ms_s = timed(lambda: chela.shortconv_fwd(x, w_s, out=y_s), 20, warm=5)
+            stage["shortconv"] = {"ms": ms_s, "GBps": 2 * x.numel() * 2 / (ms_s * 1e-3) / 1e9,
+                                  "hbm_frac": 2 * x.numel() * 2 / (ms_s * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+            z_l = torch.empty(mb, ml, md, device=dev)
+            cws = torch.zeros(chela.longconv_workspace_bytes(mb, ml, md, chela.BF16, chela.F32), dtype=torch.uint8, device=dev)
+            ms_l = timed(lambda: chela.longconv_fwd(x, k_l, w_s, out=z_l, workspace=cws), 20, warm=5)
+            m_pts = 1 << (ml - 1).bit_length()
+            fft_flops = (mb * md * 2 + md) * 5 * m_pts * (m_pts.bit_length() - 1)   # forward + inverse per row, forward per kernel
+            fp32_peak = 148 * 128 * 2 * 1.965e9 / 1e12
+            stage["longconv"] = {"ms": ms_l, "fft_TFLOPs": fft_flops / (ms_l * 1e-3) / 1e12, "alu_peak_TFLOPs": fp32_peak,
+                                 "alu_frac": fft_flops / (ms_l * 1e-3) / 1e12 / fp32_peak,
+                                 "note": "short conv + SiLU + transposes + FFT long conv, bf16 in, fp32 out; flops = 5 M log2 M "
+                                         "per M-point transform; peak = 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz (FMA counted as 2)"}
+            z_p = torch.randn(2, mb * ml, md, device=dev, generator=gen).to(torch.bfloat16)
+            q_p = torch.empty(2, mb * ml, md, device=dev, dtype=torch.bfloat16)
+            dws = torch.zeros(max(int(chela.lib().chela_dense_workspace_bytes()), 16), dtype=torch.uint8, device=dev)
+            ms_d = timed(lambda: chela.dense_fwd(z_p, w_q, a_dtype=chela.BF16_PAIR, y_dtype=chela.BF16_PAIR, out=q_p, workspace=dws), 20, warm=5)
+            mma_flops = 2 * 2.0 * mb * ml * md * md   # two tensor-core terms per product (pair operand)
+            stage["projection"] = {"ms": ms_d, "TFLOPs": mma_flops / (ms_d * 1e-3) / 1e12,
+                                   "tensor_frac": mma_flops / (ms_d * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                   "note": "one Q or K projection, bf16-pair A (token-major) and Y: both tensor-core terms counted"}
+            mixers[-1]["stages"] = stage
+            del x, k_l, mws, mo, y_s, z_l, cws, z_p, q_p, dws
         line["mixer"] = mixers
         # ---- backward of the timed workload (gradients w.r.t. Q, K, V; normaliser on) ----------------------------
         (q_, k_, v_), _ = views(L_MAIN)
