@@ -157,3 +157,26 @@ def test_bf16_pair_inputs_reach_fp32_like_accuracy(B, L, H, norm, d):
     o = chela.linattn_fwd(qd, kd, vd, chunk=64, norm=chela.NORM_RMS if norm else chela.NORM_NONE, in_dtype=chela.BF16_PAIR)
     ref = oracle.linattn_recurrent(qv, kv, vv, norm=norm)
     assert rel_err(to_numpy(o), ref) <= 5e-4
+
+
+@pytest.mark.parametrize("B,L,H,d", [(2, 8192, 2, 64), (16, 2048, 16, 64), (1, 8192, 2, 128)])
+def test_calls_can_be_captured_in_a_cuda_graph(B, L, H, d):
+    """The library only enqueues work on the caller's stream (memset, kernels, a programmatic dependent launch for
+    split sequences), so a call with caller-owned output and workspace can be captured and replayed; the replay
+    gives the eager call's bits."""
+    import torch
+    q, k, v = (to_device(a, "bf16") for a in inputs.qkv(7, B, L, H, d, d, "bf16"))
+    o_eager = torch.empty(B, L, H, d, device="cuda")
+    o_graph = torch.empty_like(o_eager)
+    ws = torch.zeros(chela.linattn_workspace_bytes(B, H, L, d, d, 64) + 16, dtype=torch.uint8, device="cuda")
+    chela.linattn_fwd(q, k, v, out=o_eager, workspace=ws)
+    torch.cuda.synchronize()
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            chela.linattn_fwd(q, k, v, out=o_graph, workspace=ws)
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert chela.async_status(ws) == chela.OK
+    assert torch.equal(o_eager, o_graph)

@@ -92,3 +92,23 @@ def test_gated_mixer(B, L, D, H, chunk, dtype):
                               dev(m["w_v"]), dev(w_a), dev(w_o), H, chunk=chunk, b_a=dev_f32(b_a), b_o=dev_f32(b_o))
     ref = oracle.mixer_gated(m["x"], m["w_short"], m["k_long"], m["w_q"], m["w_k"], m["w_v"], w_a, w_o, H, b_a=b_a, b_o=b_o)
     assert rel_err(to_numpy(u), ref) <= TOL
+
+
+def test_mixer_call_can_be_captured_in_a_cuda_graph():
+    import torch
+    B, L, D, H = 1, 2048, 512, 8
+    m = inputs.mixer(9, B, L, D)
+    args = (to_device(m["x"], "bf16"), dev_f32(m["w_short"]), dev_f32(m["k_long"]), to_device(m["w_q"], "bf16"),
+            to_device(m["w_k"], "bf16"), to_device(m["w_v"], "bf16"), H)
+    ws = torch.zeros(chela.mixer_workspace_bytes(B, L, D, H, 64), dtype=torch.uint8, device="cuda")
+    o_eager = torch.empty(B, L, D, device="cuda")
+    o_graph = torch.empty_like(o_eager)
+    chela.mixer_fwd(*args, chunk=64, out=o_eager, workspace=ws)
+    torch.cuda.synchronize()
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            chela.mixer_fwd(*args, chunk=64, out=o_graph, workspace=ws)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(o_eager, o_graph)
