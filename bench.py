@@ -521,6 +521,20 @@ def main():
             raise RuntimeError("device-side wait timed out in the backward pass")
         line["backward"] = {"ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
                             "note": "chela_linattn_bwd, bf16 in, fp32 gradients, same workload as the timed step"}
+        # forward + backward at every L of the sweep (the quantity the paper's runtime-vs-length figure plots)
+        fb = []
+        sweep_ms = {e["L"]: e["ms"] for e in sweep}
+        for L in SWEEP_L:
+            (q_, k_, v_), _ = views(L)
+            g_ = d_o.view(q_.shape)
+            need = int(chela.lib().chela_linattn_bwd_workspace_bytes(q_.shape[0], H, L, D, D))
+            if need > bws.numel():
+                bws = torch.zeros(need, dtype=torch.uint8, device=dev)
+            ms_b = timed(lambda: chela.linattn_bwd(q_, k_, v_, g_, workspace=bws), 5, warm=2)
+            if chela.async_status(bws) != chela.OK:
+                raise RuntimeError("device-side wait timed out in the backward sweep")
+            fb.append({"L": L, "fwd_ms": sweep_ms[L], "bwd_ms": ms_b, "fwd_bwd_ms": sweep_ms[L] + ms_b})
+        line["fwd_bwd_sweep"] = fb
         del d_o, bws
         # ---- decode step: one token per sequence against the carried state (bound by the state's bytes) --------
         db, dh = 256, H

@@ -60,7 +60,7 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
                                     int L, int d, int chunk, chela_dtype_t in_dtype,
                                     chela_dtype_t out_dtype, int norm, float eps, float scale,
                                     void *workspace, cudaStream_t stream, const float *state_in = nullptr,
-                                    float *state_out = nullptr, bool reverse = false, int pair_mask = 7);
+                                    float *state_out = nullptr, bool reverse = false, int pair_mask = 7, bool keep_status = false);
 
 size_t linattn_sm100_d128_workspace_bytes(int B, int H, int L);
 void linattn_sm100_d128_split(int B, int H, int L, int sms, int *G, int *cg0, int *cg);
@@ -68,7 +68,7 @@ void linattn_sm100_split(int B, int H, int L, int d, bool full_pair, int sms, in
 chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                                          chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
                                          void *workspace, cudaStream_t stream, const float *state_in = nullptr,
-                                         float *state_out = nullptr, bool reverse = false, int pair_mask = 7);
+                                         float *state_out = nullptr, bool reverse = false, int pair_mask = 7, bool keep_status = false);
 
 // backward of causal linear attention (fp32 SIMT); gradients fp32; workspace = one [B,L,H,d] fp32 buffer
 size_t linattn_bwd_workspace_bytes(int B, int H, int L, int d);

@@ -94,6 +94,9 @@ chela_status_t launch_linattn_bwd_sm100(const void *q, const void *k, const void
     chela_status_t st = CHELA_OK;
     const void *gp = g;
     float gscale = 1.0f;
+    // the launches share one status word: only the first of them clears it, so a timeout in any of them is still
+    // there when the caller looks
+    bool keep = false;
     if (!norm) {
         // G = scale * d_o: the gradient launches take d_o itself and the factor
         gp = d_o;
@@ -103,21 +106,23 @@ chela_status_t launch_linattn_bwd_sm100(const void *q, const void *k, const void
         // which therefore has to be good to fp32 rather than to bf16 scores) and writes G from its epilogue
         st = launch_linattn_sm100_grad(q, k, v, d_o, g, B, H, L, eps, scale, attn_ws, stream);
         if (st != CHELA_OK) return st;
+        keep = true;
     } else {
         // d = 128: r from the pair kernel with every low input plane absent, then G by an elementwise kernel
         st = launch_linattn_sm100(q, k, v, r, B, H, L, d, 64, CHELA_BF16_PAIR, CHELA_F32, 0, eps, scale, attn_ws, stream,
                                   nullptr, nullptr, false, 0);
         if (st != CHELA_OK) return st;
+        keep = true;
         const int blocks = (int)((rows + 7) / 8 < (size_t)148 * 16 ? (rows + 7) / 8 : (size_t)148 * 16);
         bwd_prep_kernel<128><<<blocks, 256, 0, stream>>>(r, (const __nv_bfloat16 *)d_o, g, rows, scale, norm, eps);
         if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
     }
     const chela_dtype_t dt = norm ? CHELA_BF16_PAIR : CHELA_BF16;   // the pair is G, in a different role each time
-    st = launch_linattn_sm100(gp, v, k, dq, B, H, L, d, 64, dt, CHELA_F32, 0, eps, gscale, attn_ws, stream, nullptr, nullptr, false, 1);
+    st = launch_linattn_sm100(gp, v, k, dq, B, H, L, d, 64, dt, CHELA_F32, 0, eps, gscale, attn_ws, stream, nullptr, nullptr, false, 1, keep);
     if (st != CHELA_OK) return st;
-    st = launch_linattn_sm100(v, gp, q, dk, B, H, L, d, 64, dt, CHELA_F32, 0, eps, gscale, attn_ws, stream, nullptr, nullptr, true, 2);
+    st = launch_linattn_sm100(v, gp, q, dk, B, H, L, d, 64, dt, CHELA_F32, 0, eps, gscale, attn_ws, stream, nullptr, nullptr, true, 2, true);
     if (st != CHELA_OK) return st;
-    return launch_linattn_sm100(k, q, gp, dv, B, H, L, d, 64, dt, CHELA_F32, 0, eps, gscale, attn_ws, stream, nullptr, nullptr, true, 4);
+    return launch_linattn_sm100(k, q, gp, dv, B, H, L, d, 64, dt, CHELA_F32, 0, eps, gscale, attn_ws, stream, nullptr, nullptr, true, 4, true);
 }
 
 }  // namespace chela

@@ -66,6 +66,10 @@ struct Smem {
     static constexpr int bytes = offAbort + 8;
 };
 constexpr int kTmemCols = 128;
+// Diagnostics for a wait that gave up: words 8..11 of the workspace header keep, for the first such wait since the
+// header was last zeroed by the caller, a site code (100 * kMask + site; 9000 + ... in the state kernel), the CTA,
+// the chunk and the grid size.  The library never clears them.
+#define DIAG(site, extra) do { if (atomicCAS(status + 8, 0, (site)) == 0) { status[9] = blockIdx.x; status[10] = (extra); status[11] = gridDim.x; } } while (0)
 constexpr int kColOS = 0;    // rows 0..63: output tile, rows 64..127: running state; 64 columns
 constexpr int kColPT = 64;   // rows 64..127: transposed scores; 64 columns
 
@@ -176,7 +180,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
             // G1 of a chunk; false if the chunk's tiles never arrived
             auto issue_scores = [&](int chunk) -> bool {
-                if (!mbar_wait(bar_full0 + 8 * (chunk % kStages), (chunk / kStages) & 1, abort_flag)) return false;
+                if (!mbar_wait(bar_full0 + 8 * (chunk % kStages), (chunk / kStages) & 1, abort_flag)) { DIAG(1 + 100 * kMask, chunk); return false; }
                 tc_fence_after();
                 const uint32_t qk_lo = desc_lo(stage_base(chunk));
 #pragma unroll
@@ -205,6 +209,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     // G2: rows 0..63 of OS = Q S_hi + Q S_lo; needs the state tiles of the previous chunk (or
                     // of the group's initial state) and the previous output rows out of TMEM
                     ok = mbar_wait(bar_s, par_s, abort_flag);
+                    if (!ok) DIAG(2 + 100 * kMask, i);
                     par_s ^= 1;
                     if (!ok) break;
                     tc_fence_after();
@@ -223,6 +228,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 }
                 // G3: OS += [P^T | K]^T V; atom 0 = score tile, atom 1 = K tile of this stage
                 ok = mbar_wait(bar_pt, i & 1, abort_flag);
+                if (!ok) DIAG(3 + 100 * kMask, i);
                 if (!ok) break;
                 tc_fence_after();
                 TMARK(2);
@@ -251,9 +257,11 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 TMARK(3);
                 // the stage is free once G3 has completed: prefetch the chunk that will use it next
                 ok = mbar_wait(bar_o, i & 1, abort_flag);
+                if (!ok) DIAG(4 + 100 * kMask, i);
                 if (!ok) break;
                 if (kGrad) {   // the stage also holds the d_o tile: wait until the epilogue warps have copied their rows
                     ok = mbar_wait(bar_dr, i & 1, abort_flag);
+                    if (!ok) DIAG(5 + 100 * kMask, i);
                     if (!ok) break;
                 }
                 consumed = i + 1;
@@ -340,6 +348,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             if (upper) {
                 // ---- P^T_i: TMEM -> causal mask -> bf16 -> shared (rows = s, 64 t per row) -------------
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_p, i & 1, abort_flag));
+                if (!ok && lane == 0) DIAG(6 + 100 * kMask, i);
                 if (!ok) break;
                 tc_fence_after();
                 TMARK(0);
@@ -382,15 +391,23 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             uint4 dq4[kGrad ? 8 : 1];   // kGrad: row t of d_o (64 bf16), copied out of the stage before the stage can be reloaded
             if (kGrad && !upper) {
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_full0 + 8 * (i % kStages), (i / kStages) & 1, abort_flag));
+                if (!ok && lane == 0) DIAG(7 + 100 * kMask, i);
                 if (!ok) break;
                 const uint8_t *sD = smem + SM::offStage + ((i % kStages) * kTPS + SM::iD) * kTile;
 #pragma unroll
                 for (int c8 = 0; c8 < 8; ++c8) dq4[c8] = *reinterpret_cast<const uint4 *>(sD + sw128(r, c8));
+            }
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag));
+            if (!ok && lane == 0) DIAG(8 + 100 * kMask + 10 * warp, i);
+            if (!ok) break;
+            // The d_o rows are in registers: the issuer may reload the stage.  Arriving only now, after bar_o of this
+            // chunk, keeps the arrivals in step with the issuer's waits: arrived earlier (right after the copy), the two
+            // warps could complete the phase of chunk i + 1 before the issuer had looked at the phase of chunk i, whose
+            // parity wait then never returns.
+            if (kGrad && !upper) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_dr);
             }
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag));
-            if (!ok) break;
             tc_fence_after();
             TMARK(2);
             float acc[kD];
@@ -588,6 +605,7 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             for (int i = 0; i < nchunks; ++i) {
                 const int stage = i % kStStages;
                 ok = mbar_wait(bar_full0 + 8 * stage, (i / kStStages) & 1, abort_flag);
+                if (!ok) DIAG(9001 + 100 * kMask, i);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t st = sbase + SM::offStage + stage * kTPS * kTile;
@@ -608,6 +626,7 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 consumed = i + 1;
                 if (i + kStStages < nchunks) {
                     ok = mbar_wait(bar_empty0 + 8 * stage, (i / kStStages) & 1, abort_flag);
+                    if (!ok) DIAG(9002 + 100 * kMask, i);
                     if (!ok) break;
                     issue_load(i + kStStages);
                     ++loads_issued;
@@ -728,7 +747,7 @@ constexpr size_t kWsHeader = 512;   // word 0: asynchronous status; the rest: di
 template <typename TOut, int kMask, bool kReverse>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
                         float scale, void *workspace, const float *state_in, float *state_out, cudaStream_t stream,
-                        int planes_mask)
+                        int planes_mask, bool keep_status = false)
 {
     // planes_mask: which of q, k, v are given with two planes.  An operand that the kernel treats as a pair but
     // that has one plane gets a one-plane map: its "low plane" is then out of bounds for the copy engine and
@@ -741,7 +760,8 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
     const SplitPlan plan = split_plan(B, H, L, Smem<TOut, kMask>::bytes > 113 * 1024);
     int *status = (int *)workspace;
     float *s_part = (float *)((char *)workspace + kWsHeader);
-    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+    // keep_status: a later launch of a multi-launch call must not erase what an earlier one reported
+    if (!keep_status && cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
     if (plan.G > 1) {
         auto skern = linattn_state_kernel<(kMask & 6), kReverse>;
         constexpr int ssmem = SmemState<(kMask & 6)>::bytes;
@@ -832,35 +852,35 @@ size_t linattn_sm100_workspace_bytes(int B, int H, int L, int d, int)
 chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int d,
                                     int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps,
                                     float scale, void *workspace, cudaStream_t stream, const float *state_in,
-                                    float *state_out, bool reverse, int pair_mask)
+                                    float *state_out, bool reverse, int pair_mask, bool keep_status)
 {
     if (d == 128)
         return launch_linattn_sm100_d128(q, k, v, o, B, H, L, in_dtype, out_dtype, norm, eps, scale, workspace, stream, state_in,
-                                         state_out, reverse, pair_mask);
+                                         state_out, reverse, pair_mask, keep_status);
     // The result does not depend on the chunk size: both supported values run on 64-token tiles.
     (void)chunk;
     const bool pair = in_dtype == CHELA_BF16_PAIR;
     const int pm = pair ? (pair_mask & 7) : 0;
     if (reverse) {   // anti-causal mirror: fp32 output, no state carry (the backward pass)
         if (out_dtype != CHELA_F32 || state_in || state_out) return CHELA_ERR_UNSUPPORTED;
-        if (!pair) return launch_t<float, 0, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, 0);
-        if (pm == 2) return launch_t<float, 10, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm);
-        if (pm == 4) return launch_t<float, 12, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm);
+        if (!pair) return launch_t<float, 0, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, 0, keep_status);
+        if (pm == 2) return launch_t<float, 10, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm, keep_status);
+        if (pm == 4) return launch_t<float, 12, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm, keep_status);
         return CHELA_ERR_UNSUPPORTED;
     }
     if (pair) {
         // One gradient operand of the backward pass is a pair (or none: scores and state kept as pairs only):
         // kernels without the absent low planes; fp32 output, no state carry.
         if (pm != 7 && out_dtype == CHELA_F32 && !state_in && !state_out) {
-            if (pm == 0) return launch_t<float, 8, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm);
-            if (pm == 1) return launch_t<float, 9, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm);
+            if (pm == 0) return launch_t<float, 8, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm, keep_status);
+            if (pm == 1) return launch_t<float, 9, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pm, keep_status);
         }
         if (out_dtype == CHELA_F32)
-            return launch_t<float, 15, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pm);
-        return launch_t<__nv_bfloat16, 15, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pm);
+            return launch_t<float, 15, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pm, keep_status);
+        return launch_t<__nv_bfloat16, 15, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pm, keep_status);
     }
-    if (out_dtype == CHELA_F32) return launch_t<float, 0, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 0);
-    return launch_t<__nv_bfloat16, 0, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 0);
+    if (out_dtype == CHELA_F32) return launch_t<float, 0, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 0, keep_status);
+    return launch_t<__nv_bfloat16, 0, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 0, keep_status);
 }
 
 }  // namespace chela

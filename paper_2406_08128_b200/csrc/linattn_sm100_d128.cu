@@ -586,7 +586,7 @@ constexpr size_t kWsHeader = 512;
 template <typename TOut, bool kPair, bool kReverse>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int norm, float eps,
                         float scale, void *workspace, const float *state_in, float *state_out, cudaStream_t stream,
-                        int pair_mask = 7)
+                        int pair_mask = 7, bool keep_status = false)
 {
     // pair_mask: which of q, k, v really are pairs; a single bf16 operand of a pair kernel gets a one-plane map
     // and its low plane arrives as zeros (out of bounds for the copy engine)
@@ -598,7 +598,7 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
     int *status = (int *)workspace;
     float *s_part = (float *)((char *)workspace + kWsHeader);
     const SplitPlan plan = split_plan(B, H, L);
-    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+    if (!keep_status && cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
     if (plan.G > 1) {
         auto skern = linattn_state_d128_kernel<kPair, kReverse>;
         if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemState<kPair>::bytes) != cudaSuccess)
@@ -649,21 +649,21 @@ void linattn_sm100_d128_split(int B, int H, int L, int sms, int *G, int *cg0, in
 chela_status_t launch_linattn_sm100_d128(const void *q, const void *k, const void *v, void *o, int B, int H, int L,
                                          chela_dtype_t in_dtype, chela_dtype_t out_dtype, int norm, float eps, float scale,
                                          void *workspace, cudaStream_t stream, const float *state_in, float *state_out, bool reverse,
-                                         int pair_mask)
+                                         int pair_mask, bool keep_status)
 {
     if (reverse) {
         if (out_dtype != CHELA_F32 || state_in || state_out) return CHELA_ERR_UNSUPPORTED;
         if (in_dtype == CHELA_BF16_PAIR)
-            return launch_t<float, true, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pair_mask);
-        return launch_t<float, false, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream);
+            return launch_t<float, true, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, pair_mask, keep_status);
+        return launch_t<float, false, true>(q, k, v, o, B, H, L, norm, eps, scale, workspace, nullptr, nullptr, stream, 7, keep_status);
     }
     if (in_dtype == CHELA_BF16_PAIR) {
         if (out_dtype == CHELA_F32)
-            return launch_t<float, true, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pair_mask);
-        return launch_t<__nv_bfloat16, true, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+            return launch_t<float, true, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pair_mask, keep_status);
+        return launch_t<__nv_bfloat16, true, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 7, keep_status);
     }
-    if (out_dtype == CHELA_F32) return launch_t<float, false, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
-    return launch_t<__nv_bfloat16, false, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream);
+    if (out_dtype == CHELA_F32) return launch_t<float, false, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 7, keep_status);
+    return launch_t<__nv_bfloat16, false, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 7, keep_status);
 }
 
 }  // namespace chela

@@ -83,3 +83,28 @@ def test_backward_at_the_benchmark_size_by_directional_derivatives():
                 ana = float((grow * drow).sum())
                 num = central_difference(x, go, dirs, 1e-3)
                 assert abs(num - ana) <= 1e-2 * np.linalg.norm(grow) * np.linalg.norm(drow), (b, h, which, t, num, ana)
+
+
+@pytest.mark.parametrize("B,L,H", [(1, 16384, 8), (4, 32768, 16)])
+def test_back_to_back_backward_calls_on_split_sequences(B, L, H):
+    """Calls queued without a host synchronisation in between (split sequences: every launch is a state kernel
+    plus a main kernel that starts beside it).  No wait may give up (a give-up costs about a second and sets the
+    status word, which the later launches of a call must not erase), and every call returns the first call's bits."""
+    import time
+    import torch
+    d = 64
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    q, k, v = ((torch.randn((B, L, H, d), device="cuda", generator=gen) * 0.125).to(torch.bfloat16) for _ in range(3))
+    d_o = torch.randn((B, L, H, d), device="cuda", generator=gen).to(torch.bfloat16)
+    ws = torch.zeros(int(chela.lib().chela_linattn_bwd_workspace_bytes(B, H, L, d, d)), dtype=torch.uint8, device="cuda")
+    first = [g.clone() for g in chela.linattn_bwd(q, k, v, d_o, workspace=ws)]
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(8):
+        grads = chela.linattn_bwd(q, k, v, d_o, workspace=ws)
+    torch.cuda.synchronize()
+    elapsed = time.perf_counter() - t0
+    assert chela.async_status(ws) == chela.OK
+    assert elapsed < 0.5, elapsed
+    for a, b in zip(first, grads):
+        assert torch.equal(a, b)
