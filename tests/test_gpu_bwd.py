@@ -85,14 +85,13 @@ def test_backward_at_the_benchmark_size_by_directional_derivatives():
                 assert abs(num - ana) <= 1e-2 * np.linalg.norm(grow) * np.linalg.norm(drow), (b, h, which, t, num, ana)
 
 
-@pytest.mark.parametrize("B,L,H", [(1, 16384, 8), (4, 32768, 16)])
-def test_back_to_back_backward_calls_on_split_sequences(B, L, H):
+@pytest.mark.parametrize("B,L,H,d", [(1, 16384, 8, 64), (4, 32768, 16, 64), (1, 16384, 4, 128), (16, 4096, 16, 64)])
+def test_back_to_back_backward_calls_on_split_sequences(B, L, H, d):
     """Calls queued without a host synchronisation in between (split sequences: every launch is a state kernel
     plus a main kernel that starts beside it).  No wait may give up (a give-up costs about a second and sets the
     status word, which the later launches of a call must not erase), and every call returns the first call's bits."""
     import time
     import torch
-    d = 64
     gen = torch.Generator(device="cuda").manual_seed(5)
     q, k, v = ((torch.randn((B, L, H, d), device="cuda", generator=gen) * 0.125).to(torch.bfloat16) for _ in range(3))
     d_o = torch.randn((B, L, H, d), device="cuda", generator=gen).to(torch.bfloat16)
