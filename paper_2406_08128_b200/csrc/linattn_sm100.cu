@@ -61,7 +61,7 @@ struct Smem {
     // output staging; also what a 128-row operand that starts in the last tile of the last stage reads past it
     static constexpr int offO = offStage + kStages * kTilesPerStage * kTile;
     static constexpr int offBar = offO + (kOBoxes > 1 ? kOBoxes : 1) * kTile;   // full[kStages], p, o, pt, s, dr
-    static constexpr int offTmem = offBar + 8 * (kStages + 5);
+    static constexpr int offTmem = offBar + 8 * (kStages + 6);
     static constexpr int offAbort = offTmem + 8;
     static constexpr int bytes = offAbort + 8;
 };
@@ -129,7 +129,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const uint32_t bar_o = bar_p + 8;                 // G2 + G3 of a chunk have completed (-> all roles)
     const uint32_t bar_pt = bar_o + 8;                // score tile of a chunk is in shared memory (warps 2,3 -> issuer)
     const uint32_t bar_s = bar_pt + 8;                // output/state rows read, state tiles written (4 warps -> issuer)
-    const uint32_t bar_dr = bar_s + 8;                // kGrad: both epilogue warps hold their d_o rows of a chunk (-> issuer)
+    const uint32_t bar_dr0 = bar_s + 8;               // kGrad: both epilogue warps hold their d_o rows of an even / odd chunk (-> issuer)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
 
@@ -140,7 +140,8 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         mbar_init(bar_pt, 2);
         mbar_init(bar_s, 4);
         if (kGrad) {
-            mbar_init(bar_dr, 2);
+            mbar_init(bar_dr0, 2);
+            mbar_init(bar_dr0 + 8, 2);
             tma_prefetch_desc(&tm_d);
         }
         *abort_flag = 0;
@@ -260,7 +261,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (!ok) DIAG(4 + 100 * kMask, i);
                 if (!ok) break;
                 if (kGrad) {   // the stage also holds the d_o tile: wait until the epilogue warps have copied their rows
-                    ok = mbar_wait(bar_dr, i & 1, abort_flag);
+                    ok = mbar_wait(bar_dr0 + 8 * (i & 1), (i >> 1) & 1, abort_flag);
                     if (!ok) DIAG(5 + 100 * kMask, i);
                     if (!ok) break;
                 }
@@ -396,18 +397,16 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const uint8_t *sD = smem + SM::offStage + ((i % kStages) * kTPS + SM::iD) * kTile;
 #pragma unroll
                 for (int c8 = 0; c8 < 8; ++c8) dq4[c8] = *reinterpret_cast<const uint4 *>(sD + sw128(r, c8));
+                // The rows are in registers: the issuer may reload the stage once both warps have said so.  Even and odd
+                // chunks use different barriers: with one, the two warps could complete the phase of chunk i + 1 before
+                // the issuer had looked at the phase of chunk i, and its parity wait would never return.  The arrival
+                // for chunk i + 2 needs bar_o of chunk i + 1, which the issuer commits after its wait for chunk i.
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_dr0 + 8 * (i & 1));
             }
             ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag));
             if (!ok && lane == 0) DIAG(8 + 100 * kMask + 10 * warp, i);
             if (!ok) break;
-            // The d_o rows are in registers: the issuer may reload the stage.  Arriving only now, after bar_o of this
-            // chunk, keeps the arrivals in step with the issuer's waits: arrived earlier (right after the copy), the two
-            // warps could complete the phase of chunk i + 1 before the issuer had looked at the phase of chunk i, whose
-            // parity wait then never returns.
-            if (kGrad && !upper) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_dr);
-            }
             tc_fence_after();
             TMARK(2);
             float acc[kD];
