@@ -180,3 +180,24 @@ def test_calls_can_be_captured_in_a_cuda_graph(B, L, H, d):
     torch.cuda.synchronize()
     assert chela.async_status(ws) == chela.OK
     assert torch.equal(o_eager, o_graph)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("d", [64, 128])
+def test_degenerate_inputs_zero_rows_and_all_ones(dtype, d):
+    """Zero queries give exactly zero rows through the normaliser (no NaN from 0 * rsqrt(eps)); all-ones inputs give
+    the closed form r_t = (t + 1) d, whose normalised rows are all ones (a row of equal entries has RMS = |entry|)."""
+    import torch
+    B, L, H = 2, 300, 2
+    dt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    ones = torch.ones(B, L, H, d, device="cuda", dtype=dt)
+    zeros = torch.zeros_like(ones)
+    o = chela.linattn_fwd(zeros, ones, ones)
+    assert bool((o == 0).all())
+    o = chela.linattn_fwd(ones, ones, zeros)
+    assert bool((o == 0).all())
+    r = chela.linattn_fwd(ones, ones, ones, norm=chela.NORM_NONE)
+    t = torch.arange(1, L + 1, device="cuda", dtype=torch.float32)[None, :, None, None] * d
+    assert bool((r == t.expand_as(r)).all())      # exact: small integers in fp32 accumulation
+    o = chela.linattn_fwd(ones, ones, ones)
+    assert float((o - 1).abs().max()) <= 1e-6
