@@ -44,13 +44,12 @@ constexpr int kTile = kC * 128;   // one 64-row x 128-byte tile
 __host__ __device__ constexpr int popc3(int m) { return (m & 1) + ((m >> 1) & 1) + ((m >> 2) & 1); }
 // kGrad (backward pass, with kMask = 8): the epilogue does not store the output row but pulls the output gradient
 // d_o back through the normaliser, G = scale (d_o - o <o, d_o> / d) / n, and stores G as a bf16 pair; the d_o tiles
-// are one more tile of every stage.
+// come through a two-slot ring of their own.
 template <typename TOut, int kMask, bool kGrad = false>
 struct Smem {
     static constexpr int kIn = kMask & 7;
     static constexpr bool kPPair = (kMask & 8) != 0;
-    static constexpr int kTilesPerStage = 3 + popc3(kIn) + (kGrad ? 1 : 0);   // Q, K, V (hi), the low planes that exist, d_o (kGrad)
-    static constexpr int iD = 3 + popc3(kIn);
+    static constexpr int kTilesPerStage = 3 + popc3(kIn);   // Q, K, V (hi), then the low planes that exist, in that order
     static constexpr int iQlo = 3, iKlo = 3 + (kIn & 1), iVlo = 3 + popc3(kIn & 3);
     static constexpr int kStages = (kMask == 0) ? 3 : 2;
     static constexpr int kOBoxes = kGrad ? 2 : (int)sizeof(TOut) * kD / 128;   // output staged as 128-byte wide boxes (kGrad: hi, lo)
@@ -60,7 +59,8 @@ struct Smem {
     static constexpr int offStage = offSlo + kTile;       // after the score tile: the G3 descriptor reaches K from P forwards
     // output staging; also what a 128-row operand that starts in the last tile of the last stage reads past it
     static constexpr int offO = offStage + kStages * kTilesPerStage * kTile;
-    static constexpr int offBar = offO + (kOBoxes > 1 ? kOBoxes : 1) * kTile;   // full[kStages], p, o, pt, s, dr
+    static constexpr int offD = offO + (kOBoxes > 1 ? kOBoxes : 1) * kTile;      // d_o tiles, two slots (kGrad)
+    static constexpr int offBar = offD + (kGrad ? 2 : 0) * kTile;   // full[kStages], p, o, pt, s, dfull[2]
     static constexpr int offTmem = offBar + 8 * (kStages + 6);
     static constexpr int offAbort = offTmem + 8;
     static constexpr int bytes = offAbort + 8;
@@ -129,7 +129,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const uint32_t bar_o = bar_p + 8;                 // G2 + G3 of a chunk have completed (-> all roles)
     const uint32_t bar_pt = bar_o + 8;                // score tile of a chunk is in shared memory (warps 2,3 -> issuer)
     const uint32_t bar_s = bar_pt + 8;                // output/state rows read, state tiles written (4 warps -> issuer)
-    const uint32_t bar_dr0 = bar_s + 8;               // kGrad: both epilogue warps hold their d_o rows of an even / odd chunk (-> issuer)
+    const uint32_t bar_d0 = bar_s + 8;                // kGrad: the d_o tile of slot 0 / 1 has landed (copy engine -> epilogue warps)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
 
@@ -140,8 +140,8 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         mbar_init(bar_pt, 2);
         mbar_init(bar_s, 4);
         if (kGrad) {
-            mbar_init(bar_dr0, 2);
-            mbar_init(bar_dr0 + 8, 2);
+            mbar_init(bar_d0, 1);
+            mbar_init(bar_d0 + 8, 1);
             tma_prefetch_desc(&tm_d);
         }
         *abort_flag = 0;
@@ -174,7 +174,6 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (kIn & 1) tma_load_5d(dst + SM::iQlo * kTile, &tm_q, bar, 0, h, tok(chunk), b, 1);
                 if (kIn & 2) tma_load_5d(dst + SM::iKlo * kTile, &tm_k, bar, 0, h, tok(chunk), b, 1);
                 if (kIn & 4) tma_load_5d(dst + SM::iVlo * kTile, &tm_v, bar, 0, h, tok(chunk), b, 1);
-                if (kGrad) tma_load_5d(dst + SM::iD * kTile, &tm_d, bar, 0, h, tok(chunk), b, 0);
             };
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [Q;K] (K-major) x Q^T (K-major)
             constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;K] (K-major) x S (MN-major)
@@ -200,8 +199,18 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 return true;
             };
             const uint32_t shi_lo = desc_lo(sbase + SM::offShi), slo_lo = desc_lo(sbase + SM::offSlo);
-            int loads_issued = 0, consumed = 0;
+            int loads_issued = 0, consumed = 0, d_issued = 0;
+            // kGrad: d_o tile of a chunk into slot chunk % 2.  Slot and barrier are reused two chunks later, after the
+            // epilogue warps have copied their rows: they say so with their arrival on bar_s, which the issuer has
+            // waited for before it issues the reload, so the barrier never runs a phase ahead of its waiters.
+            auto issue_d = [&](int chunk) {
+                const uint32_t bar = bar_d0 + 8 * (chunk & 1);
+                mbar_expect_tx(bar, kTile);
+                tma_load_5d(sbase + SM::offD + (chunk & 1) * kTile, &tm_d, bar, 0, h, tok(chunk), b, 0);
+            };
             for (; loads_issued < kStages && loads_issued < nchunks; ++loads_issued) issue_load(loads_issued);
+            if (kGrad)
+                for (; d_issued < 2 && d_issued < nchunks; ++d_issued) issue_d(d_issued);
             bool ok = issue_scores(0);
             uint32_t par_s = 0;
             for (int i = 0; ok && i < nchunks; ++i) {
@@ -215,6 +224,10 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     if (!ok) break;
                     tc_fence_after();
                     TMARK(0);
+                    if (kGrad && i >= 1 && i + 1 < nchunks) {   // the epilogue warps hold d_o of chunk i - 1: its slot takes chunk i + 1
+                        issue_d(i + 1);
+                        ++d_issued;
+                    }
                     const uint32_t qk_lo = desc_lo(st);
 #pragma unroll
                     for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk_lo + 2 * k, shi_lo + 128 * k, idescG2, k > 0, 1);
@@ -260,11 +273,6 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 ok = mbar_wait(bar_o, i & 1, abort_flag);
                 if (!ok) DIAG(4 + 100 * kMask, i);
                 if (!ok) break;
-                if (kGrad) {   // the stage also holds the d_o tile: wait until the epilogue warps have copied their rows
-                    ok = mbar_wait(bar_dr0 + 8 * (i & 1), (i >> 1) & 1, abort_flag);
-                    if (!ok) DIAG(5 + 100 * kMask, i);
-                    if (!ok) break;
-                }
                 consumed = i + 1;
                 if (i + kStages < nchunks) {
                     issue_load(i + kStages);
@@ -278,6 +286,8 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 // drain loads that were issued but never consumed (bounded), so no copy lands after exit
                 for (int c = consumed; c < loads_issued; ++c)
                     mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1, nullptr);
+                if (kGrad)
+                    for (int c = d_issued > 2 ? d_issued - 2 : 0; c < d_issued; ++c) mbar_wait(bar_d0 + 8 * (c & 1), (c >> 1) & 1, nullptr);
             }
 #ifdef CHELA_TIMING
             if (blockIdx.x == 0) TDUMP(0);
@@ -389,21 +399,6 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (lane == 0) mbar_arrive(bar_pt);
                 TMARK(1);
             }
-            uint4 dq4[kGrad ? 8 : 1];   // kGrad: row t of d_o (64 bf16), copied out of the stage before the stage can be reloaded
-            if (kGrad && !upper) {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_full0 + 8 * (i % kStages), (i / kStages) & 1, abort_flag));
-                if (!ok && lane == 0) DIAG(7 + 100 * kMask, i);
-                if (!ok) break;
-                const uint8_t *sD = smem + SM::offStage + ((i % kStages) * kTPS + SM::iD) * kTile;
-#pragma unroll
-                for (int c8 = 0; c8 < 8; ++c8) dq4[c8] = *reinterpret_cast<const uint4 *>(sD + sw128(r, c8));
-                // The rows are in registers: the issuer may reload the stage once both warps have said so.  Even and odd
-                // chunks use different barriers: with one, the two warps could complete the phase of chunk i + 1 before
-                // the issuer had looked at the phase of chunk i, and its parity wait would never return.  The arrival
-                // for chunk i + 2 needs bar_o of chunk i + 1, which the issuer commits after its wait for chunk i.
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_dr0 + 8 * (i & 1));
-            }
             ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag));
             if (!ok && lane == 0) DIAG(8 + 100 * kMask + 10 * warp, i);
             if (!ok) break;
@@ -415,6 +410,15 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 tmem_ld32(tmem_warp + kColOS, *reinterpret_cast<float(*)[32]>(&acc[0]));
                 tmem_ld32(tmem_warp + kColOS + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
                 tmem_ld_wait();
+                uint4 dq4[kGrad ? 8 : 1];   // kGrad: row t of d_o (64 bf16), copied out of its slot before the arrival below
+                if (kGrad) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_d0 + 8 * (i & 1), (i >> 1) & 1, abort_flag));
+                    if (!ok && lane == 0) DIAG(7 + 100 * kMask, i);
+                    if (!ok) break;
+                    const uint8_t *sD = smem + SM::offD + (i & 1) * kTile;
+#pragma unroll
+                    for (int c8 = 0; c8 < 8; ++c8) dq4[c8] = *reinterpret_cast<const uint4 *>(sD + sw128(r, c8));
+                }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
