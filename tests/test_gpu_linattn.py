@@ -201,3 +201,35 @@ def test_degenerate_inputs_zero_rows_and_all_ones(dtype, d):
     assert bool((r == t.expand_as(r)).all())      # exact: small integers in fp32 accumulation
     o = chela.linattn_fwd(ones, ones, ones)
     assert float((o - 1).abs().max()) <= 1e-6
+
+
+@pytest.mark.parametrize("B,L,H,d", [(1, 2100, 1, 64), (3, 4100, 1, 64), (2, 16384, 8, 64), (8, 4096, 8, 64), (1, 65536, 2, 64),
+                                     (37, 2048, 4, 64), (1, 8192, 2, 128), (2, 16384, 4, 128)])
+@pytest.mark.parametrize("pair", [False, True])
+def test_queued_calls_are_deterministic(B, L, H, d, pair):
+    """Twelve calls queued without a host synchronisation (unsplit and split shapes, where the state kernel and the
+    main kernel of a call overlap): the same bits every time, no wait gives up, and no call takes the second that a
+    give-up would cost."""
+    import time
+    import torch
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    shape = (2, B, L, H, d) if pair else (B, L, H, d)
+    q, k, v = ((torch.randn(shape, device="cuda", generator=gen) * 0.125).to(torch.bfloat16) for _ in range(3))
+    if pair:   # low planes three orders of magnitude below the high planes, as a real hi/lo split has them
+        for t in (q, k, v):
+            t[1] *= 2.0 ** -9
+    kw = {"in_dtype": chela.BF16_PAIR} if pair else {}
+    ws = torch.zeros(chela.linattn_workspace_bytes(B, H, L, d, d, 64) + 16, dtype=torch.uint8, device="cuda")
+    o = torch.empty(B, L, H, d, device="cuda")
+    first = chela.linattn_fwd(q, k, v, out=o, workspace=ws, **kw).clone()
+    torch.cuda.synchronize()
+    outs = []
+    t0 = time.perf_counter()
+    for _ in range(12):
+        outs.append(chela.linattn_fwd(q, k, v, out=torch.empty_like(o), workspace=ws, **kw))
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 0.5
+    assert chela.async_status(ws) == chela.OK
+    assert bool(torch.isfinite(first).all())
+    for x in outs:
+        assert torch.equal(first, x)
