@@ -112,3 +112,19 @@ def test_mixer_call_can_be_captured_in_a_cuda_graph():
     graph.replay()
     torch.cuda.synchronize()
     assert torch.equal(o_eager, o_graph)
+
+
+@pytest.mark.parametrize("B,L,D,H,chunk", [(1, 2048, 512, 8, 64), (2, 1000, 256, 2, 128), (1, 4096, 1024, 8, 128)])
+def test_queued_mixer_calls_are_deterministic(B, L, D, H, chunk):
+    import torch
+    m = inputs.mixer(10, B, L, D)
+    args = (to_device(m["x"], "bf16"), dev_f32(m["w_short"]), dev_f32(m["k_long"]), to_device(m["w_q"], "bf16"),
+            to_device(m["w_k"], "bf16"), to_device(m["w_v"], "bf16"), H)
+    ws = torch.zeros(chela.mixer_workspace_bytes(B, L, D, H, chunk), dtype=torch.uint8, device="cuda")
+    first = chela.mixer_fwd(*args, chunk=chunk, workspace=ws).clone()
+    torch.cuda.synchronize()
+    outs = [chela.mixer_fwd(*args, chunk=chunk, workspace=ws) for _ in range(8)]
+    torch.cuda.synchronize()
+    assert chela.async_status(ws) == chela.OK
+    for o in outs:
+        assert torch.equal(first, o)
