@@ -32,9 +32,23 @@ MixerPlan mixer_plan(int B, int L, int D, int H, int chunk, bool gated)
     return p;
 }
 
+// what chela_debug_wait_control last set; process-wide, read by every tensor-core launch
+long long g_wait_limit_cycles = 2000000000LL;   // about one second at B200 clocks
+int g_skip_arrival = 0;
+
 }  // namespace
 
+namespace chela {
+WaitCtl current_wait_ctl() { return WaitCtl{g_wait_limit_cycles, g_skip_arrival}; }
+}  // namespace chela
+
 extern "C" {
+
+void chela_debug_wait_control(long long limit_cycles, int skip_arrival)
+{
+    g_wait_limit_cycles = limit_cycles > 0 ? limit_cycles : 2000000000LL;
+    g_skip_arrival = skip_arrival;
+}
 
 const char *chela_status_string(chela_status_t status)
 {

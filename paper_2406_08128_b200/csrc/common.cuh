@@ -45,6 +45,15 @@ __device__ __forceinline__ float load1(const __nv_bfloat16 *p) { return __bfloat
 __device__ __forceinline__ void store1(float *p, float v) { *p = v; }
 __device__ __forceinline__ void store1(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
 
+// How long a device-side wait may last, and the test hook that makes one run out: the tensor-core kernels take this
+// by value.  `limit` is in SM cycles; `skip_arrival` != 0 asks CTA 0 to leave out one mbarrier arrival (the role that
+// waits for it then gives up after `limit` cycles, records CHELA_ERR_TIMEOUT and the kernel returns by itself).
+struct WaitCtl {
+    long long limit;
+    int skip_arrival;
+};
+WaitCtl current_wait_ctl();   // what chela_debug_wait_control last set (default: about one second, no skipped arrival)
+
 // ---- launchers implemented in the other translation units ------------------------------------
 
 chela_status_t launch_linattn_simt(const void *q, const void *k, const void *v, void *o, int B, int H,
@@ -61,6 +70,12 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
                                     chela_dtype_t out_dtype, int norm, float eps, float scale,
                                     void *workspace, cudaStream_t stream, const float *state_in = nullptr,
                                     float *state_out = nullptr, bool reverse = false, int pair_mask = 7, bool keep_status = false);
+
+// chain-free kernel for plain bf16, d = 64, fewer (batch, head) pairs than SMs (one CTA per SM, `stride` CTAs per sequence)
+int linattn_sm100_pipe_stride(int B, int H, int L, int sms);
+chela_status_t launch_linattn_sm100_pipe(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int stride,
+                                         chela_dtype_t out_dtype, int norm, float eps, float scale, int *status,
+                                         const float *state_in, float *state_out, cudaStream_t stream);
 
 size_t linattn_sm100_d128_workspace_bytes(int B, int H, int L);
 void linattn_sm100_d128_split(int B, int H, int L, int sms, int *G, int *cg0, int *cg);

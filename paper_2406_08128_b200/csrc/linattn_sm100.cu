@@ -73,16 +73,6 @@ constexpr int kTmemCols = 128;
 constexpr int kColOS = 0;    // rows 0..63: output tile, rows 64..127: running state; 64 columns
 constexpr int kColPT = 64;   // rows 64..127: transposed scores; 64 columns
 
-#ifdef CHELA_TIMING
-#define TMARK(n) do { long long tn = clock64(); tacc[n] += tn - tprev; tprev = tn; } while (0)
-#define TDECL long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, tprev = clock64()
-#define TDUMP(slot) do { for (int n_ = 0; n_ < 8; ++n_) reinterpret_cast<long long *>(status)[4 + 8 * (slot) + n_] = tacc[n_]; } while (0)
-#else
-#define TMARK(n)
-#define TDECL
-#define TDUMP(slot)
-#endif
-
 // kReverse: the anti-causal mirror (token t attends keys s >= t; the state accumulates from the end of the
 // sequence).  Chunks are walked from the last to the first and the mask is the upper triangle; everything
 // else, including the split into groups, works on the mirrored chunk index.  Used by the backward pass.
@@ -94,7 +84,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                      const __grid_constant__ CUtensorMap tm_d, int H, int L,
                      float scale, int norm, float eps, int *__restrict__ status, const float *__restrict__ s_part,
-                     int G, int cg0, int cg, const float *__restrict__ state_in, float *__restrict__ state_out)
+                     int G, int cg0, int cg, const float *__restrict__ state_in, float *__restrict__ state_out, const WaitCtl wc)
 {
     // Grid: one CTA per (group, batch*head), group-major.  Group 0 covers the first cg0 chunks of its sequence, group
     // g >= 1 the next cg chunks each (the last one what is left).  Group g starts from the state
@@ -163,7 +153,6 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     if (warp == 4) {
         // =========================================== issuer: TMA loads and every tcgen05.mma ==========
         if (lane == 0) {
-            TDECL;
             auto stage_base = [&](int chunk) { return sbase + SM::offStage + (chunk % kStages) * kTPS * kTile; };
             auto issue_load = [&](int chunk) {
                 const uint32_t bar = bar_full0 + 8 * (chunk % kStages), dst = stage_base(chunk);
@@ -180,7 +169,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
             // G1 of a chunk; false if the chunk's tiles never arrived
             auto issue_scores = [&](int chunk) -> bool {
-                if (!mbar_wait(bar_full0 + 8 * (chunk % kStages), (chunk / kStages) & 1, abort_flag)) { DIAG(1 + 100 * kMask, chunk); return false; }
+                if (!mbar_wait(bar_full0 + 8 * (chunk % kStages), (chunk / kStages) & 1, abort_flag, wc.limit)) { DIAG(1 + 100 * kMask, chunk); return false; }
                 tc_fence_after();
                 const uint32_t qk_lo = desc_lo(stage_base(chunk));
 #pragma unroll
@@ -218,12 +207,11 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (i > 0 || has_init) {
                     // G2: rows 0..63 of OS = Q S_hi + Q S_lo; needs the state tiles of the previous chunk (or
                     // of the group's initial state) and the previous output rows out of TMEM
-                    ok = mbar_wait(bar_s, par_s, abort_flag);
+                    ok = mbar_wait(bar_s, par_s, abort_flag, wc.limit);
                     if (!ok) DIAG(2 + 100 * kMask, i);
                     par_s ^= 1;
                     if (!ok) break;
                     tc_fence_after();
-                    TMARK(0);
                     if (kGrad && i >= 1 && i + 1 < nchunks) {   // the epilogue warps hold d_o of chunk i - 1: its slot takes chunk i + 1
                         issue_d(i + 1);
                         ++d_issued;
@@ -238,14 +226,12 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
                         for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS, qk2_lo + 2 * k, shi_lo + 128 * k, idescG2, 1, 1);
                     }
-                    TMARK(1);
                 }
                 // G3: OS += [P^T | K]^T V; atom 0 = score tile, atom 1 = K tile of this stage
-                ok = mbar_wait(bar_pt, i & 1, abort_flag);
+                ok = mbar_wait(bar_pt, i & 1, abort_flag, wc.limit);
                 if (!ok) DIAG(3 + 100 * kMask, i);
                 if (!ok) break;
                 tc_fence_after();
-                TMARK(2);
                 const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st + 2 * kTile);
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k)
@@ -268,9 +254,8 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     ok = issue_scores(i + 1);
                     if (!ok) break;
                 }
-                TMARK(3);
                 // the stage is free once G3 has completed: prefetch the chunk that will use it next
-                ok = mbar_wait(bar_o, i & 1, abort_flag);
+                ok = mbar_wait(bar_o, i & 1, abort_flag, wc.limit);
                 if (!ok) DIAG(4 + 100 * kMask, i);
                 if (!ok) break;
                 consumed = i + 1;
@@ -278,20 +263,16 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     issue_load(i + kStages);
                     ++loads_issued;
                 }
-                TMARK(4);
             }
             if (!ok) {
                 *abort_flag = 1;
                 atomicExch(status, (int)CHELA_ERR_TIMEOUT);
                 // drain loads that were issued but never consumed (bounded), so no copy lands after exit
                 for (int c = consumed; c < loads_issued; ++c)
-                    mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1, nullptr);
+                    mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1, nullptr, wc.limit);
                 if (kGrad)
-                    for (int c = d_issued > 2 ? d_issued - 2 : 0; c < d_issued; ++c) mbar_wait(bar_d0 + 8 * (c & 1), (c >> 1) & 1, nullptr);
+                    for (int c = d_issued > 2 ? d_issued - 2 : 0; c < d_issued; ++c) mbar_wait(bar_d0 + 8 * (c & 1), (c >> 1) & 1, nullptr, wc.limit);
             }
-#ifdef CHELA_TIMING
-            if (blockIdx.x == 0) TDUMP(0);
-#endif
         }
     } else {
         // =========================================== compute warps ====================================
@@ -301,7 +282,6 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const int r = tid & 63;
         const uint32_t tmem_warp = tmem + ((uint32_t)(warp * 32) << 16);
         bool ok = true;
-        TDECL;
         // state row r -> bf16 hi + lo -> shared (MN-major B operand of G2)
         auto write_state_tiles = [&](const float(&sv)[kD]) {
             uint8_t *sHi = smem + SM::offShi, *sLo = smem + SM::offSlo;
@@ -358,11 +338,10 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int i = 0; i < nchunks; ++i) {
             if (upper) {
                 // ---- P^T_i: TMEM -> causal mask -> bf16 -> shared (rows = s, 64 t per row) -------------
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_p, i & 1, abort_flag));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_p, i & 1, abort_flag, wc.limit));
                 if (!ok && lane == 0) DIAG(6 + 100 * kMask, i);
                 if (!ok) break;
                 tc_fence_after();
-                TMARK(0);
                 // row s keeps t >= s (mirrored: t <= s); all-zero blocks are not read from TMEM
                 float p[2][32];
                 // causal: rows s >= 32 (warp 3) have nothing at t < 32; mirrored: rows s < 32 (warp 2) nothing at t >= 32
@@ -396,14 +375,12 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 fence_proxy_async();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_pt);
-                TMARK(1);
+                if (lane == 0 && !(wc.skip_arrival && blockIdx.x == 0 && i == 0)) mbar_arrive(bar_pt);   // test hook: one arrival left out
             }
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag));
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag, wc.limit));
             if (!ok && lane == 0) DIAG(8 + 100 * kMask + 10 * warp, i);
             if (!ok) break;
             tc_fence_after();
-            TMARK(2);
             float acc[kD];
             if (!upper) {
                 // ---- output row t: scale, normaliser -> swizzled staging -> TMA store (per warp: 32 rows) ----
@@ -412,7 +389,7 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 tmem_ld_wait();
                 uint4 dq4[kGrad ? 8 : 1];   // kGrad: row t of d_o (64 bf16), copied out of its slot before the arrival below
                 if (kGrad) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_d0 + 8 * (i & 1), (i >> 1) & 1, abort_flag));
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_d0 + 8 * (i & 1), (i >> 1) & 1, abort_flag, wc.limit));
                     if (!ok && lane == 0) DIAG(7 + 100 * kMask, i);
                     if (!ok) break;
                     const uint8_t *sD = smem + SM::offD + (i & 1) * kTile;
@@ -486,7 +463,6 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                                          tok(i) + warp * 32, b, 0);   // the map's rank is 5 (plane = 0)
                     bulk_commit();
                 }
-                TMARK(3);
             } else {
                 // ---- state row d_k: bf16 hi + lo -> shared (MN-major B operand of the next chunk's G2) ------
                 if (i + 1 < nchunks) {
@@ -507,7 +483,6 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
                     for (int j = 0; j < kD / 4; ++j) dst[j] = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
                 }
-                TMARK(3);
             }
         }
         if (!ok && lane == 0) {
@@ -515,9 +490,6 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             atomicExch(status, (int)CHELA_ERR_TIMEOUT);
         }
         if (!upper && lane == 0) bulk_wait0();   // output boxes fully written before the CTA retires
-#ifdef CHELA_TIMING
-        if (blockIdx.x == 0 && (tid == 0 || tid == 64)) TDUMP(tid == 0 ? 1 : 2);
-#endif
     }
     tc_fence_before();
     __syncthreads();
@@ -547,7 +519,7 @@ struct SmemState {
 template <int kMask, bool kReverse>
 __global__ void __launch_bounds__(kThreads)
 linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                     float *__restrict__ s_part, int H, int L, int G, int cg0, int cg, int *__restrict__ status)
+                     float *__restrict__ s_part, int H, int L, int G, int cg0, int cg, int *__restrict__ status, const WaitCtl wc)
 {
     using SM = SmemState<kMask>;
     constexpr int kKV = SM::kKV;
@@ -607,7 +579,7 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             bool ok = true;
             for (int i = 0; i < nchunks; ++i) {
                 const int stage = i % kStStages;
-                ok = mbar_wait(bar_full0 + 8 * stage, (i / kStStages) & 1, abort_flag);
+                ok = mbar_wait(bar_full0 + 8 * stage, (i / kStStages) & 1, abort_flag, wc.limit);
                 if (!ok) DIAG(9001 + 100 * kMask, i);
                 if (!ok) break;
                 tc_fence_after();
@@ -628,7 +600,7 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 umma_commit(bar_empty0 + 8 * stage);
                 consumed = i + 1;
                 if (i + kStStages < nchunks) {
-                    ok = mbar_wait(bar_empty0 + 8 * stage, (i / kStStages) & 1, abort_flag);
+                    ok = mbar_wait(bar_empty0 + 8 * stage, (i / kStStages) & 1, abort_flag, wc.limit);
                     if (!ok) DIAG(9002 + 100 * kMask, i);
                     if (!ok) break;
                     issue_load(i + kStStages);
@@ -640,11 +612,11 @@ linattn_state_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 *abort_flag = 1;
                 atomicExch(status, (int)CHELA_ERR_TIMEOUT);
                 for (int c = consumed; c < loads_issued; ++c)
-                    mbar_wait(bar_full0 + 8 * (c % kStStages), (c / kStStages) & 1, nullptr);
+                    mbar_wait(bar_full0 + 8 * (c % kStStages), (c / kStStages) & 1, nullptr, wc.limit);
             }
         }
     } else if (warp < 2) {
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_done, 0, abort_flag));
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_done, 0, abort_flag, wc.limit));
         if (ok) {
             tc_fence_after();
             float sv[kD];
@@ -761,6 +733,7 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
         !make_map(&mv, v, B, H, L, kC, false, pv) || !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4, 1))
         return CHELA_ERR_CUDA;
     const SplitPlan plan = split_plan(B, H, L, Smem<TOut, kMask>::bytes > 113 * 1024);
+    const WaitCtl wc = current_wait_ctl();
     int *status = (int *)workspace;
     float *s_part = (float *)((char *)workspace + kWsHeader);
     // keep_status: a later launch of a multi-launch call must not erase what an earlier one reported
@@ -769,7 +742,7 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
         auto skern = linattn_state_kernel<(kMask & 6), kReverse>;
         constexpr int ssmem = SmemState<(kMask & 6)>::bytes;
         if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, ssmem) != cudaSuccess) return CHELA_ERR_CUDA;
-        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cg0, plan.cg, status);
+        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cg0, plan.cg, status, wc);
         if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
     }
     auto kern = linattn_sm100_kernel<TOut, kMask, kReverse>;
@@ -778,9 +751,9 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
         return CHELA_ERR_CUDA;
     if (plan.G > 1)
         return launch_dependent(kern, B * H * plan.G, smem, stream, mq, mk, mv, mo, mo, H, L, scale, norm, eps, status,
-                                (const float *)s_part, plan.G, plan.cg0, plan.cg, state_in, state_out);
+                                (const float *)s_part, plan.G, plan.cg0, plan.cg, state_in, state_out, wc);
     kern<<<B * H, kThreads, smem, stream>>>(mq, mk, mv, mo, mo, H, L, scale, norm, eps, status, s_part, 1, plan.cg0, plan.cg,
-                                            state_in, state_out);
+                                            state_in, state_out, wc);
     return last_launch_status();
 }
 
@@ -795,6 +768,7 @@ chela_status_t launch_grad(const void *q, const void *k, const void *v, const vo
         return CHELA_ERR_CUDA;
     using SM = Smem<__nv_bfloat16, 8, true>;
     const SplitPlan plan = split_plan(B, H, L, SM::bytes > 113 * 1024);
+    const WaitCtl wc = current_wait_ctl();
     int *status = (int *)workspace;
     float *s_part = (float *)((char *)workspace + kWsHeader);
     if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
@@ -802,16 +776,16 @@ chela_status_t launch_grad(const void *q, const void *k, const void *v, const vo
         auto skern = linattn_state_kernel<0, false>;
         constexpr int ssmem = SmemState<0>::bytes;
         if (cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, ssmem) != cudaSuccess) return CHELA_ERR_CUDA;
-        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cg0, plan.cg, status);
+        skern<<<B * H * (plan.G - 1), kThreads, ssmem, stream>>>(mk, mv, s_part, H, L, plan.G, plan.cg0, plan.cg, status, wc);
         if (cudaGetLastError() != cudaSuccess) return CHELA_ERR_CUDA;
     }
     auto kern = linattn_sm100_kernel<__nv_bfloat16, 8, false, true>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::bytes) != cudaSuccess) return CHELA_ERR_CUDA;
     if (plan.G > 1)
         return launch_dependent(kern, B * H * plan.G, SM::bytes, stream, mq, mk, mv, mg, md, H, L, scale, 1, eps, status,
-                                (const float *)s_part, plan.G, plan.cg0, plan.cg, (const float *)nullptr, (float *)nullptr);
+                                (const float *)s_part, plan.G, plan.cg0, plan.cg, (const float *)nullptr, (float *)nullptr, wc);
     kern<<<B * H, kThreads, SM::bytes, stream>>>(mq, mk, mv, mg, md, H, L, scale, 1, eps, status, s_part, 1, plan.cg0, plan.cg,
-                                                 nullptr, nullptr);
+                                                 nullptr, nullptr, wc);
     return last_launch_status();
 }
 
@@ -881,6 +855,11 @@ chela_status_t launch_linattn_sm100(const void *q, const void *k, const void *v,
         if (out_dtype == CHELA_F32)
             return launch_t<float, 15, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pm, keep_status);
         return launch_t<__nv_bfloat16, 15, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, pm, keep_status);
+    }
+    // plain bf16 with fewer (batch, head) pairs than SMs: the chain-free kernel, one CTA per SM, sequences shared by stride
+    if (const int stride = linattn_sm100_pipe_stride(B, H, L, 0)) {
+        if (!keep_status && cudaMemsetAsync(workspace, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
+        return launch_linattn_sm100_pipe(q, k, v, o, B, H, L, stride, out_dtype, norm, eps, scale, (int *)workspace, state_in, state_out, stream);
     }
     if (out_dtype == CHELA_F32) return launch_t<float, 0, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 0, keep_status);
     return launch_t<__nv_bfloat16, 0, false>(q, k, v, o, B, H, L, norm, eps, scale, workspace, state_in, state_out, stream, 0, keep_status);

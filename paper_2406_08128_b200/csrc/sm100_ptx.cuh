@@ -32,13 +32,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kWaitCycles, or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag)
+// Bounded wait: false if the phase did not complete within `limit` cycles, or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag, long long limit = kWaitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity))
-        if (clock64() - t0 > kWaitCycles || (abort_flag && *abort_flag)) return false;
+        if (clock64() - t0 > limit || (abort_flag && *abort_flag)) return false;
     return true;
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
