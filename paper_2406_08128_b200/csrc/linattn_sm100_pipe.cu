@@ -8,9 +8,9 @@
 //   G1_i : [V_i ; K_i] Q_i^T                  -> TMEM PT[i%2]; rows 64..127 are P^T = K_i Q_i^T
 //   G3_i : [P_i^T | K_i]^T V_i   (fresh)      -> TMEM OS[i%2]; rows 0..63 = P_i V_i, rows 64..127 = dS_i = K_i^T V_i
 //   G2_i : rows 0..63 of OS[i%2] += Q_i S_{i-1}   (S_{i-1} as bf16 hi + lo tiles in shared memory)
-// and the recurrence S_i = S_{i-1} + dS_i is an fp32 add in the registers of the two state warps, which write the
-// hi/lo tiles for the next chunk's G2.  G3_{i+1} and G1_{i+2} are issued before G2_{i+1}, so the tensor core always has
-// work while the state warps turn dS_i into tiles.  Accumulators, score tiles and state tiles are double-buffered.
+// and the recurrence S_i = S_{i-1} + dS_i is an fp32 add in the registers of the state warps, which write the hi/lo
+// tiles for the next chunk's G2.  G3_{i+1} and G1_{i+2} are issued before G2_{i+1}, so the tensor core always has work
+// while the state warps turn dS_i into tiles.  Accumulators, score tiles and state tiles are double-buffered.
 //
 // Sequences are shared between CTAs by stride (B*H*stride <= SMs): CTA g of a sequence owns the chunks g, g + stride, ...
 // and produces their output rows.  The state needs every chunk, so for a chunk it does not own a CTA loads K and V only
@@ -18,10 +18,12 @@
 // before the next own chunk.  The CTAs of a sequence read the same K, V tiles at about the same time, so all but the
 // first read are served by L2: HBM traffic stays the algorithmic Q + K + V + O, with no second kernel and no workspace.
 //
-// Warps: 0,1 output rows (scale, normaliser, TMA store); 2,3 score rows (mask, bf16, shared tile); 4 issues G1 and G3,
-// 5 issues G2 (one thread each; two issuers because a thread issues a tcgen05.mma about every 50 cycles and one chunk
-// has 16 of them); 6,7 state rows; 8 TMA producer.  Roles meet only through mbarriers, every wait bounded: on a timeout the CTA
-// records CHELA_ERR_TIMEOUT, waits (bounded) for its loads and products in flight, frees its TMEM and returns.
+// Warps (16): 0,1,4,5 output rows (scale, normaliser, TMA store; 0,1 take the even own chunks, 4,5 the odd ones);
+// 2,3,6,7 score rows (mask, bf16, shared tile; same alternation); 10,11,14,15 state rows (two warps per half of the
+// columns); one issuing thread in each of: 8 (G1 and G3), 9 (G2), 12 (K^T V of chunks that are not owned), 13 (TMA
+// producer).  One thread issues a tcgen05.mma about every 50 cycles and a chunk has 16 of them, hence several issuers.
+// Roles meet only through mbarriers, every wait bounded: on a timeout the CTA records CHELA_ERR_TIMEOUT, waits
+// (bounded) for its loads and products in flight, frees its TMEM and returns.
 #include "sm100_ptx.cuh"
 
 namespace chela {
@@ -32,15 +34,15 @@ using namespace sm100;
 constexpr int kD = 64;            // head dimension (d_k = d_v)
 constexpr int kC = 64;            // tokens per chunk
 constexpr int kTile = kC * 128;   // one 64-row x 128-byte tile
-constexpr int kThreads = 544;
-// warps 0,1,4,5: output rows; 2,3,6,7: score rows; 10,11,14,15: state rows; one issuing thread each in the following
-constexpr int kWarpG1 = 8, kWarpG3 = 9, kWarpG2 = 12, kWarpRun = 13, kWarpProducer = 16;
-// Ring depths (template parameters): kKV stages of [V | K] (16 KB each) and kQ stages of Q (8 KB each).  The producer
+constexpr int kThreads = 512;
+constexpr int kWarpA = 8, kWarpG2 = 9, kWarpRun = 12, kWarpProducer = 13;
+
+// kShared: stride > 1.  Ring depths: kKV stages of [V | K] (16 KB each) and kQ stages of Q (8 KB each).  The producer
 // loads a chunk's Q with its K and V, so with one CTA per sequence the Q ring is as deep as the K, V ring (6 + 6); a CTA
 // that owns every second to fourth chunk needs fewer Q stages and gets one more K, V stage (7 + 4).
-
-template <typename TOut, int kKV, int kQ>
+template <typename TOut, bool kShared>
 struct SmemP {
+    static constexpr int kKV = kShared ? 7 : 6, kQ = kShared ? 4 : 6;
     static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as 128-byte wide boxes
     static constexpr int offPT = 0;                               // masked scores, transposed (rows = s), two buffers
     static constexpr int offS = offPT + 2 * kTile;                // state tiles: [buffer][hi, lo], rows = d_k
@@ -48,62 +50,50 @@ struct SmemP {
     static constexpr int offQ = offKV + kKV * 2 * kTile;
     static constexpr int offO = offQ + kQ * kTile;                // output staging, two buffers; also what G2's 128-row operand reads past Q
     static constexpr int offBar = offO + 2 * kOBoxes * kTile;
-    static constexpr int nBar = 2 * kKV + 2 * kQ + 2 * 8 + 4;
+    static constexpr int nBar = 2 * kKV + 2 * kQ + 2 * 8 + 3;
     static constexpr int offTmem = offBar + 8 * nBar;
     static constexpr int offAbort = offTmem + 8;
-    static constexpr int bytes = offAbort + 8;
+    static constexpr int offProbe = offAbort + 8;                 // wait-time counters of a timing build
+    static constexpr int bytes = offProbe + 8 * 32;
 };
-// TMEM columns: PT[2] at 0, 64; OS[2] at 128, 192; DS[2] at 256, 320 (strided only)
+// TMEM columns: PT[2] at 0, 64; OS[2] at 128, 192; DS[2] at 256, 320 (kShared only)
 constexpr int kColPT = 0, kColOS = 128, kColDS = 256;
 
-// A waiting warp backs off between polls: with a dozen roles per SM, spinning warps that poll without a pause take
-// issue slots and shared-memory pipeline slots from the few warps that have work (measured: 0.54 -> 0.45 ms at L = 32K).
-#ifndef PIPE_NANOSLEEP
-#define PIPE_NANOSLEEP 20
-#endif
-constexpr unsigned kSpinSleepNs = PIPE_NANOSLEEP;
-
-// The spin of a bounded wait, out of line: the issuing threads run long straight-line code, one lane at a time, and
-// every inlined spin loop is instruction-cache footprint they pay for.
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const volatile int *abort_flag, long long limit)
+// The spin of a bounded wait, out of line: the roles run long straight-line code and every inlined spin loop is
+// instruction-cache footprint they pay for (inlined: 0.54 ms at L = 32K, out of line: 0.43 ms).
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const volatile int *abort_flag, long long limit, unsigned long long *probe)
 {
     const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        __nanosleep(kSpinSleepNs);
-        if (clock64() - t0 > limit || *abort_flag) return false;
-    }
-    return true;
+    bool ok = true;
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > limit || *abort_flag) {
+            ok = false;
+            break;
+        }
+#ifdef PIPE_TIMING
+    atomicAdd(probe, (unsigned long long)(clock64() - t0));
+#endif
+    return ok;
 }
 
-#ifdef PIPE_TIMING
-#define TW(slot, expr) ([&]() { const long long t_ = clock64(); const bool r_ = (expr); tacc[slot] += clock64() - t_; return r_; }())
-#define TMARK(n) do { const long long tn_ = clock64(); tb[n] += tn_ - tprev; tprev = tn_; } while (0)
-#define TDECL long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long tstart = clock64(); long long tb[8] = {0, 0, 0, 0, 0, 0, 0, 0}, tprev = tstart
-#define TBDUMP(slot) do { if (blockIdx.x == 0 && lane == 0) for (int n_ = 0; n_ < 8; ++n_) reinterpret_cast<long long *>(status)[80 + 8 * (slot) + n_] = tb[n_]; } while (0)
-#define TDUMP(role) do { if (blockIdx.x == 0 && lane == 0) { tacc[7] = clock64() - tstart; for (int n_ = 0; n_ < 8; ++n_) reinterpret_cast<long long *>(status)[8 + 8 * (role) + n_] = tacc[n_]; } } while (0)
-#else
-#define TW(slot, expr) (expr)
-#define TMARK(n)
-#define TBDUMP(slot)
-#define TDECL
-#define TDUMP(role)
-#endif
 #define PDIAG(site, extra) do { if (atomicCAS(status + 8, 0, 7000 + (site)) == 0) { status[9] = blockIdx.x; status[10] = (extra); status[11] = gridDim.x; } } while (0)
 
-template <typename TOut, int kKV, int kQ>
+template <typename TOut, bool kShared>
 __global__ void __launch_bounds__(kThreads, 1)
 linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int H, int L,
-                          float scale, int norm, float eps, int *__restrict__ status, int stride,
+                          float scale, int norm, float eps, int *__restrict__ status, int stride_arg,
                           const float *__restrict__ state_in, float *__restrict__ state_out, const WaitCtl wc)
 {
-    using SM = SmemP<TOut, kKV, kQ>;
+    using SM = SmemP<TOut, kShared>;
+    constexpr int kKV = SM::kKV, kQ = SM::kQ;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     if (sbase & 1023u) {  // swizzled tiles need a 1024-byte aligned base: report instead of corrupting
         if (threadIdx.x == 0) atomicExch(status, (int)CHELA_ERR_CUDA);
         return;
     }
+    const int stride = kShared ? stride_arg : 1;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.x / stride, g = blockIdx.x % stride;
     const int b = bh / H, h = bh % H;
@@ -112,7 +102,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const int n_own = g < nch_total ? (nch_total - 1 - g) / stride + 1 : 0;
     const int nchunks = n_own ? g + (n_own - 1) * stride + 1 : 0;
     const bool have_state = state_in != nullptr;
-    const uint32_t tmem_cols = stride > 1 ? 512u : 256u;
+    constexpr uint32_t tmem_cols = kShared ? 512u : 256u;
 
     // ---- barriers -------------------------------------------------------------------------------------------------
     const uint32_t bar_kv_full = sbase + SM::offBar;                 // [kKV] K, V of a chunk have landed
@@ -121,15 +111,16 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const uint32_t bar_q_empty = bar_q_full + 8 * kQ;                // [kQ]
     const uint32_t bar_p = bar_q_empty + 8 * kQ;                     // [2] G1 completed (tensor core -> score warps)
     const uint32_t bar_pt = bar_p + 16;                              // [2] score tile in shared memory (score warps -> issuer)
-    const uint32_t bar_ds = bar_pt + 16;                             // [2] G3 completed (-> state warps)
+    const uint32_t bar_ds = bar_pt + 16;                             // [2] G3 completed (-> state warps, G2 issuer, score warps)
     const uint32_t bar_o = bar_ds + 16;                              // [2] G2 completed (-> output warps, state warps)
     const uint32_t bar_of = bar_o + 16;                              // [2] OS buffer read by output and state warps (-> issuer)
-    const uint32_t bar_s = bar_of + 16;                              // [2] state tiles written (state warps -> issuer)
+    const uint32_t bar_s = bar_of + 16;                              // [2] state tiles written (state warps -> G2 issuer)
     const uint32_t bar_dn = bar_s + 16;                              // [2] K^T V of a run of chunks that are not owned completed (-> state warps)
-    const uint32_t bar_df = bar_dn + 16;                             // [2] DS buffer read (state warps -> issuer)
-    const uint32_t bar_fin = bar_df + 16;                            // [4] every product an issuer has issued has completed (exit path)
+    const uint32_t bar_df = bar_dn + 16;                             // [2] DS buffer read (state warps -> run issuer)
+    const uint32_t bar_fin = bar_df + 16;                            // [3] every product an issuer has issued has completed (exit path)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
+    unsigned long long *probe = reinterpret_cast<unsigned long long *>(smem + SM::offProbe);
 
     if (tid == 0) {
         for (int s = 0; s < kKV; ++s) {
@@ -150,7 +141,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             mbar_init(bar_dn + 8 * s, 1);
             mbar_init(bar_df + 8 * s, 4);
         }
-        for (int s = 0; s < 4; ++s) mbar_init(bar_fin + 8 * s, 1);
+        for (int s = 0; s < 3; ++s) mbar_init(bar_fin + 8 * s, 1);
         *abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tm_q);
@@ -158,6 +149,9 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         tma_prefetch_desc(&tm_v);
         tma_prefetch_desc(&tm_o);
     }
+#ifdef PIPE_TIMING
+    if (tid < 32) probe[tid] = 0;
+#endif
     if (warp == 0) {
         tmem_alloc(sbase + SM::offTmem, tmem_cols);
         tmem_relinquish();
@@ -167,11 +161,14 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    auto own = [&](int chunk) { return chunk % stride == g; };
-    auto pwait = [&](uint32_t bar, uint32_t parity) { return mbar_try_wait(bar, parity) || wait_slow(bar, parity, abort_flag, wc.limit); };
+    // `site` names the wait in the timing build's counters and, plus 7000, in the diagnostics of a wait that gave up
+    auto pwait = [&](uint32_t bar, uint32_t parity, int site) {
+        return mbar_try_wait(bar, parity) || wait_slow(bar, parity, abort_flag, wc.limit, probe + site);
+    };
     auto kv_stage = [&](int chunk) { return sbase + SM::offKV + (chunk % kKV) * 2 * kTile; };   // V tile, then K tile
     auto q_stage = [&](int oi) { return sbase + SM::offQ + (oi % kQ) * kTile; };
     auto give_up = [&](int site, int extra) {
+        if (*abort_flag) return;   // another role gave up first: its diagnostics stand
         PDIAG(site, extra);
         *abort_flag = 1;
         atomicExch(status, (int)CHELA_ERR_TIMEOUT);
@@ -180,20 +177,13 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     if (warp == kWarpProducer) {
         // =========================================== TMA producer ======================================================
         if (lane == 0) {
-            TDECL;
-            int issued = 0, oi = 0;
+            int issued = 0, oi = 0, next_own = g;
             bool ok = true;
             for (int j = 0; ok && j < nchunks; ++j) {
                 const int s = j % kKV;
-                if (j >= kKV) {
-                    ok = TW(0, pwait(bar_kv_empty + 8 * s, (j / kKV - 1) & 1));
-                    if (!ok) { if (!*abort_flag) give_up(1, j); break; }
-                }
-                const bool mine = own(j);
-                if (mine && oi >= kQ) {
-                    ok = TW(1, pwait(bar_q_empty + 8 * (oi % kQ), (oi / kQ - 1) & 1));
-                    if (!ok) { if (!*abort_flag) give_up(2, j); break; }
-                }
+                if (j >= kKV && !(ok = pwait(bar_kv_empty + 8 * s, (j / kKV - 1) & 1, 1))) { give_up(1, j); break; }
+                const bool mine = j == next_own;
+                if (mine && oi >= kQ && !(ok = pwait(bar_q_empty + 8 * (oi % kQ), (oi / kQ - 1) & 1, 2))) { give_up(2, j); break; }
                 mbar_expect_tx(bar_kv_full + 8 * s, 2 * kTile);
                 tma_load_5d(kv_stage(j), &tm_v, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
                 tma_load_5d(kv_stage(j) + kTile, &tm_k, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
@@ -201,6 +191,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     mbar_expect_tx(bar_q_full + 8 * (oi % kQ), kTile);
                     tma_load_5d(q_stage(oi), &tm_q, bar_q_full + 8 * (oi % kQ), 0, h, j * kC, b, 0);
                     ++oi;
+                    next_own += stride;
                 }
                 issued = j + 1;
             }
@@ -210,62 +201,45 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     mbar_wait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, nullptr, wc.limit);
                 for (int q = oi > kQ ? oi - kQ : 0; q < oi; ++q) mbar_wait(bar_q_full + 8 * (q % kQ), (q / kQ) & 1, nullptr, wc.limit);
             }
-            TDUMP(0);
         }
-    } else if (warp == kWarpG1) {
-        // =========================================== issuer of G1: PT[buf] = [V;K] Q^T ================================
+    } else if (warp == kWarpA) {
+        // =========================================== issuer of G1 and G3 ================================================
         if (lane == 0) {
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [V;K] (K-major) x Q^T (K-major)
+            constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
             bool ok = true;
-            TDECL;
-            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
-                const int buf = oi & 1;
-                ok = TW(0, pwait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1));
-                if (!ok) { if (!*abort_flag) give_up(11, j); break; }
-                ok = TW(1, pwait(bar_q_full + 8 * (oi % kQ), (oi / kQ) & 1));
-                if (!ok) { if (!*abort_flag) give_up(12, j); break; }
-                if (oi >= 2) {   // the score warps have taken own chunk oi - 2 out of PT[buf]
-                    ok = TW(2, pwait(bar_pt + 8 * buf, ((oi >> 1) - 1) & 1));
-                    if (!ok) { if (!*abort_flag) give_up(13, j); break; }
-                }
+            // G1 of own chunk number oi (chunk j): PT[oi & 1] = [V;K] Q^T.  The score warps have taken own chunk oi - 2 out of
+            // that buffer: this thread has waited for their tile (bar_pt) before it issued G3 of that chunk.
+            auto issue_scores = [&](int oi, int j) -> bool {
+                if (!pwait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, 3)) { give_up(3, j); return false; }
+                if (!pwait(bar_q_full + 8 * (oi % kQ), (oi / kQ) & 1, 4)) { give_up(4, j); return false; }
                 tc_fence_after();
                 const uint32_t vk_lo = desc_lo(kv_stage(j)), q_lo = desc_lo(q_stage(oi));
 #pragma unroll
-                for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT + 64 * buf, vk_lo + 2 * k, q_lo + 2 * k, idescG1, k > 0);
-                umma_commit(bar_p + 8 * buf);
-            }
-            umma_commit(bar_fin);   // every product issued by this thread has completed before TMEM and shared memory go away
-            pwait(bar_fin, 0);
-            TDUMP(1);
-        }
-    } else if (warp == kWarpG3) {
-        // =========================================== issuer of G3: OS[buf] = [P^T | K]^T V (fresh) ====================
-        if (lane == 0) {
-            constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
-            bool ok = true;
-            TDECL;
+                for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT + 64 * (oi & 1), vk_lo + 2 * k, q_lo + 2 * k, idescG1, k > 0);
+                umma_commit(bar_p + 8 * (oi & 1));
+                return true;
+            };
+            if (n_own > 0) ok = issue_scores(0, g);
             for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
                 const int buf = oi & 1;
                 const uint32_t ph = (oi >> 1) & 1;
-                ok = TW(0, pwait(bar_pt + 8 * buf, ph));
-                if (!ok) { if (!*abort_flag) give_up(15, j); break; }
-                if (oi >= 2) {   // output and state warps have taken own chunk oi - 2 out of OS[buf]
-                    ok = TW(1, pwait(bar_of + 8 * buf, ph ^ 1));
-                    if (!ok) { if (!*abort_flag) give_up(16, j); break; }
-                }
-                ok = TW(2, pwait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1));   // long complete: makes the copy visible to this thread
-                if (!ok) { if (!*abort_flag) give_up(14, j); break; }
+                // G1 of the next own chunk first: its score tile is ready long before its G3 is due
+                if (oi + 1 < n_own && !(ok = issue_scores(oi + 1, j + stride))) break;
+                // ---- G3: OS[buf] = [P^T | K]^T V (fresh) ----------------------------------------------------------------
+                if (!(ok = pwait(bar_pt + 8 * buf, ph, 5))) { give_up(5, j); break; }
+                // output and state warps have taken own chunk oi - 2 out of OS[buf]
+                if (oi >= 2 && !(ok = pwait(bar_of + 8 * buf, ph ^ 1, 6))) { give_up(6, j); break; }
                 tc_fence_after();
                 const uint32_t st = kv_stage(j), pt = sbase + SM::offPT + buf * kTile;
                 const uint32_t a_lo = desc_lo(pt, st + kTile - pt), v_lo = desc_lo(st);
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS + 64 * buf, a_lo + 128 * k, v_lo + 128 * k, idescG3, k > 0);
                 umma_commit(bar_ds + 8 * buf);
-                umma_commit(bar_kv_empty + 8 * (j % kKV));   // K and V are read by G1 (completed: its scores were consumed) and G3 only
+                umma_commit(bar_kv_empty + 8 * (j % kKV));   // K and V are read by G1 and G3 only
             }
-            umma_commit(bar_fin + 8);
-            pwait(bar_fin + 8, 0);
-            TDUMP(5);
+            umma_commit(bar_fin);   // every product issued by this thread has completed before TMEM and shared memory go away
+            pwait(bar_fin, 0, 7);
         }
     } else if (warp == kWarpG2) {
         // =========================================== issuer of G2: rows 0..63 of OS[buf] += Q S_hi + Q S_lo ==========
@@ -273,19 +247,16 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         if (lane == 0) {
             constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;..] (K-major) x S (MN-major)
             bool ok = true;
-            TDECL;
             for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
                 const int buf = oi & 1;
                 const uint32_t ph = (oi >> 1) & 1;
                 // after G3 of the same chunk (same accumulator), with the state tiles as of the previous chunk (the state
                 // warps arrive for every own chunk, also when there is nothing to add)
-                ok = TW(0, pwait(bar_ds + 8 * buf, ph));
-                if (!ok) { if (!*abort_flag) give_up(18, j); break; }
-                ok = TW(1, pwait(bar_s + 8 * buf, ph));
-                if (!ok) { if (!*abort_flag) give_up(17, j); break; }
+                if (!(ok = pwait(bar_ds + 8 * buf, ph, 8))) { give_up(8, j); break; }
+                if (!(ok = pwait(bar_s + 8 * buf, ph, 9))) { give_up(9, j); break; }
                 if (j > 0 || have_state) {
-                    ok = TW(2, pwait(bar_q_full + 8 * (oi % kQ), (oi / kQ) & 1));   // long complete: makes the copy visible to this thread
-                    if (!ok) { if (!*abort_flag) give_up(19, j); break; }
+                    // long complete: makes the copy visible to this thread
+                    if (!(ok = pwait(bar_q_full + 8 * (oi % kQ), (oi / kQ) & 1, 10))) { give_up(10, j); break; }
                     tc_fence_after();
                     const uint32_t q_lo = desc_lo(q_stage(oi));
                     const uint32_t shi_lo = desc_lo(sbase + SM::offS + buf * 2 * kTile), slo_lo = desc_lo(sbase + SM::offS + (buf * 2 + 1) * kTile);
@@ -297,28 +268,22 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 umma_commit(bar_o + 8 * buf);
                 umma_commit(bar_q_empty + 8 * (oi % kQ));
             }
-            umma_commit(bar_fin + 16);
-            pwait(bar_fin + 16, 0);
-            TDUMP(6);
+            umma_commit(bar_fin + 8);
+            pwait(bar_fin + 8, 0, 11);
         }
     } else if (warp == kWarpRun) {
-        // =========================================== issuer of the K^T V of chunks that other CTAs own (strided) ========
-        if (lane == 0 && stride > 1) {
+        // =========================================== issuer of the K^T V of chunks that other CTAs own ================
+        if (kShared && lane == 0) {
             constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
             bool ok = true;
             int ri = 0;   // runs issued so far
-            TDECL;
             // runs: the chunks before the first own one, then those between consecutive own chunks; each -> rows 64..127
-            // of DS[ri & 1] (output lanes write-disabled)
+            // of DS[ri & 1] (output lanes write-disabled), fresh for every run
             for (int first = 0, last = g - 1; ok && last < nchunks; first = last + 2, last += stride) {
                 if (last < first) continue;   // g = 0: no chunks before the first own one
-                if (ri >= 2) {
-                    ok = TW(0, pwait(bar_df + 8 * (ri & 1), ((ri >> 1) - 1) & 1));
-                    if (!ok) { if (!*abort_flag) give_up(20, first); break; }
-                }
+                if (ri >= 2 && !(ok = pwait(bar_df + 8 * (ri & 1), ((ri >> 1) - 1) & 1, 12))) { give_up(12, first); break; }
                 for (int c = first; ok && c <= last; ++c) {
-                    ok = TW(1, pwait(bar_kv_full + 8 * (c % kKV), (c / kKV) & 1));
-                    if (!ok) { if (!*abort_flag) give_up(21, c); break; }
+                    if (!(ok = pwait(bar_kv_full + 8 * (c % kKV), (c / kKV) & 1, 13))) { give_up(13, c); break; }
                     tc_fence_after();
                     const uint32_t st = kv_stage(c);
                     const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st);
@@ -331,31 +296,26 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 umma_commit(bar_dn + 8 * (ri & 1));
                 ++ri;
             }
-            umma_commit(bar_fin + 24);
-            pwait(bar_fin + 24, 0);
-            TDUMP(7);
+            umma_commit(bar_fin + 16);
+            pwait(bar_fin + 16, 0, 14);
         }
     } else if (warp < 8 && (warp & 2)) {
         // =========================================== score warps =======================================================
-        // thread = row s of P^T (TMEM lane 64 + s): causal mask (t >= s), bf16, swizzled tile with rows = s
-        // warps 2,3 take the even own chunks (buffer 0), warps 6,7 the odd ones (buffer 1)
+        // thread = row s of P^T (TMEM lane 64 + s): causal mask (t >= s), bf16, swizzled tile with rows = s.
+        // Warps 2,3 take the even own chunks (buffer 0), warps 6,7 the odd ones (buffer 1).
         const int r = tid & 63, buf = warp >> 2;
         const bool low = (warp & 1) == 0;   // rows s < 32
         const uint32_t tmem_warp = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        TDECL;
         for (int oi = buf; oi < n_own; oi += 2) {
-            const bool ok = __all_sync(0xffffffffu, TW(0, pwait(bar_p + 8 * buf, (oi >> 1) & 1)));
-            if (!ok) { if (lane == 0 && !*abort_flag) give_up(21, oi); break; }
+            if (!__all_sync(0xffffffffu, pwait(bar_p + 8 * buf, (oi >> 1) & 1, 16))) { if (lane == 0) give_up(16, oi); break; }
             tc_fence_after();
             // rows s >= 32 have nothing at t < 32: all-zero blocks are not read from TMEM
             float p[2][32];
             if (low) tmem_ld32(tmem_warp + kColPT + 64 * buf, p[0]);
             tmem_ld32(tmem_warp + kColPT + 64 * buf + 32, p[1]);
             tmem_ld_wait();
-            if (oi >= 2) {   // G3 of own chunk oi - 2 (another thread's) has finished reading this score tile
-                const bool okd = __all_sync(0xffffffffu, TW(1, pwait(bar_ds + 8 * buf, ((oi >> 1) - 1) & 1)));
-                if (!okd) { if (lane == 0 && !*abort_flag) give_up(22, oi); break; }
-            }
+            // G3 of own chunk oi - 2 (another thread's product) has finished reading this score tile
+            if (oi >= 2 && !__all_sync(0xffffffffu, pwait(bar_ds + 8 * buf, ((oi >> 1) - 1) & 1, 17))) { if (lane == 0) give_up(17, oi); break; }
             uint8_t *sP = smem + SM::offPT + buf * kTile;
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
@@ -378,7 +338,6 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             __syncwarp();
             if (lane == 0 && !(wc.skip_arrival && blockIdx.x == 0 && oi == 0)) mbar_arrive(bar_pt + 8 * buf);   // test hook: one arrival left out
         }
-        if (warp == 2) TDUMP(2);
     } else if (warp == 10 || warp == 11 || warp == 14 || warp == 15) {
         // =========================================== state warps =======================================================
         // thread = row d_k of the state (TMEM lane 64 + d_k) x 32 of its 64 columns (warps 10,11: columns 0..31; warps
@@ -407,14 +366,11 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         };
         bool ok = true;
         int ri = 0;
-        TDECL;
         for (int oi = 0; oi < n_own; ++oi) {
             const int j = g + oi * stride, buf = oi & 1;
-            TMARK(7);
             // 1. the chunks since the previous own one (or since the start) belong to other CTAs: add their K^T V
-            if (stride > 1 && j > 0) {
-                ok = __all_sync(0xffffffffu, TW(0, pwait(bar_dn + 8 * (ri & 1), (ri >> 1) & 1)));
-                if (!ok) { if (lane == 0 && !*abort_flag) give_up(31, j); break; }
+            if (kShared && j > 0) {
+                if (!(ok = __all_sync(0xffffffffu, pwait(bar_dn + 8 * (ri & 1), (ri >> 1) & 1, 20)))) { if (lane == 0) give_up(20, j); break; }
                 tc_fence_after();
                 add_tmem(kColDS + 64 * (ri & 1));
                 tc_fence_before();
@@ -422,14 +378,9 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 if (lane == 0) mbar_arrive(bar_df + 8 * (ri & 1));
                 ++ri;
             }
-            TMARK(0);
             // 2. sv = S_{j-1}: bf16 hi + lo tiles (MN-major B operand of G2_j); the buffer was last read by G2 of own chunk oi - 2
             if (j > 0 || have_state) {
-                if (oi >= 2) {
-                    ok = __all_sync(0xffffffffu, TW(1, pwait(bar_o + 8 * buf, ((oi >> 1) - 1) & 1)));
-                    if (!ok) { if (lane == 0 && !*abort_flag) give_up(32, j); break; }
-                }
-                TMARK(1);
+                if (oi >= 2 && !(ok = __all_sync(0xffffffffu, pwait(bar_o + 8 * buf, ((oi >> 1) - 1) & 1, 21)))) { if (lane == 0) give_up(21, j); break; }
                 uint8_t *sHi = smem + SM::offS + buf * 2 * kTile, *sLo = sHi + kTile;
 #pragma unroll
                 for (int c8 = 0; c8 < kCols / 8; ++c8) {
@@ -446,26 +397,18 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
                     *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
                 }
-                TMARK(2);
                 fence_proxy_async();
-                TMARK(3);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s + 8 * buf);   // also when there is nothing to write (first chunk, no initial state)
             // 3. the own chunk's K^T V (rows 64..127 of OS[buf])
-            ok = __all_sync(0xffffffffu, TW(2, pwait(bar_ds + 8 * buf, (oi >> 1) & 1)));
-            if (!ok) { if (lane == 0 && !*abort_flag) give_up(33, j); break; }
+            if (!(ok = __all_sync(0xffffffffu, pwait(bar_ds + 8 * buf, (oi >> 1) & 1, 22)))) { if (lane == 0) give_up(22, j); break; }
             tc_fence_after();
-            TMARK(4);
             add_tmem(kColOS + 64 * buf);
-            TMARK(5);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_of + 8 * buf);
-            TMARK(6);
         }
-        if (warp == 10) TDUMP(3);
-        if (warp == 10) TBDUMP(0);
         if (ok && state_out && nchunks == nch_total) {
             // this CTA owns the last chunk of the sequence: the fp32 state leaves the SM once, for the caller
             float4 *dst = reinterpret_cast<float4 *>(state_out + ((size_t)bh * kD + r) * kD + c0);
@@ -473,15 +416,14 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             for (int j = 0; j < kCols / 4; ++j) dst[j] = make_float4(sv[4 * j], sv[4 * j + 1], sv[4 * j + 2], sv[4 * j + 3]);
         }
     } else if (warp < 8) {
-        // =========================================== output warps (0, 1: even own chunks; 4, 5: odd own chunks) ===============================================
-        // thread = output row t (TMEM lane t): scale, row normaliser -> swizzled staging -> TMA store (per warp: 32 rows)
+        // =========================================== output warps ======================================================
+        // thread = output row t (TMEM lane t): scale, row normaliser -> swizzled staging -> TMA store (per warp: 32 rows).
+        // Warps 0,1 take the even own chunks (buffer 0), warps 4,5 the odd ones (buffer 1).
         const int r = tid & 63, buf = warp >> 2, half = warp & 1;
         const uint32_t tmem_warp = tmem + ((uint32_t)(half * 32) << 16);
-        TDECL;
         for (int oi = buf; oi < n_own; oi += 2) {
             const int j = g + oi * stride;
-            const bool ok = __all_sync(0xffffffffu, TW(0, pwait(bar_o + 8 * buf, (oi >> 1) & 1)));
-            if (!ok) { if (lane == 0 && !*abort_flag) give_up(41, j); break; }
+            if (!__all_sync(0xffffffffu, pwait(bar_o + 8 * buf, (oi >> 1) & 1, 24))) { if (lane == 0) give_up(24, j); break; }
             tc_fence_after();
             float acc[kD];
             tmem_ld32(tmem_warp + kColOS + 64 * buf, *reinterpret_cast<float(*)[32]>(&acc[0]));
@@ -525,11 +467,13 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             }
         }
         if (lane == 0) bulk_wait0();   // output boxes fully written before the CTA retires
-        if (warp == 0) TDUMP(4);
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, tmem_cols);
+#ifdef PIPE_TIMING
+    if (blockIdx.x == 0 && tid < 32) reinterpret_cast<unsigned long long *>(status)[8 + tid] = probe[tid];
+#endif
 }
 
 // [B, L, H, 64] viewed as a rank-5 tensor (d, H, L, B, 1); box = (128 bytes of d) x 1 x rows x 1 x 1, 128-byte swizzle.
@@ -544,7 +488,7 @@ bool make_map(CUtensorMap *map, const void *ptr, int B, int H, int L, int rows, 
     return make_map_sw128(map, ptr, f32, 5, dims, strides, box);
 }
 
-template <typename TOut, bool kShared>   // kShared: stride > 1
+template <typename TOut, bool kShared>
 chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, int B, int H, int L, int stride, int norm, float eps,
                         float scale, int *status, const float *state_in, float *state_out, cudaStream_t stream)
 {
@@ -552,8 +496,8 @@ chela_status_t launch_t(const void *q, const void *k, const void *v, void *o, in
     if (!make_map(&mq, q, B, H, L, kC, false) || !make_map(&mk, k, B, H, L, kC, false) || !make_map(&mv, v, B, H, L, kC, false) ||
         !make_map(&mo, o, B, H, L, 32, sizeof(TOut) == 4))
         return CHELA_ERR_CUDA;
-    auto kern = kShared ? linattn_sm100_pipe_kernel<TOut, 7, 4> : linattn_sm100_pipe_kernel<TOut, 6, 6>;
-    constexpr int smem = kShared ? SmemP<TOut, 7, 4>::bytes : SmemP<TOut, 6, 6>::bytes;
+    auto kern = linattn_sm100_pipe_kernel<TOut, kShared>;
+    constexpr int smem = SmemP<TOut, kShared>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
     kern<<<B * H * stride, kThreads, smem, stream>>>(mq, mk, mv, mo, H, L, scale, norm, eps, status, stride, state_in, state_out,
                                                       current_wait_ctl());
