@@ -37,27 +37,28 @@ constexpr int kTile = kC * 128;   // one 64-row x 128-byte tile
 constexpr int kThreads = 512;
 constexpr int kWarpA = 8, kWarpG2 = 9, kWarpRun = 12, kWarpProducer = 13;
 
-// kShared: stride > 1.  Ring depths: kKV stages of [V | K] (16 KB each) and kQ stages of Q (8 KB each).  The producer
-// loads a chunk's Q with its K and V, so with one CTA per sequence the Q ring is as deep as the K, V ring (6 + 6); a CTA
-// that owns every second to fourth chunk needs fewer Q stages and gets one more K, V stage (7 + 4).
+// kShared: stride > 1.  Ring depths: kKV stages of [V | K] (16 KB each) and kQ stages of Q (8 KB each).  A stage is
+// held from the issue of its load until the last product that reads it has completed: for K and V the memory latency
+// (about 3000 cycles under load) plus the way to G3 (2400), for Q plus the way to G2 (3600); the rings carry
+// stages / hold time chunks per cycle, which is what bounds the kernel once HBM does not.
 template <typename TOut, bool kShared>
 struct SmemP {
-    static constexpr int kKV = kShared ? 7 : 6, kQ = kShared ? 4 : 6;
-    static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output staged as 128-byte wide boxes
+    static constexpr int kKV = 7, kQ = 6;
+    static constexpr int kOBoxes = (int)sizeof(TOut) * kD / 128;   // output leaves as 128-byte wide boxes, one at a time per warp
     static constexpr int offPT = 0;                               // masked scores, transposed (rows = s), two buffers
     static constexpr int offS = offPT + 2 * kTile;                // state tiles: [buffer][hi, lo], rows = d_k
     static constexpr int offKV = offS + 4 * kTile;                // after the score tiles: the G3 descriptor reaches K from P forwards
     static constexpr int offQ = offKV + kKV * 2 * kTile;
-    static constexpr int offO = offQ + kQ * kTile;                // output staging, two buffers; also what G2's 128-row operand reads past Q
-    static constexpr int offBar = offO + 2 * kOBoxes * kTile;
-    static constexpr int nBar = 2 * kKV + 2 * kQ + 2 * 8 + 3;
+    static constexpr int offO = offQ + kQ * kTile;                // output staging, one tile per set of output warps; also what G2's 128-row operand reads past Q
+    static constexpr int offBar = offO + 2 * kTile;
+    static constexpr int nBar = 2 * kKV + 2 * kQ + 2 * 9 + 5;
     static constexpr int offTmem = offBar + 8 * nBar;
     static constexpr int offAbort = offTmem + 8;
     static constexpr int offProbe = offAbort + 8;                 // wait-time counters of a timing build
     static constexpr int bytes = offProbe + 8 * 32;
 };
 // TMEM columns: PT[2] at 0, 64; OS[2] at 128, 192; DS[2] at 256, 320 (kShared only)
-constexpr int kColPT = 0, kColOS = 128, kColDS = 256;
+constexpr int kColPT = 0, kColOS = 128, kColDS = 384;   // PT 2 x 64, OS 2 x 128 (Q S_hi + P V | Q S_lo), DS 2 x 64
 
 // The spin of a bounded wait, out of line: the roles run long straight-line code and every inlined spin loop is
 // instruction-cache footprint they pay for (inlined: 0.54 ms at L = 32K, out of line: 0.43 ms).
@@ -76,6 +77,11 @@ __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const vola
     return ok;
 }
 
+#ifdef PIPE_TRACE   // timestamps of CTA 0's hand-offs into the workspace past its header: trace[event][chunk]
+#define TRACE(ev, idx) do { if (blockIdx.x == PIPE_TRACE && (threadIdx.x & 31) == 0 && (idx) < 2048) reinterpret_cast<long long *>(status)[64 + (ev) * 2048 + (idx)] = clock64(); } while (0)
+#else
+#define TRACE(ev, idx)
+#endif
 #define PDIAG(site, extra) do { if (atomicCAS(status + 8, 0, 7000 + (site)) == 0) { status[9] = blockIdx.x; status[10] = (extra); status[11] = gridDim.x; } } while (0)
 
 template <typename TOut, bool kShared>
@@ -102,22 +108,22 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const int n_own = g < nch_total ? (nch_total - 1 - g) / stride + 1 : 0;
     const int nchunks = n_own ? g + (n_own - 1) * stride + 1 : 0;
     const bool have_state = state_in != nullptr;
-    constexpr uint32_t tmem_cols = kShared ? 512u : 256u;
+    constexpr uint32_t tmem_cols = 512u;
 
     // ---- barriers -------------------------------------------------------------------------------------------------
     const uint32_t bar_kv_full = sbase + SM::offBar;                 // [kKV] K, V of a chunk have landed
     const uint32_t bar_kv_empty = bar_kv_full + 8 * kKV;             // [kKV] every product that reads the stage has completed
-    const uint32_t bar_q_full = bar_kv_empty + 8 * kKV;              // [kQ]
-    const uint32_t bar_q_empty = bar_q_full + 8 * kQ;                // [kQ]
+    const uint32_t bar_q_empty = bar_kv_empty + 8 * kKV;             // [kQ] G2 has read the stage
     const uint32_t bar_p = bar_q_empty + 8 * kQ;                     // [2] G1 completed (tensor core -> score warps)
-    const uint32_t bar_pt = bar_p + 16;                              // [2] score tile in shared memory (score warps -> issuer)
+    const uint32_t bar_pt = bar_p + 16;                              // [2] PT buffer read by the score warps (-> G1 issuer)
     const uint32_t bar_ds = bar_pt + 16;                             // [2] G3 completed (-> state warps, G2 issuer, score warps)
     const uint32_t bar_o = bar_ds + 16;                              // [2] G2 completed (-> output warps, state warps)
     const uint32_t bar_of = bar_o + 16;                              // [2] OS buffer read by output and state warps (-> issuer)
     const uint32_t bar_s = bar_of + 16;                              // [2] state tiles written (state warps -> G2 issuer)
     const uint32_t bar_dn = bar_s + 16;                              // [2] K^T V of a run of chunks that are not owned completed (-> state warps)
     const uint32_t bar_df = bar_dn + 16;                             // [2] DS buffer read (state warps -> run issuer)
-    const uint32_t bar_fin = bar_df + 16;                            // [3] every product an issuer has issued has completed (exit path)
+    const uint32_t bar_tile = bar_df + 16;                           // [2] score tile in shared memory (both score warps of a set -> the one that issues G3)
+    const uint32_t bar_fin = bar_tile + 16;                            // [3] every product an issuer has issued has completed (exit path)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
     unsigned long long *probe = reinterpret_cast<unsigned long long *>(smem + SM::offProbe);
@@ -128,7 +134,6 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             mbar_init(bar_kv_empty + 8 * s, 1);
         }
         for (int s = 0; s < kQ; ++s) {
-            mbar_init(bar_q_full + 8 * s, 1);
             mbar_init(bar_q_empty + 8 * s, 1);
         }
         for (int s = 0; s < 2; ++s) {
@@ -140,8 +145,9 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             mbar_init(bar_s + 8 * s, 4);
             mbar_init(bar_dn + 8 * s, 1);
             mbar_init(bar_df + 8 * s, 4);
+            mbar_init(bar_tile + 8 * s, 2);
         }
-        for (int s = 0; s < 3; ++s) mbar_init(bar_fin + 8 * s, 1);
+        for (int s = 0; s < 5; ++s) mbar_init(bar_fin + 8 * s, 1);
         *abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tm_q);
@@ -165,6 +171,12 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     auto pwait = [&](uint32_t bar, uint32_t parity, int site) {
         return mbar_try_wait(bar, parity) || wait_slow(bar, parity, abort_flag, wc.limit, probe + site);
     };
+    // two waits at once: the polls are issued back to back, so their latencies overlap (a lone issuing thread pays every
+    // instruction's latency in full)
+    auto pwait2 = [&](uint32_t bar_a, uint32_t par_a, int site_a, uint32_t bar_b, uint32_t par_b, int site_b) {
+        const bool a = mbar_try_wait(bar_a, par_a), b = mbar_try_wait(bar_b, par_b);
+        return (a || wait_slow(bar_a, par_a, abort_flag, wc.limit, probe + site_a)) && (b || wait_slow(bar_b, par_b, abort_flag, wc.limit, probe + site_b));
+    };
     auto kv_stage = [&](int chunk) { return sbase + SM::offKV + (chunk % kKV) * 2 * kTile; };   // V tile, then K tile
     auto q_stage = [&](int oi) { return sbase + SM::offQ + (oi % kQ) * kTile; };
     auto give_up = [&](int site, int extra) {
@@ -184,12 +196,13 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 if (j >= kKV && !(ok = pwait(bar_kv_empty + 8 * s, (j / kKV - 1) & 1, 1))) { give_up(1, j); break; }
                 const bool mine = j == next_own;
                 if (mine && oi >= kQ && !(ok = pwait(bar_q_empty + 8 * (oi % kQ), (oi / kQ - 1) & 1, 2))) { give_up(2, j); break; }
-                mbar_expect_tx(bar_kv_full + 8 * s, 2 * kTile);
+                TRACE(0, j);
+                // one barrier per chunk: K, V and (own chunks) Q
+                mbar_expect_tx(bar_kv_full + 8 * s, (mine ? 3 : 2) * kTile);
                 tma_load_5d(kv_stage(j), &tm_v, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
                 tma_load_5d(kv_stage(j) + kTile, &tm_k, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
                 if (mine) {
-                    mbar_expect_tx(bar_q_full + 8 * (oi % kQ), kTile);
-                    tma_load_5d(q_stage(oi), &tm_q, bar_q_full + 8 * (oi % kQ), 0, h, j * kC, b, 0);
+                    tma_load_5d(q_stage(oi), &tm_q, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
                     ++oi;
                     next_own += stride;
                 }
@@ -199,71 +212,50 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 // drain: every load that was issued lands before the CTA retires (a phase already consumed reads as complete)
                 for (int j = issued > kKV ? issued - kKV : 0; j < issued; ++j)
                     mbar_wait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, nullptr, wc.limit);
-                for (int q = oi > kQ ? oi - kQ : 0; q < oi; ++q) mbar_wait(bar_q_full + 8 * (q % kQ), (q / kQ) & 1, nullptr, wc.limit);
             }
         }
     } else if (warp == kWarpA) {
-        // =========================================== issuer of G1 and G3 ================================================
+        // =========================================== issuer of G1: PT[oi & 1] = [V;K] Q^T ==============================
         if (lane == 0) {
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [V;K] (K-major) x Q^T (K-major)
-            constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
             bool ok = true;
-            // G1 of own chunk number oi (chunk j): PT[oi & 1] = [V;K] Q^T.  The score warps have taken own chunk oi - 2 out of
-            // that buffer: this thread has waited for their tile (bar_pt) before it issued G3 of that chunk.
-            auto issue_scores = [&](int oi, int j) -> bool {
-                if (!pwait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, 3)) { give_up(3, j); return false; }
-                if (!pwait(bar_q_full + 8 * (oi % kQ), (oi / kQ) & 1, 4)) { give_up(4, j); return false; }
+            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
+                const int buf = oi & 1;
+                // the chunk's K, V and Q have landed; the score warps have taken own chunk oi - 2 out of PT[buf]
+                ok = oi >= 2 ? pwait2(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, 3, bar_pt + 8 * buf, ((oi >> 1) - 1) & 1, 5)
+                             : pwait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, 3);
+                if (!ok) { give_up(3, j); break; }
+                TRACE(1, oi);
                 tc_fence_after();
                 const uint32_t vk_lo = desc_lo(kv_stage(j)), q_lo = desc_lo(q_stage(oi));
 #pragma unroll
-                for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT + 64 * (oi & 1), vk_lo + 2 * k, q_lo + 2 * k, idescG1, k > 0);
-                umma_commit(bar_p + 8 * (oi & 1));
-                return true;
-            };
-            if (n_own > 0) ok = issue_scores(0, g);
-            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
-                const int buf = oi & 1;
-                const uint32_t ph = (oi >> 1) & 1;
-                // G1 of the next own chunk first: its score tile is ready long before its G3 is due
-                if (oi + 1 < n_own && !(ok = issue_scores(oi + 1, j + stride))) break;
-                // ---- G3: OS[buf] = [P^T | K]^T V (fresh) ----------------------------------------------------------------
-                if (!(ok = pwait(bar_pt + 8 * buf, ph, 5))) { give_up(5, j); break; }
-                // output and state warps have taken own chunk oi - 2 out of OS[buf]
-                if (oi >= 2 && !(ok = pwait(bar_of + 8 * buf, ph ^ 1, 6))) { give_up(6, j); break; }
-                tc_fence_after();
-                const uint32_t st = kv_stage(j), pt = sbase + SM::offPT + buf * kTile;
-                const uint32_t a_lo = desc_lo(pt, st + kTile - pt), v_lo = desc_lo(st);
-#pragma unroll
-                for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS + 64 * buf, a_lo + 128 * k, v_lo + 128 * k, idescG3, k > 0);
-                umma_commit(bar_ds + 8 * buf);
-                umma_commit(bar_kv_empty + 8 * (j % kKV));   // K and V are read by G1 and G3 only
+                for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT + 64 * buf, vk_lo + 2 * k, q_lo + 2 * k, idescG1, k > 0);
+                umma_commit(bar_p + 8 * buf);
             }
             umma_commit(bar_fin);   // every product issued by this thread has completed before TMEM and shared memory go away
             pwait(bar_fin, 0, 7);
         }
     } else if (warp == kWarpG2) {
-        // =========================================== issuer of G2: rows 0..63 of OS[buf] += Q S_hi + Q S_lo ==========
-        // (one thread for both terms: the order of the accumulation, and with it the last bit of the result, is fixed)
+        // =========================================== issuer of G2: rows 0..63 of OS[buf] += Q [S_hi | S_lo] ==========
         if (lane == 0) {
-            constexpr uint32_t idescG2 = make_idesc(128, kD, 0, 1);   // [Q;..] (K-major) x S (MN-major)
+            constexpr uint32_t idescG2 = make_idesc(128, 2 * kD, 0, 1);   // [Q;..] (K-major) x [S_hi | S_lo] (MN-major)
             bool ok = true;
             for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
                 const int buf = oi & 1;
                 const uint32_t ph = (oi >> 1) & 1;
                 // after G3 of the same chunk (same accumulator), with the state tiles as of the previous chunk (the state
                 // warps arrive for every own chunk, also when there is nothing to add)
-                if (!(ok = pwait(bar_ds + 8 * buf, ph, 8))) { give_up(8, j); break; }
-                if (!(ok = pwait(bar_s + 8 * buf, ph, 9))) { give_up(9, j); break; }
+                if (!(ok = pwait2(bar_ds + 8 * buf, ph, 8, bar_s + 8 * buf, ph, 9))) { give_up(8, j); break; }
+                TRACE(6, oi);
                 if (j > 0 || have_state) {
-                    // long complete: makes the copy visible to this thread
-                    if (!(ok = pwait(bar_q_full + 8 * (oi % kQ), (oi / kQ) & 1, 10))) { give_up(10, j); break; }
+                    // Q's copy completed long ago (G1 has used it); this thread has not observed its barrier, the
+                    // product that it issues follows the completed G1 and G3 of the chunk in the tensor core's order
                     tc_fence_after();
-                    const uint32_t q_lo = desc_lo(q_stage(oi));
-                    const uint32_t shi_lo = desc_lo(sbase + SM::offS + buf * 2 * kTile), slo_lo = desc_lo(sbase + SM::offS + (buf * 2 + 1) * kTile);
+                    // B = [S_hi | S_lo]: two 64-column atoms, MN-major, one tile apart; columns 0..63 of OS[buf] take Q S_hi on top of
+                    // P V, columns 64..127 take Q S_lo on top of the zeros the output warps left there
+                    const uint32_t q_lo = desc_lo(q_stage(oi)), s_lo = desc_lo(sbase + SM::offS + buf * 2 * kTile, kTile);
 #pragma unroll
-                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS + 64 * buf, q_lo + 2 * k, shi_lo + 128 * k, idescG2, 1, 1);
-#pragma unroll
-                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS + 64 * buf, q_lo + 2 * k, slo_lo + 128 * k, idescG2, 1, 1);
+                    for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS + 128 * buf, q_lo + 2 * k, s_lo + 128 * k, idescG2, 1, 1);
                 }
                 umma_commit(bar_o + 8 * buf);
                 umma_commit(bar_q_empty + 8 * (oi % kQ));
@@ -284,6 +276,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 if (ri >= 2 && !(ok = pwait(bar_df + 8 * (ri & 1), ((ri >> 1) - 1) & 1, 12))) { give_up(12, first); break; }
                 for (int c = first; ok && c <= last; ++c) {
                     if (!(ok = pwait(bar_kv_full + 8 * (c % kKV), (c / kKV) & 1, 13))) { give_up(13, c); break; }
+                    TRACE(7, ri);
                     tc_fence_after();
                     const uint32_t st = kv_stage(c);
                     const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st);
@@ -294,6 +287,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 }
                 if (!ok) break;
                 umma_commit(bar_dn + 8 * (ri & 1));
+                TRACE(8, ri);
                 ++ri;
             }
             umma_commit(bar_fin + 16);
@@ -308,13 +302,17 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         const uint32_t tmem_warp = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         for (int oi = buf; oi < n_own; oi += 2) {
             if (!__all_sync(0xffffffffu, pwait(bar_p + 8 * buf, (oi >> 1) & 1, 16))) { if (lane == 0) give_up(16, oi); break; }
+            if ((warp & 1) == 0) TRACE(9, oi);
             tc_fence_after();
             // rows s >= 32 have nothing at t < 32: all-zero blocks are not read from TMEM
             float p[2][32];
             if (low) tmem_ld32(tmem_warp + kColPT + 64 * buf, p[0]);
             tmem_ld32(tmem_warp + kColPT + 64 * buf + 32, p[1]);
             tmem_ld_wait();
-            // G3 of own chunk oi - 2 (another thread's product) has finished reading this score tile
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0 && !(wc.skip_arrival && blockIdx.x == 0 && oi == 0)) mbar_arrive(bar_pt + 8 * buf);   // PT[buf] is free (test hook: one arrival left out)
+            // G3 of own chunk oi - 2 has finished reading this score tile
             if (oi >= 2 && !__all_sync(0xffffffffu, pwait(bar_ds + 8 * buf, ((oi >> 1) - 1) & 1, 17))) { if (lane == 0) give_up(17, oi); break; }
             uint8_t *sP = smem + SM::offPT + buf * kTile;
 #pragma unroll
@@ -334,9 +332,30 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 }
             }
             fence_proxy_async();
-            tc_fence_before();
             __syncwarp();
-            if (lane == 0 && !(wc.skip_arrival && blockIdx.x == 0 && oi == 0)) mbar_arrive(bar_pt + 8 * buf);   // test hook: one arrival left out
+            if (lane == 0) mbar_arrive(bar_tile + 8 * buf);
+            // once both warps of the set have written their half of the tile, one thread issues G3, OS[buf] = [P^T | K]^T V
+            // (fresh); output and state warps have taken own chunk oi - 2 out of OS[buf] (they arrive once at the start, too)
+            if (low && lane == 0) {
+                constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
+                const int j = g + oi * stride;
+                if (!pwait2(bar_tile + 8 * buf, (oi >> 1) & 1, 5, bar_of + 8 * buf, (oi >> 1) & 1, 6)) {
+                    give_up(6, j);
+                    break;
+                }
+                TRACE(4, oi);
+                tc_fence_after();
+                const uint32_t st = kv_stage(j), pt = sbase + SM::offPT + buf * kTile;
+                const uint32_t a_lo = desc_lo(pt, st + kTile - pt), v_lo = desc_lo(st);
+#pragma unroll
+                for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS + 128 * buf, a_lo + 128 * k, v_lo + 128 * k, idescG3, k > 0);
+                umma_commit(bar_ds + 8 * buf);
+                umma_commit(bar_kv_empty + 8 * (j % kKV));   // K and V are read by G1 and G3 only
+            }
+        }
+        if (low && lane == 0) {   // every product issued by this thread has completed before TMEM and shared memory go away
+            umma_commit(bar_fin + 24 + 8 * buf);
+            pwait(bar_fin + 24 + 8 * buf, 0, 15);
         }
     } else if (warp == 10 || warp == 11 || warp == 14 || warp == 15) {
         // =========================================== state warps =======================================================
@@ -366,6 +385,10 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         };
         bool ok = true;
         int ri = 0;
+        if (lane == 0) {   // both accumulators start free
+            mbar_arrive(bar_of);
+            mbar_arrive(bar_of + 8);
+        }
         for (int oi = 0; oi < n_own; ++oi) {
             const int j = g + oi * stride, buf = oi & 1;
             // 1. the chunks since the previous own one (or since the start) belong to other CTAs: add their K^T V
@@ -381,6 +404,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             // 2. sv = S_{j-1}: bf16 hi + lo tiles (MN-major B operand of G2_j); the buffer was last read by G2 of own chunk oi - 2
             if (j > 0 || have_state) {
                 if (oi >= 2 && !(ok = __all_sync(0xffffffffu, pwait(bar_o + 8 * buf, ((oi >> 1) - 1) & 1, 21)))) { if (lane == 0) give_up(21, j); break; }
+                if (warp == 10) TRACE(16, oi);
                 uint8_t *sHi = smem + SM::offS + buf * 2 * kTile, *sLo = sHi + kTile;
 #pragma unroll
                 for (int c8 = 0; c8 < kCols / 8; ++c8) {
@@ -395,19 +419,25 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     }
                     const uint32_t off = sw128(r, c0 / 8 + c8);
                     *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+#ifndef PIPE_EXP_NOLO
                     *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+#endif
                 }
+                if (warp == 10) TRACE(17, oi);
                 fence_proxy_async();
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s + 8 * buf);   // also when there is nothing to write (first chunk, no initial state)
+            if (warp == 10) TRACE(11, oi);
             // 3. the own chunk's K^T V (rows 64..127 of OS[buf])
             if (!(ok = __all_sync(0xffffffffu, pwait(bar_ds + 8 * buf, (oi >> 1) & 1, 22)))) { if (lane == 0) give_up(22, j); break; }
             tc_fence_after();
-            add_tmem(kColOS + 64 * buf);
+            if (warp == 10) TRACE(12, oi);
+            add_tmem(kColOS + 128 * buf);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_of + 8 * buf);
+            if (warp == 10) TRACE(13, oi);
         }
         if (ok && state_out && nchunks == nch_total) {
             // this CTA owns the last chunk of the sequence: the fp32 state leaves the SM once, for the caller
@@ -421,21 +451,38 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         // Warps 0,1 take the even own chunks (buffer 0), warps 4,5 the odd ones (buffer 1).
         const int r = tid & 63, buf = warp >> 2, half = warp & 1;
         const uint32_t tmem_warp = tmem + ((uint32_t)(half * 32) << 16);
+        auto zero_lo = [&]() {   // columns 64..127 of this thread's row of OS[buf] = 0
+            float z[32];
+#pragma unroll
+            for (int c = 0; c < 32; ++c) z[c] = 0.f;
+            tmem_st32(tmem_warp + kColOS + 128 * buf + 64, z);
+            tmem_st32(tmem_warp + kColOS + 128 * buf + 96, z);
+            tmem_st_wait();
+        };
+        zero_lo();   // OS[buf] starts free and with a zero lo half
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_of + 8 * buf);
         for (int oi = buf; oi < n_own; oi += 2) {
             const int j = g + oi * stride;
             if (!__all_sync(0xffffffffu, pwait(bar_o + 8 * buf, (oi >> 1) & 1, 24))) { if (lane == 0) give_up(24, j); break; }
+            if (half == 0) TRACE(14, oi);
             tc_fence_after();
+            // columns 0..63: Q S_hi + P V, columns 64..127: Q S_lo; the latter are zeroed again for the chunk after next
             float acc[kD];
-            tmem_ld32(tmem_warp + kColOS + 64 * buf, *reinterpret_cast<float(*)[32]>(&acc[0]));
-            tmem_ld32(tmem_warp + kColOS + 64 * buf + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
-            tmem_ld_wait();
+#pragma unroll
+            for (int hc = 0; hc < 2; ++hc) {
+                float lo[32];
+                tmem_ld32(tmem_warp + kColOS + 128 * buf + 32 * hc, *reinterpret_cast<float(*)[32]>(&acc[32 * hc]));
+                tmem_ld32(tmem_warp + kColOS + 128 * buf + 64 + 32 * hc, lo);
+                tmem_ld_wait();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) acc[32 * hc + c] += lo[c];
+            }
+            zero_lo();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar_of + 8 * buf);   // the output rows are out of TMEM
-                bulk_wait_read0();               // the boxes this warp stored two chunks ago have left its staging buffer
-            }
-            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_of + 8 * buf);   // the output rows are out of TMEM
             float ss = 0.f;
 #pragma unroll
             for (int c = 0; c < kD; ++c) {
@@ -443,28 +490,32 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 ss = fmaf(acc[c], acc[c], ss);
             }
             const float inv = norm ? rsqrtf(ss * (1.0f / kD) + eps) : 1.0f;
-            uint8_t *sO = smem + SM::offO + buf * SM::kOBoxes * kTile;
-            if (sizeof(TOut) == 4) {
+            // this warp's 32 rows x 128 bytes of the set's staging tile, one 128-byte wide box after the other
+            uint8_t *sO = smem + SM::offO + buf * kTile;
 #pragma unroll
-                for (int c = 0; c < kD; c += 4)
-                    *reinterpret_cast<float4 *>(sO + (c / 32) * kTile + sw128(r, (c % 32) / 4)) =
-                        make_float4(acc[c] * inv, acc[c + 1] * inv, acc[c + 2] * inv, acc[c + 3] * inv);
-            } else {
+            for (int bx = 0; bx < SM::kOBoxes; ++bx) {
+                if (lane == 0) bulk_wait_read0();   // the box this warp stored last has left the staging tile
+                __syncwarp();
+                if (sizeof(TOut) == 4) {
 #pragma unroll
-                for (int c = 0; c < kD; c += 8)
-                    *reinterpret_cast<uint4 *>(sO + sw128(r, c / 8)) =
-                        make_uint4(pack_bf16(acc[c] * inv, acc[c + 1] * inv), pack_bf16(acc[c + 2] * inv, acc[c + 3] * inv),
-                                   pack_bf16(acc[c + 4] * inv, acc[c + 5] * inv), pack_bf16(acc[c + 6] * inv, acc[c + 7] * inv));
+                    for (int c = 0; c < 32; c += 4)
+                        *reinterpret_cast<float4 *>(sO + sw128(r, c / 4)) =
+                            make_float4(acc[32 * bx + c] * inv, acc[32 * bx + c + 1] * inv, acc[32 * bx + c + 2] * inv, acc[32 * bx + c + 3] * inv);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < kD; c += 8)
+                        *reinterpret_cast<uint4 *>(sO + sw128(r, c / 8)) =
+                            make_uint4(pack_bf16(acc[c] * inv, acc[c + 1] * inv), pack_bf16(acc[c + 2] * inv, acc[c + 3] * inv),
+                                       pack_bf16(acc[c + 4] * inv, acc[c + 5] * inv), pack_bf16(acc[c + 6] * inv, acc[c + 7] * inv));
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {   // rows past L are clipped by the copy engine
+                    tma_store_5d(&tm_o, sbase + SM::offO + buf * kTile + half * 32 * 128, bx * (128 / (int)sizeof(TOut)), h, j * kC + half * 32, b, 0);
+                    bulk_commit();
+                }
             }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) {   // rows past L are clipped by the copy engine
-#pragma unroll
-                for (int bx = 0; bx < SM::kOBoxes; ++bx)
-                    tma_store_5d(&tm_o, sbase + SM::offO + (buf * SM::kOBoxes + bx) * kTile + half * 32 * 128, bx * (128 / (int)sizeof(TOut)), h,
-                                 j * kC + half * 32, b, 0);
-                bulk_commit();
-            }
+            if (half == 0) TRACE(15, oi);
         }
         if (lane == 0) bulk_wait0();   // output boxes fully written before the CTA retires
     }
