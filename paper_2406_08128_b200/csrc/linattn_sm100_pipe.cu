@@ -25,6 +25,9 @@
 // Roles meet only through mbarriers, every wait bounded: on a timeout the CTA records CHELA_ERR_TIMEOUT, waits
 // (bounded) for its loads and products in flight, frees its TMEM and returns.
 #include "sm100_ptx.cuh"
+#ifdef PIPE_STRIDE_ENV
+#include <cstdlib>
+#endif
 
 namespace chela {
 namespace {
@@ -35,7 +38,7 @@ constexpr int kD = 64;            // head dimension (d_k = d_v)
 constexpr int kC = 64;            // tokens per chunk
 constexpr int kTile = kC * 128;   // one 64-row x 128-byte tile
 constexpr int kThreads = 512;
-constexpr int kWarpA = 8, kWarpG2 = 9, kWarpRun = 12, kWarpProducer = 13;
+constexpr int kWarpA = 8, kWarpG2 = 9, kWarpG3 = 12, kWarpProducer = 13;
 
 // kShared: stride > 1.  Ring depths: kKV stages of [V | K] (16 KB each) and kQ stages of Q (8 KB each).  A stage is
 // held from the issue of its load until the last product that reads it has completed: for K and V the memory latency
@@ -121,8 +124,8 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const uint32_t bar_of = bar_o + 16;                              // [2] OS buffer read by output and state warps (-> issuer)
     const uint32_t bar_s = bar_of + 16;                              // [2] state tiles written (state warps -> G2 issuer)
     const uint32_t bar_dn = bar_s + 16;                              // [2] K^T V of a run of chunks that are not owned completed (-> state warps)
-    const uint32_t bar_df = bar_dn + 16;                             // [2] DS buffer read (state warps -> run issuer)
-    const uint32_t bar_tile = bar_df + 16;                           // [2] score tile in shared memory (both score warps of a set -> the one that issues G3)
+    const uint32_t bar_d0 = bar_dn + 16;                             // K^T V of the chunks before the first own one completed (-> state warps)
+    const uint32_t bar_tile = bar_d0 + 8;                           // [2] score tile in shared memory (both score warps of a set -> the one that issues G3)
     const uint32_t bar_fin = bar_tile + 16;                            // [3] every product an issuer has issued has completed (exit path)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
@@ -138,16 +141,16 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar_p + 8 * s, 1);
-            mbar_init(bar_pt + 8 * s, 2);
+            mbar_init(bar_pt + 8 * s, 3);
             mbar_init(bar_ds + 8 * s, 1);
             mbar_init(bar_o + 8 * s, 1);
             mbar_init(bar_of + 8 * s, 6);
             mbar_init(bar_s + 8 * s, 4);
             mbar_init(bar_dn + 8 * s, 1);
-            mbar_init(bar_df + 8 * s, 4);
-            mbar_init(bar_tile + 8 * s, 2);
+            mbar_init(bar_tile + 8 * s, 3);
         }
-        for (int s = 0; s < 5; ++s) mbar_init(bar_fin + 8 * s, 1);
+        mbar_init(bar_d0, 1);
+        for (int s = 0; s < 3; ++s) mbar_init(bar_fin + 8 * s, 1);
         *abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tm_q);
@@ -263,99 +266,91 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             umma_commit(bar_fin + 8);
             pwait(bar_fin + 8, 0, 11);
         }
-    } else if (warp == kWarpRun) {
-        // =========================================== issuer of the K^T V of chunks that other CTAs own ================
-        if (kShared && lane == 0) {
+    } else if (warp == kWarpG3) {
+        // =========================================== issuer of G3 and of the K^T V of chunks that other CTAs own ========
+        if (lane == 0) {
             constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
             bool ok = true;
-            int ri = 0;   // runs issued so far
-            // runs: the chunks before the first own one, then those between consecutive own chunks; each -> rows 64..127
-            // of DS[ri & 1] (output lanes write-disabled), fresh for every run
-            for (int first = 0, last = g - 1; ok && last < nchunks; first = last + 2, last += stride) {
-                if (last < first) continue;   // g = 0: no chunks before the first own one
-                if (ri >= 2 && !(ok = pwait(bar_df + 8 * (ri & 1), ((ri >> 1) - 1) & 1, 12))) { give_up(12, first); break; }
-                for (int c = first; ok && c <= last; ++c) {
-                    if (!(ok = pwait(bar_kv_full + 8 * (c % kKV), (c / kKV) & 1, 13))) { give_up(13, c); break; }
-                    TRACE(7, ri);
-                    tc_fence_after();
-                    const uint32_t st = kv_stage(c);
-                    const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st);
+            // K^T V of chunk c summed onto rows 64..127 of the accumulator at column `col` (output lanes write-disabled)
+            auto issue_ktv = [&](int c, uint32_t col, bool fresh) -> bool {
+                if (!pwait(bar_kv_full + 8 * (c % kKV), (c / kKV) & 1, 13)) { give_up(13, c); return false; }
+                tc_fence_after();
+                const uint32_t st = kv_stage(c);
+                const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st);
 #pragma unroll
-                    for (int k = 0; k < kC / 16; ++k)
-                        umma_bf16(tmem + kColDS + 64 * (ri & 1), a_lo + 128 * k, v_lo + 128 * k, idescG3, (c > first || k > 0) ? 1u : 0u, 2);
-                    umma_commit(bar_kv_empty + 8 * (c % kKV));
-                }
-                if (!ok) break;
-                umma_commit(bar_dn + 8 * (ri & 1));
-                TRACE(8, ri);
-                ++ri;
+                for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + col, a_lo + 128 * k, v_lo + 128 * k, idescG3, (!fresh || k > 0) ? 1u : 0u, 2);
+                umma_commit(bar_kv_empty + 8 * (c % kKV));
+                return true;
+            };
+            if (kShared && n_own > 0 && g > 0) {
+                // the chunks before the first own one -> DS, read once by the state warps
+                for (int c = 0; ok && c < g; ++c) ok = issue_ktv(c, kColDS, c == 0);
+                if (ok) umma_commit(bar_d0);
             }
-            umma_commit(bar_fin + 16);
-            pwait(bar_fin + 16, 0, 14);
-        }
-    } else if (warp < 8 && (warp & 2)) {
-        // =========================================== score warps =======================================================
-        // thread = row s of P^T (TMEM lane 64 + s): causal mask (t >= s), bf16, swizzled tile with rows = s.
-        // Warps 2,3 take the even own chunks (buffer 0), warps 6,7 the odd ones (buffer 1).
-        const int r = tid & 63, buf = warp >> 2;
-        const bool low = (warp & 1) == 0;   // rows s < 32
-        const uint32_t tmem_warp = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        for (int oi = buf; oi < n_own; oi += 2) {
-            if (!__all_sync(0xffffffffu, pwait(bar_p + 8 * buf, (oi >> 1) & 1, 16))) { if (lane == 0) give_up(16, oi); break; }
-            if ((warp & 1) == 0) TRACE(9, oi);
-            tc_fence_after();
-            // rows s >= 32 have nothing at t < 32: all-zero blocks are not read from TMEM
-            float p[2][32];
-            if (low) tmem_ld32(tmem_warp + kColPT + 64 * buf, p[0]);
-            tmem_ld32(tmem_warp + kColPT + 64 * buf + 32, p[1]);
-            tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0 && !(wc.skip_arrival && blockIdx.x == 0 && oi == 0)) mbar_arrive(bar_pt + 8 * buf);   // PT[buf] is free (test hook: one arrival left out)
-            // G3 of own chunk oi - 2 has finished reading this score tile
-            if (oi >= 2 && !__all_sync(0xffffffffu, pwait(bar_ds + 8 * buf, ((oi >> 1) - 1) & 1, 17))) { if (lane == 0) give_up(17, oi); break; }
-            uint8_t *sP = smem + SM::offPT + buf * kTile;
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                const bool live = cb == 1 || low;
-#pragma unroll
-                for (int c8 = 0; c8 < 4; ++c8) {
-                    uint32_t w[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int t = cb * 32 + c8 * 8 + e * 2;
-                        const float x0 = (live && t >= r) ? p[cb][c8 * 8 + e * 2] : 0.f;
-                        const float x1 = (live && t + 1 >= r) ? p[cb][c8 * 8 + e * 2 + 1] : 0.f;
-                        w[e] = pack_bf16(x0, x1);
-                    }
-                    *reinterpret_cast<uint4 *>(sP + sw128(r, cb * 4 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
-                }
-            }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tile + 8 * buf);
-            // once both warps of the set have written their half of the tile, one thread issues G3, OS[buf] = [P^T | K]^T V
-            // (fresh); output and state warps have taken own chunk oi - 2 out of OS[buf] (they arrive once at the start, too)
-            if (low && lane == 0) {
-                constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
-                const int j = g + oi * stride;
-                if (!pwait2(bar_tile + 8 * buf, (oi >> 1) & 1, 5, bar_of + 8 * buf, (oi >> 1) & 1, 6)) {
-                    give_up(6, j);
-                    break;
-                }
+            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
+                const int buf = oi & 1;
+                const uint32_t ph = (oi >> 1) & 1;
+                // the score tile is in shared memory; output and state warps have taken own chunk oi - 2 out of OS[buf]
+                // (they arrive once at the start, too)
+                if (!(ok = pwait2(bar_tile + 8 * buf, ph, 5, bar_of + 8 * buf, ph, 6))) { give_up(6, j); break; }
                 TRACE(4, oi);
                 tc_fence_after();
                 const uint32_t st = kv_stage(j), pt = sbase + SM::offPT + buf * kTile;
                 const uint32_t a_lo = desc_lo(pt, st + kTile - pt), v_lo = desc_lo(st);
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS + 128 * buf, a_lo + 128 * k, v_lo + 128 * k, idescG3, k > 0);
-                umma_commit(bar_ds + 8 * buf);
                 umma_commit(bar_kv_empty + 8 * (j % kKV));   // K and V are read by G1 and G3 only
+                // strided: the chunks up to the next own one, onto the rows where G3 has just put this chunk's own K^T V (same
+                // thread, so in this order), and the state warps read one sum per own chunk
+                if (kShared)
+                    for (int c = j + 1; ok && c < j + stride && c < nchunks; ++c) ok = issue_ktv(c, kColOS + 128 * buf, false);
+                umma_commit(bar_ds + 8 * buf);
             }
+            umma_commit(bar_fin + 16);
+            pwait(bar_fin + 16, 0, 14);
         }
-        if (low && lane == 0) {   // every product issued by this thread has completed before TMEM and shared memory go away
-            umma_commit(bar_fin + 24 + 8 * buf);
-            pwait(bar_fin + 24 + 8 * buf, 0, 15);
+    } else if (warp == 2 || warp == 3 || warp == 6) {
+        // =========================================== score warps =======================================================
+        // thread = row s of P^T (TMEM lane 64 + s) x 32 columns t: causal mask (t >= s), bf16, swizzled tile with rows = s.
+        // Warp 2: rows 0..31, t 0..31 (triangle); warp 6: rows 0..31, t 32..63 (full); warp 3: rows 32..63, t 32..63
+        // (triangle).  Rows 32..63, t 0..31 are zero in every chunk: written once.
+        const int r = (warp & 1) * 32 + lane, t0 = warp == 2 ? 0 : 32;
+        const bool full = warp == 6;
+        const uint32_t tmem_warp = tmem + ((uint32_t)((warp & 3) * 32) << 16) + t0;
+        if (warp == 3)
+            for (int bufz = 0; bufz < 2; ++bufz)
+#pragma unroll
+                for (int c8 = 0; c8 < 4; ++c8) *reinterpret_cast<uint4 *>(smem + SM::offPT + bufz * kTile + sw128(r, c8)) = make_uint4(0, 0, 0, 0);
+        for (int oi = 0; oi < n_own; ++oi) {
+            const int buf = oi & 1;
+            if (!__all_sync(0xffffffffu, pwait(bar_p + 8 * buf, (oi >> 1) & 1, 16))) { if (lane == 0) give_up(16, oi); break; }
+            if (warp == 2) TRACE(9, oi);
+            tc_fence_after();
+            float p[32];
+            tmem_ld32(tmem_warp + kColPT + 64 * buf, p);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0 && !(wc.skip_arrival && blockIdx.x == 0 && oi == 0 && warp == 2)) mbar_arrive(bar_pt + 8 * buf);   // PT[buf] is free (test hook: one arrival left out)
+            // G3 of own chunk oi - 2 has finished reading this score tile
+            if (oi >= 2 && !__all_sync(0xffffffffu, pwait(bar_ds + 8 * buf, ((oi >> 1) - 1) & 1, 17))) { if (lane == 0) give_up(17, oi); break; }
+            uint8_t *sP = smem + SM::offPT + buf * kTile;
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int t = t0 + c8 * 8 + e * 2;
+                    const float x0 = (full || t >= r) ? p[c8 * 8 + e * 2] : 0.f;
+                    const float x1 = (full || t + 1 >= r) ? p[c8 * 8 + e * 2 + 1] : 0.f;
+                    w[e] = pack_bf16(x0, x1);
+                }
+                *reinterpret_cast<uint4 *>(sP + sw128(r, t0 / 8 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tile + 8 * buf);
+            if (warp == 2) TRACE(10, oi);
         }
     } else if (warp == 10 || warp == 11 || warp == 14 || warp == 15) {
         // =========================================== state warps =======================================================
@@ -384,24 +379,21 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             for (int j = 0; j < kCols; ++j) sv[j] += t[j];
         };
         bool ok = true;
-        int ri = 0;
         if (lane == 0) {   // both accumulators start free
             mbar_arrive(bar_of);
             mbar_arrive(bar_of + 8);
         }
-        for (int oi = 0; oi < n_own; ++oi) {
-            const int j = g + oi * stride, buf = oi & 1;
-            // 1. the chunks since the previous own one (or since the start) belong to other CTAs: add their K^T V
-            if (kShared && j > 0) {
-                if (!(ok = __all_sync(0xffffffffu, pwait(bar_dn + 8 * (ri & 1), (ri >> 1) & 1, 20)))) { if (lane == 0) give_up(20, j); break; }
+        if (kShared && g > 0 && n_own > 0) {
+            // the chunks before the first own one belong to other CTAs: their K^T V, summed in DS
+            if (!(ok = __all_sync(0xffffffffu, pwait(bar_d0, 0, 20)))) { if (lane == 0) give_up(20, 0); }
+            if (ok) {
                 tc_fence_after();
-                add_tmem(kColDS + 64 * (ri & 1));
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_df + 8 * (ri & 1));
-                ++ri;
+                add_tmem(kColDS);
             }
-            // 2. sv = S_{j-1}: bf16 hi + lo tiles (MN-major B operand of G2_j); the buffer was last read by G2 of own chunk oi - 2
+        }
+        for (int oi = 0; ok && oi < n_own; ++oi) {
+            const int j = g + oi * stride, buf = oi & 1;
+            // 1. sv = S_{j-1}: bf16 hi + lo tiles (MN-major B operand of G2_j); the buffer was last read by G2 of own chunk oi - 2
             if (j > 0 || have_state) {
                 if (oi >= 2 && !(ok = __all_sync(0xffffffffu, pwait(bar_o + 8 * buf, ((oi >> 1) - 1) & 1, 21)))) { if (lane == 0) give_up(21, j); break; }
                 if (warp == 10) TRACE(16, oi);
@@ -429,7 +421,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s + 8 * buf);   // also when there is nothing to write (first chunk, no initial state)
             if (warp == 10) TRACE(11, oi);
-            // 3. the own chunk's K^T V (rows 64..127 of OS[buf])
+            // 2. rows 64..127 of OS[buf]: the chunk's K^T V, plus (strided) that of the chunks up to the next own one
             if (!(ok = __all_sync(0xffffffffu, pwait(bar_ds + 8 * buf, (oi >> 1) & 1, 22)))) { if (lane == 0) give_up(22, j); break; }
             tc_fence_after();
             if (warp == 10) TRACE(12, oi);
@@ -445,7 +437,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
 #pragma unroll
             for (int j = 0; j < kCols / 4; ++j) dst[j] = make_float4(sv[4 * j], sv[4 * j + 1], sv[4 * j + 2], sv[4 * j + 3]);
         }
-    } else if (warp < 8) {
+    } else if (warp == 0 || warp == 1 || warp == 4 || warp == 5) {
         // =========================================== output warps ======================================================
         // thread = output row t (TMEM lane t): scale, row normaliser -> swizzled staging -> TMA store (per warp: 32 rows).
         // Warps 0,1 take the even own chunks (buffer 0), warps 4,5 the odd ones (buffer 1).
@@ -572,6 +564,9 @@ int linattn_sm100_pipe_stride(int B, int H, int L, int sms)
     int stride = (int)(sms / bh);
     if (stride > 4) stride = 4;
     if (stride > nchunks / 4) stride = nchunks / 4;
+#ifdef PIPE_STRIDE_ENV
+    if (const char *e = getenv("CHELA_STRIDE_TMP")) stride = atoi(e);
+#endif
     return stride < 1 ? 1 : stride;
 }
 
