@@ -7,27 +7,28 @@
 // a lone CTA, hidden only by a second CTA on the SM.  Here the per-chunk products are independent of each other:
 //   G1_i : [V_i ; K_i] Q_i^T                  -> TMEM PT[i%2]; rows 64..127 are P^T = K_i Q_i^T
 //   G3_i : [P_i^T | K_i]^T V_i   (fresh)      -> TMEM OS[i%2]; rows 0..63 = P_i V_i, rows 64..127 = dS_i = K_i^T V_i
-//   G2_i : rows 0..63 of OS[i%2] += Q_i S_{i-1}   (S_{i-1} as bf16 hi + lo tiles in shared memory)
+//   G2_i : rows 0..63 of OS[i%2] += Q_i [S_hi | S_lo]   (S_{i-1} as bf16 hi and lo tiles in shared memory, one N = 128
+//          series: columns 0..63 take Q S_hi on top of P V, columns 64..127 take Q S_lo on top of zeros; the output warps
+//          add the halves)
 // and the recurrence S_i = S_{i-1} + dS_i is an fp32 add in the registers of the state warps, which write the hi/lo
-// tiles for the next chunk's G2.  G3_{i+1} and G1_{i+2} are issued before G2_{i+1}, so the tensor core always has work
-// while the state warps turn dS_i into tiles.  Accumulators, score tiles and state tiles are double-buffered.
+// tiles for the next chunk's G2.  G1 and G3 of later chunks do not wait for G2, so the tensor core has work while the
+// state warps turn dS_i into tiles.  Accumulators, score tiles and state tiles are double-buffered.
 //
 // Sequences are shared between CTAs by stride (B*H*stride <= SMs): CTA g of a sequence owns the chunks g, g + stride, ...
 // and produces their output rows.  The state needs every chunk, so for a chunk it does not own a CTA loads K and V only
-// and accumulates K^T V into a TMEM tile DS (output lanes write-disabled) that the state warps add to their registers
-// before the next own chunk.  The CTAs of a sequence read the same K, V tiles at about the same time, so all but the
-// first read are served by L2: HBM traffic stays the algorithmic Q + K + V + O, with no second kernel and no workspace.
+// and adds K^T V (output lanes write-disabled) onto the rows where G3 of the preceding own chunk has just put that
+// chunk's own K^T V (same issuing thread, so in that order): the state warps still read one sum per own chunk.  The CTAs
+// of a sequence read the same K, V tiles at about the same time, so all but the first read are served by L2: HBM
+// traffic stays the algorithmic Q + K + V + O (measured), with no second kernel and no workspace.
 //
-// Warps (16): 0,1,4,5 output rows (scale, normaliser, TMA store; 0,1 take the even own chunks, 4,5 the odd ones);
-// 2,3,6,7 score rows (mask, bf16, shared tile; same alternation); 10,11,14,15 state rows (two warps per half of the
-// columns); one issuing thread in each of: 8 (G1 and G3), 9 (G2), 12 (K^T V of chunks that are not owned), 13 (TMA
-// producer).  One thread issues a tcgen05.mma about every 50 cycles and a chunk has 16 of them, hence several issuers.
+// Warps (16): 0,1,4,5 output rows (add the halves, scale, normaliser, TMA store; 0,1 take the even own chunks, 4,5 the
+// odd ones); 8,9,12 score rows (mask, bf16, shared tile: a third of the live 64 x 64 triangle each); 10,11,14,15 state
+// rows (two warps per half of the columns); one issuing thread in each of 2 (G1), 3 (G2), 6 (G3 and the K^T V of chunks
+// that are not owned) and 7 (TMA producer).  A lone thread issues a tcgen05.mma about every 50 to 80 cycles and pays
+// the latency of every instruction between them, hence several issuers and no divisions in their loops.
 // Roles meet only through mbarriers, every wait bounded: on a timeout the CTA records CHELA_ERR_TIMEOUT, waits
 // (bounded) for its loads and products in flight, frees its TMEM and returns.
 #include "sm100_ptx.cuh"
-#ifdef PIPE_STRIDE_ENV
-#include <cstdlib>
-#endif
 
 namespace chela {
 namespace {
@@ -57,15 +58,14 @@ struct SmemP {
     static constexpr int nBar = 2 * kKV + 2 * kQ + 2 * 9 + 5;
     static constexpr int offTmem = offBar + 8 * nBar;
     static constexpr int offAbort = offTmem + 8;
-    static constexpr int offProbe = offAbort + 8;                 // wait-time counters of a timing build
-    static constexpr int bytes = offProbe + 8 * 32;
+    static constexpr int bytes = offAbort + 8;
 };
 // TMEM columns: PT[2] at 0, 64; OS[2] at 128, 192; DS[2] at 256, 320 (kShared only)
 constexpr int kColPT = 0, kColOS = 128, kColDS = 384;   // PT 2 x 64, OS 2 x 128 (Q S_hi + P V | Q S_lo), DS 2 x 64
 
 // The spin of a bounded wait, out of line: the roles run long straight-line code and every inlined spin loop is
 // instruction-cache footprint they pay for (inlined: 0.54 ms at L = 32K, out of line: 0.43 ms).
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const volatile int *abort_flag, long long limit, unsigned long long *probe)
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const volatile int *abort_flag, long long limit)
 {
     const long long t0 = clock64();
     bool ok = true;
@@ -74,17 +74,24 @@ __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const vola
             ok = false;
             break;
         }
-#ifdef PIPE_TIMING
-    atomicAdd(probe, (unsigned long long)(clock64() - t0));
-#endif
     return ok;
 }
 
-#ifdef PIPE_TRACE   // timestamps of CTA 0's hand-offs into the workspace past its header: trace[event][chunk]
-#define TRACE(ev, idx) do { if (blockIdx.x == PIPE_TRACE && (threadIdx.x & 31) == 0 && (idx) < 2048) reinterpret_cast<long long *>(status)[64 + (ev) * 2048 + (idx)] = clock64(); } while (0)
-#else
-#define TRACE(ev, idx)
-#endif
+// Position in a ring of n stages and the parity of its current pass, advanced without divisions (the issuing threads
+// run one lane at a time: every instruction of theirs is latency).
+struct Ring {
+    int s;
+    uint32_t ph;
+    __device__ void advance(int n, int by = 1)
+    {
+        s += by;
+        if (s >= n) {
+            s -= n;
+            ph ^= 1;
+        }
+    }
+};
+
 #define PDIAG(site, extra) do { if (atomicCAS(status + 8, 0, 7000 + (site)) == 0) { status[9] = blockIdx.x; status[10] = (extra); status[11] = gridDim.x; } } while (0)
 
 template <typename TOut, bool kShared>
@@ -129,7 +136,6 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const uint32_t bar_fin = bar_tile + 16;                            // [3] every product an issuer has issued has completed (exit path)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + SM::offTmem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + SM::offAbort);
-    unsigned long long *probe = reinterpret_cast<unsigned long long *>(smem + SM::offProbe);
 
     if (tid == 0) {
         for (int s = 0; s < kKV; ++s) {
@@ -158,9 +164,6 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         tma_prefetch_desc(&tm_v);
         tma_prefetch_desc(&tm_o);
     }
-#ifdef PIPE_TIMING
-    if (tid < 32) probe[tid] = 0;
-#endif
     if (warp == 0) {
         tmem_alloc(sbase + SM::offTmem, tmem_cols);
         tmem_relinquish();
@@ -170,18 +173,18 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    // `site` names the wait in the timing build's counters and, plus 7000, in the diagnostics of a wait that gave up
+    // `site` names the wait in the diagnostics of one that gave up (7000 + site)
     auto pwait = [&](uint32_t bar, uint32_t parity, int site) {
-        return mbar_try_wait(bar, parity) || wait_slow(bar, parity, abort_flag, wc.limit, probe + site);
+        return mbar_try_wait(bar, parity) || wait_slow(bar, parity, abort_flag, wc.limit);
     };
     // two waits at once: the polls are issued back to back, so their latencies overlap (a lone issuing thread pays every
     // instruction's latency in full)
     auto pwait2 = [&](uint32_t bar_a, uint32_t par_a, int site_a, uint32_t bar_b, uint32_t par_b, int site_b) {
         const bool a = mbar_try_wait(bar_a, par_a), b = mbar_try_wait(bar_b, par_b);
-        return (a || wait_slow(bar_a, par_a, abort_flag, wc.limit, probe + site_a)) && (b || wait_slow(bar_b, par_b, abort_flag, wc.limit, probe + site_b));
+        return (a || wait_slow(bar_a, par_a, abort_flag, wc.limit)) && (b || wait_slow(bar_b, par_b, abort_flag, wc.limit));
     };
-    auto kv_stage = [&](int chunk) { return sbase + SM::offKV + (chunk % kKV) * 2 * kTile; };   // V tile, then K tile
-    auto q_stage = [&](int oi) { return sbase + SM::offQ + (oi % kQ) * kTile; };
+    auto kv_stage = [&](int s) { return sbase + SM::offKV + s * 2 * kTile; };   // stage s of the ring: V tile, then K tile
+    auto q_stage = [&](int s) { return sbase + SM::offQ + s * kTile; };
     auto give_up = [&](int site, int extra) {
         if (*abort_flag) return;   // another role gave up first: its diagnostics stand
         PDIAG(site, extra);
@@ -193,19 +196,20 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         // =========================================== TMA producer ======================================================
         if (lane == 0) {
             int issued = 0, oi = 0, next_own = g;
+            Ring kv = {0, 0}, qr = {0, 0};
             bool ok = true;
-            for (int j = 0; ok && j < nchunks; ++j) {
-                const int s = j % kKV;
-                if (j >= kKV && !(ok = pwait(bar_kv_empty + 8 * s, (j / kKV - 1) & 1, 1))) { give_up(1, j); break; }
+            for (int j = 0; ok && j < nchunks; ++j, kv.advance(kKV)) {
+                const int s = kv.s;
+                if (j >= kKV && !(ok = pwait(bar_kv_empty + 8 * s, kv.ph ^ 1, 1))) { give_up(1, j); break; }
                 const bool mine = j == next_own;
-                if (mine && oi >= kQ && !(ok = pwait(bar_q_empty + 8 * (oi % kQ), (oi / kQ - 1) & 1, 2))) { give_up(2, j); break; }
-                TRACE(0, j);
+                if (mine && oi >= kQ && !(ok = pwait(bar_q_empty + 8 * qr.s, qr.ph ^ 1, 2))) { give_up(2, j); break; }
                 // one barrier per chunk: K, V and (own chunks) Q
                 mbar_expect_tx(bar_kv_full + 8 * s, (mine ? 3 : 2) * kTile);
-                tma_load_5d(kv_stage(j), &tm_v, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
-                tma_load_5d(kv_stage(j) + kTile, &tm_k, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
+                tma_load_5d(kv_stage(s), &tm_v, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
+                tma_load_5d(kv_stage(s) + kTile, &tm_k, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
                 if (mine) {
-                    tma_load_5d(q_stage(oi), &tm_q, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
+                    tma_load_5d(q_stage(qr.s), &tm_q, bar_kv_full + 8 * s, 0, h, j * kC, b, 0);
+                    qr.advance(kQ);
                     ++oi;
                     next_own += stride;
                 }
@@ -214,7 +218,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             if (!ok) {
                 // drain: every load that was issued lands before the CTA retires (a phase already consumed reads as complete)
                 for (int j = issued > kKV ? issued - kKV : 0; j < issued; ++j)
-                    mbar_wait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, nullptr, wc.limit);
+                    mbar_wait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, nullptr, wc.limit);   // (exit path: divisions are fine)
             }
         }
     } else if (warp == kWarpA) {
@@ -222,15 +226,15 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         if (lane == 0) {
             constexpr uint32_t idescG1 = make_idesc(128, kC, 0, 0);   // [V;K] (K-major) x Q^T (K-major)
             bool ok = true;
-            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
+            Ring kv = {g, 0}, qr = {0, 0};   // g < kKV
+            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride, kv.advance(kKV, stride), qr.advance(kQ)) {
                 const int buf = oi & 1;
                 // the chunk's K, V and Q have landed; the score warps have taken own chunk oi - 2 out of PT[buf]
-                ok = oi >= 2 ? pwait2(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, 3, bar_pt + 8 * buf, ((oi >> 1) - 1) & 1, 5)
-                             : pwait(bar_kv_full + 8 * (j % kKV), (j / kKV) & 1, 3);
+                ok = oi >= 2 ? pwait2(bar_kv_full + 8 * kv.s, kv.ph, 3, bar_pt + 8 * buf, ((oi >> 1) - 1) & 1, 5)
+                             : pwait(bar_kv_full + 8 * kv.s, kv.ph, 3);
                 if (!ok) { give_up(3, j); break; }
-                TRACE(1, oi);
                 tc_fence_after();
-                const uint32_t vk_lo = desc_lo(kv_stage(j)), q_lo = desc_lo(q_stage(oi));
+                const uint32_t vk_lo = desc_lo(kv_stage(kv.s)), q_lo = desc_lo(q_stage(qr.s));
 #pragma unroll
                 for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColPT + 64 * buf, vk_lo + 2 * k, q_lo + 2 * k, idescG1, k > 0);
                 umma_commit(bar_p + 8 * buf);
@@ -243,25 +247,25 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         if (lane == 0) {
             constexpr uint32_t idescG2 = make_idesc(128, 2 * kD, 0, 1);   // [Q;..] (K-major) x [S_hi | S_lo] (MN-major)
             bool ok = true;
-            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
+            Ring qr = {0, 0};
+            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride, qr.advance(kQ)) {
                 const int buf = oi & 1;
                 const uint32_t ph = (oi >> 1) & 1;
                 // after G3 of the same chunk (same accumulator), with the state tiles as of the previous chunk (the state
                 // warps arrive for every own chunk, also when there is nothing to add)
                 if (!(ok = pwait2(bar_ds + 8 * buf, ph, 8, bar_s + 8 * buf, ph, 9))) { give_up(8, j); break; }
-                TRACE(6, oi);
                 if (j > 0 || have_state) {
                     // Q's copy completed long ago (G1 has used it); this thread has not observed its barrier, the
                     // product that it issues follows the completed G1 and G3 of the chunk in the tensor core's order
                     tc_fence_after();
                     // B = [S_hi | S_lo]: two 64-column atoms, MN-major, one tile apart; columns 0..63 of OS[buf] take Q S_hi on top of
                     // P V, columns 64..127 take Q S_lo on top of the zeros the output warps left there
-                    const uint32_t q_lo = desc_lo(q_stage(oi)), s_lo = desc_lo(sbase + SM::offS + buf * 2 * kTile, kTile);
+                    const uint32_t q_lo = desc_lo(q_stage(qr.s)), s_lo = desc_lo(sbase + SM::offS + buf * 2 * kTile, kTile);
 #pragma unroll
                     for (int k = 0; k < kD / 16; ++k) umma_bf16(tmem + kColOS + 128 * buf, q_lo + 2 * k, s_lo + 128 * k, idescG2, 1, 1);
                 }
                 umma_commit(bar_o + 8 * buf);
-                umma_commit(bar_q_empty + 8 * (oi % kQ));
+                umma_commit(bar_q_empty + 8 * qr.s);
             }
             umma_commit(bar_fin + 8);
             pwait(bar_fin + 8, 0, 11);
@@ -272,38 +276,42 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             constexpr uint32_t idescG3 = make_idesc(128, kD, 1, 1);   // [P^T|K] (MN-major) x V (MN-major)
             bool ok = true;
             // K^T V of chunk c summed onto rows 64..127 of the accumulator at column `col` (output lanes write-disabled)
-            auto issue_ktv = [&](int c, uint32_t col, bool fresh) -> bool {
-                if (!pwait(bar_kv_full + 8 * (c % kKV), (c / kKV) & 1, 13)) { give_up(13, c); return false; }
+            auto issue_ktv = [&](int c, const Ring &kv, uint32_t col, bool fresh) -> bool {
+                if (!pwait(bar_kv_full + 8 * kv.s, kv.ph, 13)) { give_up(13, c); return false; }
                 tc_fence_after();
-                const uint32_t st = kv_stage(c);
+                const uint32_t st = kv_stage(kv.s);
                 const uint32_t a_lo = desc_lo(sbase + SM::offPT, st + kTile - (sbase + SM::offPT)), v_lo = desc_lo(st);
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + col, a_lo + 128 * k, v_lo + 128 * k, idescG3, (!fresh || k > 0) ? 1u : 0u, 2);
-                umma_commit(bar_kv_empty + 8 * (c % kKV));
+                umma_commit(bar_kv_empty + 8 * kv.s);
                 return true;
             };
             if (kShared && n_own > 0 && g > 0) {
                 // the chunks before the first own one -> DS, read once by the state warps
-                for (int c = 0; ok && c < g; ++c) ok = issue_ktv(c, kColDS, c == 0);
+                Ring kc = {0, 0};
+                for (int c = 0; ok && c < g; ++c, kc.advance(kKV)) ok = issue_ktv(c, kc, kColDS, c == 0);
                 if (ok) umma_commit(bar_d0);
             }
-            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride) {
+            Ring kv = {g, 0};   // g < kKV
+            for (int oi = 0, j = g; ok && oi < n_own; ++oi, j += stride, kv.advance(kKV, stride)) {
                 const int buf = oi & 1;
                 const uint32_t ph = (oi >> 1) & 1;
                 // the score tile is in shared memory; output and state warps have taken own chunk oi - 2 out of OS[buf]
                 // (they arrive once at the start, too)
                 if (!(ok = pwait2(bar_tile + 8 * buf, ph, 5, bar_of + 8 * buf, ph, 6))) { give_up(6, j); break; }
-                TRACE(4, oi);
                 tc_fence_after();
-                const uint32_t st = kv_stage(j), pt = sbase + SM::offPT + buf * kTile;
+                const uint32_t st = kv_stage(kv.s), pt = sbase + SM::offPT + buf * kTile;
                 const uint32_t a_lo = desc_lo(pt, st + kTile - pt), v_lo = desc_lo(st);
 #pragma unroll
                 for (int k = 0; k < kC / 16; ++k) umma_bf16(tmem + kColOS + 128 * buf, a_lo + 128 * k, v_lo + 128 * k, idescG3, k > 0);
-                umma_commit(bar_kv_empty + 8 * (j % kKV));   // K and V are read by G1 and G3 only
+                umma_commit(bar_kv_empty + 8 * kv.s);   // K and V are read by G1 and G3 only
                 // strided: the chunks up to the next own one, onto the rows where G3 has just put this chunk's own K^T V (same
                 // thread, so in this order), and the state warps read one sum per own chunk
-                if (kShared)
-                    for (int c = j + 1; ok && c < j + stride && c < nchunks; ++c) ok = issue_ktv(c, kColOS + 128 * buf, false);
+                if (kShared) {
+                    Ring kc = kv;
+                    kc.advance(kKV);
+                    for (int c = j + 1; ok && c < j + stride && c < nchunks; ++c, kc.advance(kKV)) ok = issue_ktv(c, kc, kColOS + 128 * buf, false);
+                }
                 umma_commit(bar_ds + 8 * buf);
             }
             umma_commit(bar_fin + 16);
@@ -324,7 +332,6 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         for (int oi = 0; oi < n_own; ++oi) {
             const int buf = oi & 1;
             if (!__all_sync(0xffffffffu, pwait(bar_p + 8 * buf, (oi >> 1) & 1, 16))) { if (lane == 0) give_up(16, oi); break; }
-            if (warp == 2) TRACE(9, oi);
             tc_fence_after();
             float p[32];
             tmem_ld32(tmem_warp + kColPT + 64 * buf, p);
@@ -350,7 +357,6 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             fence_proxy_async();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_tile + 8 * buf);
-            if (warp == 2) TRACE(10, oi);
         }
     } else if (warp == 10 || warp == 11 || warp == 14 || warp == 15) {
         // =========================================== state warps =======================================================
@@ -396,7 +402,6 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             // 1. sv = S_{j-1}: bf16 hi + lo tiles (MN-major B operand of G2_j); the buffer was last read by G2 of own chunk oi - 2
             if (j > 0 || have_state) {
                 if (oi >= 2 && !(ok = __all_sync(0xffffffffu, pwait(bar_o + 8 * buf, ((oi >> 1) - 1) & 1, 21)))) { if (lane == 0) give_up(21, j); break; }
-                if (warp == 10) TRACE(16, oi);
                 uint8_t *sHi = smem + SM::offS + buf * 2 * kTile, *sLo = sHi + kTile;
 #pragma unroll
                 for (int c8 = 0; c8 < kCols / 8; ++c8) {
@@ -411,25 +416,19 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     }
                     const uint32_t off = sw128(r, c0 / 8 + c8);
                     *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
-#ifndef PIPE_EXP_NOLO
                     *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-#endif
                 }
-                if (warp == 10) TRACE(17, oi);
                 fence_proxy_async();
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s + 8 * buf);   // also when there is nothing to write (first chunk, no initial state)
-            if (warp == 10) TRACE(11, oi);
             // 2. rows 64..127 of OS[buf]: the chunk's K^T V, plus (strided) that of the chunks up to the next own one
             if (!(ok = __all_sync(0xffffffffu, pwait(bar_ds + 8 * buf, (oi >> 1) & 1, 22)))) { if (lane == 0) give_up(22, j); break; }
             tc_fence_after();
-            if (warp == 10) TRACE(12, oi);
             add_tmem(kColOS + 128 * buf);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_of + 8 * buf);
-            if (warp == 10) TRACE(13, oi);
         }
         if (ok && state_out && nchunks == nch_total) {
             // this CTA owns the last chunk of the sequence: the fp32 state leaves the SM once, for the caller
@@ -458,7 +457,6 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         for (int oi = buf; oi < n_own; oi += 2) {
             const int j = g + oi * stride;
             if (!__all_sync(0xffffffffu, pwait(bar_o + 8 * buf, (oi >> 1) & 1, 24))) { if (lane == 0) give_up(24, j); break; }
-            if (half == 0) TRACE(14, oi);
             tc_fence_after();
             // columns 0..63: Q S_hi + P V, columns 64..127: Q S_lo; the latter are zeroed again for the chunk after next
             float acc[kD];
@@ -507,16 +505,12 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     bulk_commit();
                 }
             }
-            if (half == 0) TRACE(15, oi);
         }
         if (lane == 0) bulk_wait0();   // output boxes fully written before the CTA retires
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, tmem_cols);
-#ifdef PIPE_TIMING
-    if (blockIdx.x == 0 && tid < 32) reinterpret_cast<unsigned long long *>(status)[8 + tid] = probe[tid];
-#endif
 }
 
 // [B, L, H, 64] viewed as a rank-5 tensor (d, H, L, B, 1); box = (128 bytes of d) x 1 x rows x 1 x 1, 128-byte swizzle.
@@ -564,9 +558,6 @@ int linattn_sm100_pipe_stride(int B, int H, int L, int sms)
     int stride = (int)(sms / bh);
     if (stride > 4) stride = 4;
     if (stride > nchunks / 4) stride = nchunks / 4;
-#ifdef PIPE_STRIDE_ENV
-    if (const char *e = getenv("CHELA_STRIDE_TMP")) stride = atoi(e);
-#endif
     return stride < 1 ? 1 : stride;
 }
 
