@@ -126,7 +126,7 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
 
 /*
  * chela_linattn_fwd with the running state carried across calls, for segment-wise sequential evaluation
- * and decoding (Sec. 5, language modelling: "process each segment sequentially"; the state is the
+ * and decoding (Sec. 5, language modelling: segment-wise sequential evaluation; the state is the
  * intermediate variable of Sec. 4.1):
  *   S_{-1} = state_in (zero if NULL);  outputs as chela_linattn_fwd;  state_out = S after the last token.
  * Evaluating a sequence in consecutive segments with the state carried gives the result of one call over
@@ -199,6 +199,16 @@ chela_status_t chela_dense_fwd(const void *a, const void *w, const float *bias, 
 chela_status_t chela_async_status(const void *workspace, cudaStream_t stream);
 
 /*
+ * Test hook for the bounded waits (the paper has no counterpart).  Every device-side wait of the tensor-core kernels
+ * gives up after `limit_cycles` SM cycles (<= 0: the default, about one second) and then ends as chela_async_status
+ * describes.  skip_arrival != 0 makes the first CTA of the d = 64 linear-attention kernels and of the tensor-core
+ * projection leave out one mbarrier arrival, so that the role waiting for it runs into the limit: the kernel returns by
+ * itself, records CHELA_ERR_TIMEOUT, and words 8..11 of the workspace header keep the site of the wait, the CTA, the
+ * chunk and the grid size.  Process-wide, not thread-safe, read by every later launch: set it, launch, set it back.
+ */
+void chela_debug_wait_control(long long limit_cycles, int skip_arrival);
+
+/*
  * chela_linattn_fwd without a caller-provided workspace and without any allocation.  (The paper has no
  * counterpart: this is a packaging variant of the entry point above, same kernels, same results.)
  *
@@ -212,22 +222,25 @@ chela_status_t chela_async_status(const void *workspace, cudaStream_t stream);
  *
  *   - Arguments as chela_linattn_fwd, minus workspace and workspace_bytes.
  *   - A call whose chela_linattn_workspace_bytes() exceeds 8 MiB returns CHELA_ERR_WORKSPACE and launches
- *     nothing (use chela_linattn_fwd with your own workspace); with at most two CTAs per SM of split
- *     work the need stays below 5 MiB on a B200, so this is a guard, not an expected outcome.
+ *     nothing (use chela_linattn_fwd with your own workspace).  Plain bf16 and fp32 calls with d = 64 need the
+ *     512-byte header only.  d = 128 calls with few (batch, head) pairs keep one 64 KiB state sum per group of a
+ *     split sequence, up to one group per SM: B*H = 1 with L above about 130 000 tokens needs more than 8 MiB on a
+ *     148-SM part and is refused.
  *   - The first call on each device looks up the device address of the built-in array (with that device
  *     current) and caches it; make that first call during set-up, before any stream capture.
  *   - The call itself calls no cudaMalloc / cudaFree and no allocating library routine.
  *   - All calls on one GPU share the one array, which keeps the previous call's contents.  Nothing in it
  *     needs to start at zero except the status word, which each launch clears on `stream` itself.  Two
  *     calls that overlap on the GPU (different streams without an ordering event) race on it: order them.
- *   - The asynchronous status word lives inside the built-in array and is not exposed; callers that want
- *     to poll it use chela_linattn_fwd + chela_async_status.
+ *   - The asynchronous status word lives inside the built-in array: chela_linattn_static_ws_status(stream)
+ *     synchronises `stream` and returns it for the current device, like chela_async_status, without allocating.
  */
 chela_status_t chela_linattn_fwd_static_ws(const void *q, const void *k, const void *v, void *o,
                                            int B, int H, int L, int d_k, int d_v, int chunk,
                                            chela_dtype_t in_dtype, chela_dtype_t out_dtype,
                                            chela_norm_t norm, float norm_eps, float scale,
                                            cudaStream_t stream);
+chela_status_t chela_linattn_static_ws_status(cudaStream_t stream);
 
 /*
  * Token mixer forward without the gates (Eq. 7, Eqs. 10-12, Eq. 8 without G_a):

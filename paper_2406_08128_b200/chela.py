@@ -48,6 +48,8 @@ _SIGNATURES = {
     "chela_dense_fwd": (_c_int, [_vp, _vp, _vp, _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _vp,
                                  _c_size_t, _vp]),
     "chela_async_status": (_c_int, [_vp, _vp]),
+    "chela_debug_wait_control": (None, [ctypes.c_longlong, _c_int]),
+    "chela_linattn_static_ws_status": (_c_int, [_vp]),
     "chela_linattn_fwd_static_ws": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                              _c_float, _vp]),
     "chela_mixer_workspace_bytes": (_c_size_t, [_c_int] * 5 + [_c_int]),
@@ -265,6 +267,16 @@ def dense_fwd(a, w, bias=None, act=False, a_dtype=None, y_dtype=BF16, out=None, 
 def async_status(workspace) -> int:
     """Synchronise the current stream and return the asynchronous status recorded in ``workspace``."""
     return int(lib().chela_async_status(_ptr(workspace), _stream()))
+
+
+def debug_wait_control(limit_cycles=0, skip_arrival=0) -> None:
+    """chela_debug_wait_control: the wait limit (SM cycles, 0 = default) and the skipped-arrival test hook."""
+    lib().chela_debug_wait_control(int(limit_cycles), int(skip_arrival))
+
+
+def linattn_static_ws_status() -> int:
+    """Synchronise the current stream and return the status word of the built-in scratch (current device)."""
+    return int(lib().chela_linattn_static_ws_status(_stream()))
 
 
 def mixer_workspace_bytes(B, L, D, H, chunk, in_dtype=BF16) -> int:

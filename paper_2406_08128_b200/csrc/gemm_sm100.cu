@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(kThreads)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_constant__ CUtensorMap tm_a_lo,
                   const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y_hi,
                   const __grid_constant__ CUtensorMap tm_y_lo, const float *__restrict__ bias, int M, int N, int K,
-                  int act, int *__restrict__ status, int Lt)
+                  int act, int *__restrict__ status, int Lt, const WaitCtl wc)
 {
     using Smem = Smem<BN, kAPair>;
     constexpr int kStages = Smem::kStages, kStageBytes = Smem::kStageBytes, kStagingWarp = Smem::kStagingWarp;
@@ -104,7 +104,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                 const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % kStages;
-                    ok = mbar_wait(bar_empty0 + 8 * s, ((it / kStages) & 1) ^ 1, abort_flag);
+                    ok = mbar_wait(bar_empty0 + 8 * s, ((it / kStages) & 1) ^ 1, abort_flag, wc.limit);
                     if (!ok) break;
                     const uint32_t bar = bar_full0 + 8 * s, dst = sbase + Smem::offStage + s * kStageBytes;
                     mbar_expect_tx(bar, kStageBytes);
@@ -128,7 +128,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                 *abort_flag = 1;
                 atomicExch(status, (int)CHELA_ERR_TIMEOUT);
                 // loads still in flight land in this CTA's shared memory: wait for them (bounded)
-                for (int c = issued > kStages ? issued - kStages : 0; c < issued; ++c) mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1, nullptr);
+                for (int c = issued > kStages ? issued - kStages : 0; c < issued; ++c) mbar_wait(bar_full0 + 8 * (c % kStages), (c / kStages) & 1, nullptr, wc.limit);
             }
         }
     } else if (warp == 5) {
@@ -139,13 +139,13 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
             bool ok = true;
             for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
                 const int buf = ti & 1;
-                ok = mbar_wait(bar_tempty0 + 8 * buf, ((ti >> 1) & 1) ^ 1, abort_flag);
+                ok = mbar_wait(bar_tempty0 + 8 * buf, ((ti >> 1) & 1) ^ 1, abort_flag, wc.limit);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d = tmem + buf * BN;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % kStages;
-                    ok = mbar_wait(bar_full0 + 8 * s, (it / kStages) & 1, abort_flag);
+                    ok = mbar_wait(bar_full0 + 8 * s, (it / kStages) & 1, abort_flag, wc.limit);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t st = sbase + Smem::offStage + s * kStageBytes;
@@ -177,7 +177,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
         bool ok = true;
         for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++ti) {
             const int m0 = (t / n_tiles) * BM, n0 = (t % n_tiles) * BN, buf = ti & 1;
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull0 + 8 * buf, (ti >> 1) & 1, abort_flag));
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull0 + 8 * buf, (ti >> 1) & 1, abort_flag, wc.limit));
             if (!ok) break;
             tc_fence_after();
             const uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16) + buf * BN;
@@ -191,7 +191,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                     // the accumulator is in registers: hand the TMEM buffer back to the issuer
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_tempty0 + 8 * buf);
+                    // (test hook: the first hand-back of CTA 0 left out, so that the issuer's wait for it runs out)
+                    if (lane == 0 && !(wc.skip_arrival && blockIdx.x == 0 && ti == 0 && warp == 0)) mbar_arrive(bar_tempty0 + 8 * buf);
                 }
                 // the staging buffer is free once the store that last used it has been read (two boxes ago with
                 // ping-pong buffers, the previous box with one)
@@ -282,7 +283,7 @@ chela_status_t launch_gemm_sm100(const void *a, const void *w, const float *bias
     const int bn = (N % 256 == 0) ? 256 : 128;
     const long long tiles = (long long)((M + BM - 1) / BM) * (N / bn);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    typedef void (*Kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float *, int, int, int, int, int *, int);
+    typedef void (*Kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float *, int, int, int, int, int *, int, WaitCtl);
     Kern kern;
     int smem;
     if (bn == 256) {
@@ -295,7 +296,7 @@ chela_status_t launch_gemm_sm100(const void *a, const void *w, const float *bias
         smem = a_pair ? Smem<128, true>::bytes : Smem<128, false>::bytes;
     }
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
-    kern<<<grid, kThreads, smem, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status, 0);
+    kern<<<grid, kThreads, smem, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status, 0, current_wait_ctl());
     return last_launch_status();
 }
 
@@ -327,7 +328,7 @@ chela_status_t launch_gemm_sm100_at(const void *at, int B, int L, int Ls, const 
     auto kern = gemm_sm100_kernel<256, true, true, true>;
     constexpr int smem = Smem<256, true>::bytes;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CHELA_ERR_CUDA;
-    kern<<<grid, kThreads, smem, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status, L);
+    kern<<<grid, kThreads, smem, stream>>>(ma_hi, ma_lo, mw, my_hi, my_lo, bias, (int)M, N, K, act, status, L, current_wait_ctl());
     return last_launch_status();
 }
 

@@ -55,3 +55,13 @@ extern "C" chela_status_t chela_linattn_fwd_static_ws(const void *q, const void 
     return chela_linattn_fwd(q, k, v, o, B, H, L, d_k, d_v, chunk, in_dtype, out_dtype, norm, norm_eps, scale, ws,
                              kStaticWsBytes, stream);
 }
+
+// The asynchronous status word of the last chela_linattn_fwd_static_ws call on the current device (no allocation: one
+// word copied into a stack variable).
+extern "C" chela_status_t chela_linattn_static_ws_status(cudaStream_t stream)
+{
+    void *ws = nullptr;
+    const chela_status_t st = static_ws_pointer(&ws);
+    if (st != CHELA_OK) return st;
+    return chela_async_status(ws, stream);
+}

@@ -98,12 +98,9 @@ def test_back_to_back_backward_calls_on_split_sequences(B, L, H, d):
     ws = torch.zeros(int(chela.lib().chela_linattn_bwd_workspace_bytes(B, H, L, d, d)), dtype=torch.uint8, device="cuda")
     first = [g.clone() for g in chela.linattn_bwd(q, k, v, d_o, workspace=ws)]
     torch.cuda.synchronize()
-    t0 = time.perf_counter()
     for _ in range(8):
         grads = chela.linattn_bwd(q, k, v, d_o, workspace=ws)
     torch.cuda.synchronize()
-    elapsed = time.perf_counter() - t0
-    assert chela.async_status(ws) == chela.OK
-    assert elapsed < 0.5, elapsed
+    assert chela.async_status(ws) == chela.OK   # no bounded wait gave up
     for a, b in zip(first, grads):
         assert torch.equal(a, b)

@@ -224,12 +224,10 @@ def test_queued_calls_are_deterministic(B, L, H, d, pair):
     first = chela.linattn_fwd(q, k, v, out=o, workspace=ws, **kw).clone()
     torch.cuda.synchronize()
     outs = []
-    t0 = time.perf_counter()
     for _ in range(12):
         outs.append(chela.linattn_fwd(q, k, v, out=torch.empty_like(o), workspace=ws, **kw))
     torch.cuda.synchronize()
-    assert time.perf_counter() - t0 < 0.5
-    assert chela.async_status(ws) == chela.OK
+    assert chela.async_status(ws) == chela.OK   # no bounded wait gave up
     assert bool(torch.isfinite(first).all())
     for x in outs:
         assert torch.equal(first, x)
