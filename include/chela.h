@@ -59,12 +59,14 @@ int chela_version(void);
 int chela_linattn_kernel_kind(int B, int H, int L, int d_k, int d_v, int chunk,
                               chela_dtype_t in_dtype, chela_dtype_t out_dtype);
 
-/* How the tensor-core kernels split a sequence along L when there are fewer (batch, head) pairs than SMs (host
+/* How the tensor-core kernels share a sequence between CTAs when there are fewer (batch, head) pairs than SMs (host
  * logic only, no launch; the paper's tiling of Sec. 4.1 has no counterpart: it walks each sequence in one block).
- * The sequence's 64-token chunks are divided into *groups consecutive groups: the first of *first_chunks chunks, the
- * others of *other_chunks (the last one what is left); every group but the last is full and none is empty.
- * sms: SM count to plan for, <= 0 = the current device's.  in_dtype CHELA_BF16_PAIR plans for the full-pair kernel
- * (one CTA per SM).  Returns 1, or 0 for arguments no tensor-core kernel takes (d not 64 or 128, null pointers). */
+ * bf16-pair inputs (in_dtype CHELA_BF16_PAIR, one CTA per SM) and d = 128: the sequence's 64-token chunks are divided
+ * into *groups consecutive groups: the first of *first_chunks chunks, the others of *other_chunks (the last one what is
+ * left); every group but the last is full and none is empty.  Plain bf16 with d = 64: *groups CTAs, CTA g owning the
+ * chunks g, g + *groups, ...; *first_chunks = *other_chunks = 0 then (or the whole sequence when *groups = 1).
+ * sms: SM count to plan for, <= 0 = the current device's.  Returns 1, or 0 for arguments no tensor-core kernel takes
+ * (d not 64 or 128, null pointers). */
 int chela_linattn_split_plan(int B, int H, int L, int d, chela_dtype_t in_dtype, int sms,
                              int *groups, int *first_chunks, int *other_chunks);
 
@@ -114,8 +116,8 @@ chela_status_t chela_longconv_fwd(const void *x, const float *k_long, const floa
  * q, k : [B, L, H, d_k] in_dtype.  v : [B, L, H, d_v] in_dtype.  o : [B, L, H, d_v] out_dtype.
  * L need not be a multiple of chunk.  The result does not depend on chunk beyond rounding.
  * Supported: d_k = d_v in {64, 128}, chunk in {64, 128}.
- * Long sequences with few (batch, head) pairs are split along L; the per-split states live in
- * `workspace` (fp32).
+ * With fewer (batch, head) pairs than SMs a sequence is shared between several CTAs (plain bf16, d = 64: by stride,
+ * each CTA accumulating the whole state) or split along L (the per-split states then live in `workspace`, fp32).
  */
 size_t chela_linattn_workspace_bytes(int B, int H, int L, int d_k, int d_v, int chunk);
 chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, void *o,
@@ -131,7 +133,8 @@ chela_status_t chela_linattn_fwd(const void *q, const void *k, const void *v, vo
  *   S_{-1} = state_in (zero if NULL);  outputs as chela_linattn_fwd;  state_out = S after the last token.
  * Evaluating a sequence in consecutive segments with the state carried gives the result of one call over
  * the whole sequence (up to rounding).  state_in, state_out : [B, H, d_k, d_v] fp32, nullable, may alias
- * each other.  Supported: everything chela_linattn_fwd supports.
+ * each other (the initial state is then read from a copy that the call takes on `stream` first, in `workspace`,
+ * because several CTAs may work on one sequence).  Supported: everything chela_linattn_fwd supports.
  */
 chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void *v, void *o,
                                        const float *state_in, float *state_out,

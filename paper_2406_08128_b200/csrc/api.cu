@@ -32,6 +32,18 @@ MixerPlan mixer_plan(int B, int L, int D, int H, int chunk, bool gated)
     return p;
 }
 
+// Room for a copy of the initial state of chela_linattn_carry_fwd, behind the kernels' own workspace: needed when
+// state_in and state_out are the same buffer and a sequence may be shared between CTAs (fewer pairs than SMs).
+size_t carry_staging_bytes(int B, int H, int d)
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+    (void)cudaGetLastError();
+    if ((long long)B * H >= sms) return 0;
+    return 256 + (size_t)B * H * d * d * sizeof(float);
+}
+
 // what chela_debug_wait_control last set; process-wide, read by every tensor-core launch
 long long g_wait_limit_cycles = 2000000000LL;   // about one second at B200 clocks
 int g_skip_arrival = 0;
@@ -134,7 +146,7 @@ size_t chela_linattn_workspace_bytes(int B, int H, int L, int d_k, int d_v, int 
 {
     if (B < 1 || H < 1 || L < 1 || d_k != d_v || (d_k != 64 && d_k != 128) || (chunk != 64 && chunk != 128))
         return 0;
-    return linattn_sm100_workspace_bytes(B, H, L, d_k, chunk);
+    return linattn_sm100_workspace_bytes(B, H, L, d_k, chunk) + carry_staging_bytes(B, H, d_k);
 }
 
 chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void *v, void *o, const float *state_in,
@@ -153,8 +165,17 @@ chela_status_t chela_linattn_carry_fwd(const void *q, const void *k, const void 
     const int kind = chela_linattn_kernel_kind(B, H, L, d_k, d_v, chunk, in_dtype, out_dtype);
     if (kind == 0) return CHELA_ERR_UNSUPPORTED;
     if (kind == 2) {
-        const size_t need = linattn_sm100_workspace_bytes(B, H, L, d_k, chunk);
-        if (need && (!workspace || workspace_bytes < need)) return CHELA_ERR_WORKSPACE;
+        const size_t base = linattn_sm100_workspace_bytes(B, H, L, d_k, chunk), staging = carry_staging_bytes(B, H, d_k);
+        if (!workspace || workspace_bytes < base + staging) return CHELA_ERR_WORKSPACE;
+        if (state_in && state_in == state_out && staging) {
+            // A sequence may be shared between several CTAs (few (batch, head) pairs): every one of them reads the initial
+            // state when it starts, one writes the final state when it ends, and nothing orders the two across CTAs.  With
+            // aliased pointers the initial state is therefore read from a copy taken on the stream first.
+            float *copy = reinterpret_cast<float *>(static_cast<char *>(workspace) + align_up(base, 256));
+            if (cudaMemcpyAsync(copy, state_in, (size_t)B * H * d_k * d_k * sizeof(float), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+                return CHELA_ERR_CUDA;
+            state_in = copy;
+        }
         return launch_linattn_sm100(q, k, v, o, B, H, L, d_k, chunk, in_dtype, out_dtype, (int)norm, norm_eps,
                                     scale, workspace, stream, state_in, state_out);
     }

@@ -803,6 +803,13 @@ void linattn_sm100_split(int B, int H, int L, int d, bool full_pair, int sms, in
         linattn_sm100_d128_split(B, H, L, sms, G, cg0, cg);
         return;
     }
+    if (!full_pair) {
+        // plain bf16: no groups of consecutive chunks; with fewer pairs than SMs a sequence is shared by stride
+        const int stride = linattn_sm100_pipe_stride(B, H, L, sms);
+        *G = stride > 1 ? stride : 1;
+        *cg0 = *cg = stride > 1 ? 0 : (L + kC - 1) / kC;
+        return;
+    }
     const SplitPlan p = split_plan(B, H, L, full_pair, sms);
     *G = p.G;
     *cg0 = p.cg0;

@@ -95,9 +95,11 @@ def test_missing_library_fails_loudly(monkeypatch):
 
 
 def test_split_plan_covers_every_sequence_exactly(lib):
-    """Host logic of the split along L (no GPU: the SM count is passed in).  For every shape: the groups tile the
-    sequence's chunks exactly, none is empty, all but the last are full, no more CTAs than are resident at once,
-    and no split at all once there are as many (batch, head) pairs as SMs."""
+    """Host logic of how a sequence is shared between CTAs (no GPU: the SM count is passed in).  Grouped plans: the
+    groups tile the sequence's chunks exactly, none is empty, all but the last are full.  Strided plans (plain bf16,
+    d = 64; reported with zero chunk counts): every CTA owns at least four chunks and there is one CTA per SM at most.
+    Both: no more CTAs than are resident at once, and one CTA per sequence once there are as many (batch, head)
+    pairs as SMs."""
     sms = 148
     for d, pair in ((64, False), (64, True), (128, False)):
         dt = chela.BF16_PAIR if pair else chela.BF16
@@ -107,6 +109,10 @@ def test_split_plan_covers_every_sequence_exactly(lib):
                 assert plan is not None
                 G, c0, c = plan
                 nch = (L + 63) // 64
+                if G > 1 and c0 == 0:   # strided: CTA g owns chunks g, g + G, ...
+                    assert d == 64 and not pair and c == 0
+                    assert 2 <= G <= 4 and nch // G >= 4 and bh * G <= sms, (d, pair, bh, L, plan)
+                    continue
                 assert G >= 1 and c0 >= 1 and c >= 1, (d, pair, bh, L, plan)
                 if G == 1:
                     assert c0 >= nch

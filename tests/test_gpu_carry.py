@@ -28,6 +28,24 @@ def test_segments_with_carried_state_equal_one_call(dtype, tol, d, B, H, cuts):
     assert np.abs(to_numpy(state) - ref_state).max() <= (2e-3 if dtype == "bf16" else 1e-5) * np.abs(ref_state).max()
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_aliased_state_on_sequences_that_several_ctas_share(d):
+    """state_in and state_out the same buffer, on a shape where a sequence is shared between CTAs (d = 64: by stride)
+    or split along L (d = 128): every CTA starts from the initial state although one of them overwrites the buffer."""
+    import torch
+    B, H, L = 1, 2, 8192
+    q, k, v = inputs.qkv(66 + d, B, 2 * L, H, d, d, "bf16")
+    ref, ref_state = oracle.linattn_recurrent(q, k, v, return_state=True)
+    state = torch.zeros(B, H, d, d, device="cuda")
+    outs = []
+    for a in (0, L):
+        qs, ks, vs = (to_device(np.ascontiguousarray(x[:, a:a + L]), "bf16") for x in (q, k, v))
+        o, _ = chela.linattn_carry_fwd(qs, ks, vs, state_in=state, state_out=state)
+        outs.append(to_numpy(o))
+    assert rel_err(np.concatenate(outs, axis=1), ref) <= 2e-2
+    assert np.abs(to_numpy(state) - ref_state).max() <= 2e-3 * np.abs(ref_state).max()
+
+
 def test_state_out_without_state_in_and_oracle_state_in():
     import torch
     B, L, H, d = 1, 300, 2, 64
