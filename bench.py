@@ -160,6 +160,31 @@ def job_tokens_per_s(ms_step: float, world: int, tokens_per_rank: int) -> float:
     return world * tokens_per_rank / (ms_step * 1e-3)
 
 
+def mixer_flops_per_token(D_model: int, n_heads: int, gated: bool = False) -> float:
+    """Algorithmic tensor flops of the token mixer per token: three (five with the gates) D x D projections and the
+    attention tiles.  The attention kernels walk 64-token tiles whatever `chunk` says (the result does not depend on
+    it), so the tile term is 4*64*d + 4*d*d per token-head for chunk = 64 and chunk = 128 alike."""
+    d_head = D_model // n_heads
+    return (5 if gated else 3) * 2 * D_model * D_model + n_heads * (4 * 64 * d_head + 4 * d_head * d_head)
+
+
+def sweep_linearity(sweep):
+    """Time vs L at fixed B*L: spread of the times around their mean and the log-log slope of per-sequence time
+    against L (a method that is linear in L has slope 1 and a flat time at fixed tokens)."""
+    import math
+    ms = [e["ms"] for e in sweep]
+    mean = sum(ms) / len(ms)
+    xs = [math.log(e["L"]) for e in sweep]
+    ys = [math.log(e["ms"] / e["B"]) for e in sweep]   # per-sequence time
+    n = len(xs)
+    mx, my = sum(xs) / n, sum(ys) / n
+    slope = sum((x - mx) * (y - my) for x, y in zip(xs, ys)) / sum((x - mx) ** 2 for x in xs)
+    lo, hi = min(ms) / mean - 1.0, max(ms) / mean - 1.0
+    return {"loglog_slope_time_per_sequence_vs_L": slope, "mean_ms": mean, "spread_vs_mean": [lo, hi],
+            "max_over_min": max(ms) / min(ms), "within_pm10pct_of_mean": bool(lo >= -0.10 and hi <= 0.10),
+            "slope_within_1_pm_0p05": bool(abs(slope - 1.0) <= 0.05), "min_hbm_frac": min(e["hbm_frac"] for e in sweep)}
+
+
 def workload_config():
     return {"workload": "linattn_fwd sweep point L=%d: B=%d, H=16, d_k=d_v=64, chunk=64, bf16 in, fp32 out" % (
                 L_MAIN, TOTAL_TOKENS // L_MAIN),
@@ -182,7 +207,8 @@ def run_mixer_mode(args):
     w_q, w_k, w_v = [(torch.randn(md, md, device=dev, generator=gen) / md ** 0.5).to(torch.bfloat16) for _ in range(3)]
     ws = torch.zeros(chela.mixer_workspace_bytes(mb, ml, md, mh, mc), dtype=torch.uint8, device=dev)
     out = torch.empty(mb, ml, md, device=dev)
-    step = lambda: chela.mixer_fwd(x, w_s, k_l, w_q, w_k, w_v, mh, chunk=mc, out=out, workspace=ws)
+    spec = chela.longconv_prepare(k_l)   # the long kernels' spectra: weights do not change between steps
+    step = lambda: chela.mixer_prepared_fwd(x, w_s, spec, w_q, w_k, w_v, mh, chunk=mc, out=out, workspace=ws)
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -197,7 +223,7 @@ def run_mixer_mode(args):
     ms = e0.elapsed_time(e1) / args.steps
     peaks, peak_kind = measured_peaks()
     d_head = md // mh
-    flops_tok = 3 * 2 * md * md + mh * (4 * 64 * d_head + 4 * d_head * d_head)
+    flops_tok = mixer_flops_per_token(md, mh)
     achieved = flops_tok * mb * ml / (ms * 1e-3) / 1e12
     print(json.dumps({"metric": "mixer_fwd_tokens_per_s", "value": mb * ml / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
                       "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
@@ -416,7 +442,8 @@ def main():
     achieved = alg_bytes / (ms_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES_PER_TOKEN * TOTAL_TOKENS,
-                "traffic_source": "ncu capture of a 32768-token case scaled by tokens", "peak_source": peak_kind,
+                "traffic_source": "ncu capture of a 32768-token case scaled by tokens; a lower bound (the tail of the output is still "
+                                  "in L2 when that small kernel ends), reads equal the algorithmic reads", "peak_source": peak_kind,
                 "kernel": "linattn_sm100_kernel<64,float>" if kind == 2 else "linattn_simt_kernel",
                 "algorithmic_bytes_per_launch": alg_bytes, "launch_ms": ms_step}
 
@@ -445,6 +472,20 @@ def main():
             sweep.append({"L": L, "B": TOTAL_TOKENS // L, "ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
                           "hbm_frac": alg_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]})
         line["sweep"] = sweep
+        line["sweep_linearity"] = sweep_linearity(sweep)
+        # ---- d = 128 (config 4's head size) plain bf16 linear attention at the same token count: H = 8 ----------
+        n128 = TOTAL_TOKENS * 8 * 128
+        q8, k8, v8 = (flat[j][:n128].view(16, TOTAL_TOKENS // 16, 8, 128) for j in range(3))
+        o8 = out_flat[:n128].view(16, TOTAL_TOKENS // 16, 8, 128)
+        ws8 = torch.zeros(chela.linattn_workspace_bytes(16, 8, TOTAL_TOKENS // 16, 128, 128, 128), dtype=torch.uint8, device=dev)
+        ms = timed(lambda: chela.linattn_fwd(q8, k8, v8, chunk=128, out_dtype=chela.F32, out=o8, workspace=ws8), 20, warm=5)
+        if chela.async_status(ws8) != chela.OK:
+            raise RuntimeError("device-side wait timed out in the d = 128 extra")
+        b128 = TOTAL_TOKENS * 8 * (3 * 128 * 2 + 128 * 4)
+        line["linattn_d128"] = {"B": 16, "L": TOTAL_TOKENS // 16, "H": 8, "d": 128, "ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
+                                "hbm_frac": b128 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                "note": "plain bf16 in, fp32 out, d_k = d_v = 128; algorithmic bytes 1280 per token-head"}
+        del ws8
         # ---- config 2: B=8, H=8, L=4096 (134 MB in + 67 MB out; four rotating buffer sets exceed L2) ----
         sets = []
         for s in range(4):
@@ -467,6 +508,15 @@ def main():
         del sets
         # ---- token mixer forward (configs 3 and 4): short conv + SiLU, long conv, Q/K/V, attention --------
         # roofline: bf16 tensor peak over the algorithmic flops (3 dense projections + the attention tiles)
+        # fp32 FMA rate of this GPU, measured now: a cuBLAS fp32 GEMM with TF32 off runs on the plain FMA pipes
+        # (library kernel, used only as the denominator of the long convolution's ALU fraction)
+        tf32_was = torch.backends.cuda.matmul.allow_tf32
+        torch.backends.cuda.matmul.allow_tf32 = False
+        ga, gb = torch.randn(8192, 8192, device=dev), torch.randn(8192, 8192, device=dev)
+        ms_g = timed(lambda: torch.matmul(ga, gb), 5, warm=2)
+        torch.backends.cuda.matmul.allow_tf32 = tf32_was
+        fp32_peak = 2 * 8192.0 ** 3 / (ms_g * 1e-3) / 1e12
+        del ga, gb
         mixers = []
         for (mb, ml, md, mh, mc) in ((4, 16384, 512, 8, 64), (8, 8192, 1024, 8, 128)):
             x = torch.randn(mb, ml, md, device=dev, generator=gen).to(torch.bfloat16)
@@ -475,12 +525,15 @@ def main():
             w_q, w_k, w_v = [(torch.randn(md, md, device=dev, generator=gen) / md ** 0.5).to(torch.bfloat16) for _ in range(3)]
             mws = torch.zeros(chela.mixer_workspace_bytes(mb, ml, md, mh, mc), dtype=torch.uint8, device=dev)
             mo = torch.empty(mb, ml, md, device=dev)
-            ms = timed(lambda: chela.mixer_fwd(x, w_s, k_l, w_q, w_k, w_v, mh, chunk=mc, out=mo, workspace=mws), 20, warm=5)
+            spec = chela.longconv_prepare(k_l)   # the long kernels' spectra, once: the weights do not change between calls
+            ms = timed(lambda: chela.mixer_prepared_fwd(x, w_s, spec, w_q, w_k, w_v, mh, chunk=mc, out=mo, workspace=mws), 20, warm=5)
+            ms_unprepared = timed(lambda: chela.mixer_fwd(x, w_s, k_l, w_q, w_k, w_v, mh, chunk=mc, out=mo, workspace=mws), 10, warm=3)
             if chela.async_status(mws) != chela.OK:
                 raise RuntimeError("device-side wait timed out in the mixer")
             d_head = md // mh
-            flops_tok = 3 * 2 * md * md + mh * (4 * mc * d_head + 4 * d_head * d_head)
-            mixers.append({"B": mb, "L": ml, "D": md, "H": mh, "chunk": mc, "ms": ms,
+            flops_tok = mixer_flops_per_token(md, mh)
+            mixers.append({"B": mb, "L": ml, "D": md, "H": mh, "chunk": mc, "attention_tile_tokens": 64, "ms": ms, "ms_spectra_recomputed_every_call": ms_unprepared,
+                           "call": "chela_mixer_prepared_fwd (kernel spectra prepared once with chela_longconv_prepare)",
                            "tokens_per_s": mb * ml / (ms * 1e-3),
                            "tensor_frac": flops_tok * mb * ml / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                            "attention_kernel_kind": chela.linattn_kernel_kind(mb, mh, ml, d_head, d_head, mc,
@@ -496,11 +549,11 @@ def main():
             ms_l = timed(lambda: chela.longconv_fwd(x, k_l, w_s, out=z_l, workspace=cws), 20, warm=5)
             m_pts = 1 << (ml - 1).bit_length()
             fft_flops = (mb * md * 2 + md) * 5 * m_pts * (m_pts.bit_length() - 1)   # forward + inverse per row, forward per kernel
-            fp32_peak = 148 * 128 * 2 * 1.965e9 / 1e12
             stage["longconv"] = {"ms": ms_l, "fft_TFLOPs": fft_flops / (ms_l * 1e-3) / 1e12, "alu_peak_TFLOPs": fp32_peak,
                                  "alu_frac": fft_flops / (ms_l * 1e-3) / 1e12 / fp32_peak,
+                                 "alu_peak_source": "measured in this run: fp32 GEMM 8192^3 with TF32 off (plain FMA pipes)",
                                  "note": "short conv + SiLU + transposes + FFT long conv, bf16 in, fp32 out; flops = 5 M log2 M "
-                                         "per M-point transform; peak = 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz (FMA counted as 2)"}
+                                         "per M-point transform"}
             z_p = torch.randn(2, mb * ml, md, device=dev, generator=gen).to(torch.bfloat16)
             q_p = torch.empty(2, mb * ml, md, device=dev, dtype=torch.bfloat16)
             dws = torch.zeros(max(int(chela.lib().chela_dense_workspace_bytes()), 16), dtype=torch.uint8, device=dev)
@@ -510,7 +563,16 @@ def main():
                                    "tensor_frac": mma_flops / (ms_d * 1e-3) / 1e12 / peaks["bf16_tflops"],
                                    "note": "one Q or K projection, bf16-pair A (token-major) and Y: both tensor-core terms counted"}
             mixers[-1]["stages"] = stage
-            del x, k_l, mws, mo, y_s, z_l, cws, z_p, q_p, dws
+            # the gated form (Eqs. 8-14): two more projections and the gate epilogue
+            w_a, w_o2 = [(torch.randn(md, md, device=dev, generator=gen) / md ** 0.5).to(torch.bfloat16) for _ in range(2)]
+            gws = torch.zeros(chela.mixer_gated_workspace_bytes(mb, ml, md, mh, mc), dtype=torch.uint8, device=dev)
+            ms_gt = timed(lambda: chela.mixer_prepared_fwd(x, w_s, spec, w_q, w_k, w_v, mh, w_a=w_a, w_o=w_o2, chunk=mc, out=mo, workspace=gws), 10, warm=3)
+            if chela.async_status(gws) != chela.OK:
+                raise RuntimeError("device-side wait timed out in the gated mixer")
+            mixers[-1]["gated"] = {"ms": ms_gt, "tokens_per_s": mb * ml / (ms_gt * 1e-3),
+                                   "tensor_frac": mixer_flops_per_token(md, mh, True) * mb * ml / (ms_gt * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+            del gws, w_a, w_o2
+            del x, k_l, mws, mo, y_s, z_l, cws, z_p, q_p, dws, spec
         line["mixer"] = mixers
         # ---- backward of the timed workload (gradients w.r.t. Q, K, V; normaliser on) ----------------------------
         (q_, k_, v_), _ = views(L_MAIN)
@@ -519,8 +581,13 @@ def main():
         ms = timed(lambda: chela.linattn_bwd(q_, k_, v_, d_o, workspace=bws), 10, warm=3)
         if chela.async_status(bws) != chela.OK:
             raise RuntimeError("device-side wait timed out in the backward pass")
+        bwd_alg = TOTAL_TOKENS * H * D * (4 * 2 + 3 * 4)   # read q, k, v, d_o (bf16), write dq, dk, dv (fp32): 20 B per element
         line["backward"] = {"ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
-                            "note": "chela_linattn_bwd, bf16 in, fp32 gradients, same workload as the timed step"}
+                            "roofline": {"bound": "hbm", "achieved": bwd_alg / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                         "frac": bwd_alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_kind,
+                                         "algorithmic_bytes_per_call": bwd_alg},
+                            "note": "chela_linattn_bwd, bf16 in, fp32 gradients, same workload as the timed step; algorithmic "
+                                    "bytes of a one-pass backward (20 B per element) over the time of the whole multi-launch call"}
         # forward + backward at every L of the sweep (the quantity the paper's runtime-vs-length figure plots)
         fb = []
         sweep_ms = {e["L"]: e["ms"] for e in sweep}

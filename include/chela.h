@@ -283,6 +283,31 @@ chela_status_t chela_mixer_gated_fwd(const void *x, const float *w_short, int sh
                                      float norm_eps, void *workspace, size_t workspace_bytes,
                                      cudaStream_t stream);
 
+/*
+ * The long convolution for weights that do not change between calls (Eq. 6: y = F^-1 D_K F u; D_K, the spectrum of
+ * the zero-padded kernel, depends on the weights only).  chela_longconv_prepare writes the spectra of all D kernels
+ * and the transform's twiddle table into a caller-owned device buffer of chela_longconv_spectrum_bytes(L, D) bytes
+ * (16-byte aligned; 0 = unsupported L or D); the *_prepared_fwd calls take that buffer in place of k_long and skip
+ * that part of the work, with results identical to the calls they stand for.  The buffer is only valid for the
+ * (L, D) and the weights it was prepared for, and must not be written while a call that reads it is in flight.
+ *   chela_longconv_prepared_fwd : chela_longconv_fwd with `spectrum` in place of k_long.
+ *   chela_mixer_prepared_fwd    : chela_mixer_fwd (w_a = w_o = NULL) or chela_mixer_gated_fwd (both given, with the
+ *                                 gated workspace size) with `spectrum` in place of k_long.
+ */
+size_t chela_longconv_spectrum_bytes(int L, int D);
+chela_status_t chela_longconv_prepare(const float *k_long, int L, int D, void *spectrum, size_t spectrum_bytes,
+                                      cudaStream_t stream);
+chela_status_t chela_longconv_prepared_fwd(const void *x, const void *spectrum, const float *w_short, int short_width,
+                                           void *z, int B, int L, int D, chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                                           void *workspace, size_t workspace_bytes, cudaStream_t stream);
+chela_status_t chela_mixer_prepared_fwd(const void *x, const float *w_short, int short_width, const void *spectrum,
+                                        const void *w_q, const void *w_k, const void *w_v, const float *b_q,
+                                        const float *b_k, const float *b_v, const void *w_a, const float *b_a,
+                                        const void *w_o, const float *b_o, int qk_diag, int v_silu, void *o, int B,
+                                        int L, int D, int H, int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                                        chela_norm_t norm, float norm_eps, void *workspace, size_t workspace_bytes,
+                                        cudaStream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -57,6 +57,12 @@ _SIGNATURES = {
     "chela_mixer_gated_fwd": (_c_int, [_vp, _vp, _c_int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _c_int, _c_int,
                                        _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_float,
                                        _vp, _c_size_t, _vp]),
+    "chela_longconv_spectrum_bytes": (_c_size_t, [_c_int, _c_int]),
+    "chela_longconv_prepare": (_c_int, [_vp, _c_int, _c_int, _vp, _c_size_t, _vp]),
+    "chela_longconv_prepared_fwd": (_c_int, [_vp, _vp, _vp, _c_int, _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _vp, _c_size_t, _vp]),
+    "chela_mixer_prepared_fwd": (_c_int, [_vp, _vp, _c_int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _c_int, _c_int,
+                                          _vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_float,
+                                          _vp, _c_size_t, _vp]),
     "chela_mixer_fwd": (_c_int, [_vp, _vp, _c_int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _c_int, _c_int, _vp,
                                  _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_float,
                                  _vp, _c_size_t, _vp]),
@@ -267,6 +273,45 @@ def dense_fwd(a, w, bias=None, act=False, a_dtype=None, y_dtype=BF16, out=None, 
 def async_status(workspace) -> int:
     """Synchronise the current stream and return the asynchronous status recorded in ``workspace``."""
     return int(lib().chela_async_status(_ptr(workspace), _stream()))
+
+
+def longconv_prepare(k_long, out=None):
+    """chela_longconv_prepare: the spectra of the long kernels k_long [D, L] (and the twiddle table) in a device buffer."""
+    D, L = k_long.shape
+    n = int(lib().chela_longconv_spectrum_bytes(L, D))
+    if n == 0:
+        raise ChelaError(ERR_UNSUPPORTED, "chela_longconv_spectrum_bytes")
+    spec = torch.empty(n, dtype=torch.uint8, device=k_long.device) if out is None else out
+    _check(lib().chela_longconv_prepare(_ptr(k_long), L, D, _ptr(spec), spec.numel(), _stream()), "chela_longconv_prepare")
+    return spec
+
+
+def longconv_prepared_fwd(x, spectrum, w_short=None, out_dtype=F32, out=None, workspace=None):
+    """chela_longconv_prepared_fwd: chela_longconv_fwd with prepared spectra in place of the kernels."""
+    B, L, D = x.shape
+    z = torch.empty((B, L, D), dtype=_tdtype(out_dtype), device=x.device) if out is None else out
+    if workspace is None:
+        workspace = _workspace(longconv_workspace_bytes(B, L, D, _dt(x), out_dtype), x.device)
+    _check(lib().chela_longconv_prepared_fwd(_ptr(x), _ptr(spectrum), _ptr(w_short), 0 if w_short is None else w_short.shape[1],
+                                             _ptr(z), B, L, D, _dt(x), _dt(z), _ptr(workspace), workspace.numel(), _stream()),
+           "chela_longconv_prepared_fwd")
+    return z
+
+
+def mixer_prepared_fwd(x, w_short, spectrum, w_q, w_k, w_v, H, w_a=None, w_o=None, chunk=64, b_q=None, b_k=None, b_v=None,
+                       b_a=None, b_o=None, qk_diag=False, v_silu=True, out_dtype=F32, norm=NORM_RMS, eps=1e-6, out=None,
+                       workspace=None):
+    """chela_mixer_prepared_fwd: the mixer (gated when w_a and w_o are given) with prepared long-kernel spectra."""
+    B, L, D = x.shape
+    o = torch.empty((B, L, D), dtype=_tdtype(out_dtype), device=x.device) if out is None else out
+    if workspace is None:
+        need = mixer_gated_workspace_bytes(B, L, D, H, chunk, _dt(x)) if w_a is not None else mixer_workspace_bytes(B, L, D, H, chunk, _dt(x))
+        workspace = _workspace(need, x.device)
+    _check(lib().chela_mixer_prepared_fwd(_ptr(x), _ptr(w_short), w_short.shape[1], _ptr(spectrum), _ptr(w_q), _ptr(w_k), _ptr(w_v),
+                                          _ptr(b_q), _ptr(b_k), _ptr(b_v), _ptr(w_a), _ptr(b_a), _ptr(w_o), _ptr(b_o), int(qk_diag),
+                                          int(v_silu), _ptr(o), B, L, D, H, chunk, _dt(x), _dt(o), int(norm), float(eps),
+                                          _ptr(workspace), workspace.numel(), _stream()), "chela_mixer_prepared_fwd")
+    return o
 
 
 def debug_wait_control(limit_cycles=0, skip_arrival=0) -> None:

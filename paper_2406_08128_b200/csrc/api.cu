@@ -128,6 +128,33 @@ size_t chela_longconv_workspace_bytes(int B, int L, int D, chela_dtype_t, chela_
     return longconv_workspace_bytes(B, L, D);
 }
 
+size_t chela_longconv_spectrum_bytes(int L, int D)
+{
+    if (L < 1 || L > 16384 || D < 1 || D % 8 != 0) return 0;
+    return longconv_spectrum_bytes(L, D);
+}
+
+chela_status_t chela_longconv_prepare(const float *k_long, int L, int D, void *spectrum, size_t spectrum_bytes, cudaStream_t stream)
+{
+    if (!k_long || !spectrum || L < 1 || D < 1 || !aligned16(spectrum)) return CHELA_ERR_INVALID_ARG;
+    if (L > 16384 || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
+    if (spectrum_bytes < longconv_spectrum_bytes(L, D)) return CHELA_ERR_WORKSPACE;
+    return launch_longconv_prepare(k_long, L, D, spectrum, stream);
+}
+
+chela_status_t chela_longconv_prepared_fwd(const void *x, const void *spectrum, const float *w_short, int short_width,
+                                           void *z, int B, int L, int D, chela_dtype_t in_dtype, chela_dtype_t out_dtype,
+                                           void *workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    if (!x || !spectrum || !z || B < 1 || L < 1 || D < 1 || !dtype_ok(in_dtype) || !dtype_ok(out_dtype))
+        return CHELA_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(z) || !aligned16(workspace) || !aligned16(spectrum)) return CHELA_ERR_INVALID_ARG;
+    if (L > 16384 || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
+    if (w_short && (short_width < 1 || short_width > 16)) return CHELA_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < longconv_workspace_bytes(B, L, D)) return CHELA_ERR_WORKSPACE;
+    return launch_longconv(x, nullptr, w_short, short_width, z, B, L, D, in_dtype, out_dtype, workspace, stream, false, spectrum);
+}
+
 chela_status_t chela_longconv_fwd(const void *x, const float *k_long, const float *w_short, int short_width,
                                   void *z, int B, int L, int D, chela_dtype_t in_dtype,
                                   chela_dtype_t out_dtype, void *workspace, size_t workspace_bytes,
@@ -277,7 +304,7 @@ size_t chela_mixer_gated_workspace_bytes(int B, int L, int D, int H, int chunk, 
 }  // extern "C"
 
 namespace {
-chela_status_t mixer_impl(const void *x, const float *w_short, int short_width, const float *k_long, const void *w_q,
+chela_status_t mixer_impl(const void *x, const float *w_short, int short_width, const float *k_long, const void *spectrum, const void *w_q,
                           const void *w_k, const void *w_v, const float *b_q, const float *b_k, const float *b_v,
                           const void *w_a, const float *b_a, const void *w_o, const float *b_o, int qk_diag, int v_silu,
                           void *o, int B, int L, int D, int H, int chunk, chela_dtype_t in_dtype, chela_dtype_t out_dtype,
@@ -285,7 +312,7 @@ chela_status_t mixer_impl(const void *x, const float *w_short, int short_width, 
 {
     const bool gated = w_a != nullptr;
     if (gated && !w_o) return CHELA_ERR_INVALID_ARG;
-    if (!x || !w_short || !k_long || !w_q || !w_k || !w_v || !o || B < 1 || L < 1 || D < 1 || H < 1 ||
+    if (!x || !w_short || (!k_long && !spectrum) || !aligned16(spectrum) || !w_q || !w_k || !w_v || !o || B < 1 || L < 1 || D < 1 || H < 1 ||
         !dtype_ok(in_dtype) || !dtype_ok(out_dtype) || (norm != CHELA_NORM_NONE && norm != CHELA_NORM_RMS) ||
         !(norm_eps >= 0.f))
         return CHELA_ERR_INVALID_ARG;
@@ -320,7 +347,7 @@ chela_status_t mixer_impl(const void *x, const float *w_short, int short_width, 
         // saves the transpose back to token-major
         const int Ls = longconv_row_stride(L);
         const bool zt = !qk_diag && longconv_transposed_pair_supported(L) && gemm_sm100_at_supported(B, L, Ls, D, D);
-        st = launch_longconv(x, k_long, w_short, short_width, zp, B, L, D, in_dtype, CHELA_BF16_PAIR, ws + p.off_conv, stream, zt);
+        st = launch_longconv(x, k_long, w_short, short_width, zp, B, L, D, in_dtype, CHELA_BF16_PAIR, ws + p.off_conv, stream, zt, spectrum);
         if (st != CHELA_OK) return st;
         if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return CHELA_ERR_CUDA;
         if (zt) {
@@ -354,7 +381,7 @@ chela_status_t mixer_impl(const void *x, const float *w_short, int short_width, 
     }
     // fp32 path.  Z = K_l(silu(K_s(X)))  (Eq. 7), kept in fp32
     st = launch_longconv(x, k_long, w_short, short_width, z, B, L, D, in_dtype, CHELA_F32,
-                         ws + p.off_conv, stream);
+                         ws + p.off_conv, stream, false, spectrum);
     if (st != CHELA_OK) return st;
     // Q, K from Z (Eqs. 10-11, or dense projections), V from X (Eq. 12)
     if (qk_diag) {
@@ -390,9 +417,21 @@ chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_wi
                                chela_dtype_t out_dtype, chela_norm_t norm, float norm_eps, void *workspace,
                                size_t workspace_bytes, cudaStream_t stream)
 {
-    return mixer_impl(x, w_short, short_width, k_long, w_q, w_k, w_v, b_q, b_k, b_v, nullptr, nullptr, nullptr, nullptr,
+    return mixer_impl(x, w_short, short_width, k_long, nullptr, w_q, w_k, w_v, b_q, b_k, b_v, nullptr, nullptr, nullptr, nullptr,
                       qk_diag, v_silu, o, B, L, D, H, chunk, in_dtype, out_dtype, norm, norm_eps, workspace, workspace_bytes,
                       stream);
+}
+
+chela_status_t chela_mixer_prepared_fwd(const void *x, const float *w_short, int short_width, const void *spectrum,
+                                        const void *w_q, const void *w_k, const void *w_v, const float *b_q, const float *b_k,
+                                        const float *b_v, const void *w_a, const float *b_a, const void *w_o, const float *b_o,
+                                        int qk_diag, int v_silu, void *o, int B, int L, int D, int H, int chunk,
+                                        chela_dtype_t in_dtype, chela_dtype_t out_dtype, chela_norm_t norm, float norm_eps,
+                                        void *workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    if (!spectrum || (w_a != nullptr) != (w_o != nullptr)) return CHELA_ERR_INVALID_ARG;
+    return mixer_impl(x, w_short, short_width, nullptr, spectrum, w_q, w_k, w_v, b_q, b_k, b_v, w_a, b_a, w_o, b_o, qk_diag, v_silu, o,
+                      B, L, D, H, chunk, in_dtype, out_dtype, norm, norm_eps, workspace, workspace_bytes, stream);
 }
 
 chela_status_t chela_mixer_gated_fwd(const void *x, const float *w_short, int short_width, const float *k_long,
@@ -404,7 +443,7 @@ chela_status_t chela_mixer_gated_fwd(const void *x, const float *w_short, int sh
                                      cudaStream_t stream)
 {
     if (!w_a || !w_o) return CHELA_ERR_INVALID_ARG;
-    return mixer_impl(x, w_short, short_width, k_long, w_q, w_k, w_v, b_q, b_k, b_v, w_a, b_a, w_o, b_o, qk_diag, v_silu, u,
+    return mixer_impl(x, w_short, short_width, k_long, nullptr, w_q, w_k, w_v, b_q, b_k, b_v, w_a, b_a, w_o, b_o, qk_diag, v_silu, u,
                       B, L, D, H, chunk, in_dtype, out_dtype, norm, norm_eps, workspace, workspace_bytes, stream);
 }
 

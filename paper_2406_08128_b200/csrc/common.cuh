@@ -117,7 +117,10 @@ bool longconv_transposed_pair_supported(int L);
 int longconv_row_stride(int L);
 chela_status_t launch_longconv(const void *x, const float *k_long, const float *w_short, int short_width,
                                void *z, int B, int L, int D, chela_dtype_t in_dtype,
-                               chela_dtype_t out_dtype, void *workspace, cudaStream_t stream, bool transposed_pair = false);
+                               chela_dtype_t out_dtype, void *workspace, cudaStream_t stream, bool transposed_pair = false,
+                               const void *spectrum = nullptr);
+size_t longconv_spectrum_bytes(int L, int D);
+chela_status_t launch_longconv_prepare(const float *k_long, int L, int D, void *spectrum, cudaStream_t stream);
 
 // y[M,N] = act(a[M,K] w[K,N] + bias[N]); a: a_dtype, w: w_dtype, y: y_dtype.
 chela_status_t launch_gemm_simt(const void *a, const void *w, const float *bias, void *y, size_t M, int K,

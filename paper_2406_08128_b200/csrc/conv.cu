@@ -665,6 +665,13 @@ LongconvPlan longconv_plan(int B, int L, int D)
 }  // namespace
 
 size_t longconv_workspace_bytes(int B, int L, int D) { return longconv_plan(B, L, D).total; }
+// twiddle table followed by the kernel spectra, as launch_longconv_prepare writes them
+static size_t spectrum_off_spec(int L) { return align_up((size_t)longconv_plan(1, L, 1).M * sizeof(float2), 256); }
+size_t longconv_spectrum_bytes(int L, int D)
+{
+    const LongconvPlan p = longconv_plan(1, L, D);
+    return align_up(spectrum_off_spec(L) + (size_t)D * (p.M + 2) * sizeof(float2), 256);
+}
 int longconv_row_stride(int L) { return (int)align_up((size_t)L, 8); }
 // the FFT kernels that can write bf16 pair rows cover 2^10 .. 2^14 points
 bool longconv_transposed_pair_supported(int L) { return L > 512 && L <= 16384; }
@@ -683,18 +690,38 @@ static chela_status_t finish_longconv(const float *at, void *z, int B, int L, in
     return last_launch_status();
 }
 
+// The part of the long convolution that depends on the weights only (Eq. 6: the spectrum of each zero-padded kernel)
+// and the twiddle table, into a caller-owned buffer of longconv_spectrum_bytes(L, D).
+chela_status_t launch_longconv_prepare(const float *k_long, int L, int D, void *spectrum, cudaStream_t stream)
+{
+    const LongconvPlan p = longconv_plan(1, L, D);
+    float2 *tw = (float2 *)spectrum;
+    float2 *spec = (float2 *)((char *)spectrum + spectrum_off_spec(L));
+    twiddle_kernel<<<(p.M + 255) / 256, 256, 0, stream>>>(tw, p.M);
+    const int spec_stride = p.M + 2;
+    if (launch_fft_conv_fast(0, const_cast<float *>(k_long), L, L, D, D, p.logM, tw, spec, spec_stride, stream)) return last_launch_status();
+    const size_t smem = (size_t)(p.M + 256) * sizeof(float2);
+    int threads = p.M / 16;
+    threads = threads < 32 ? 32 : (threads > 1024 ? 1024 : threads);
+    if (cudaFuncSetAttribute(fft_conv_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return CHELA_ERR_CUDA;
+    fft_conv_kernel<0><<<D, threads, smem, stream>>>(const_cast<float *>(k_long), L, L, D, p.M, p.logM, tw, spec, spec_stride);
+    return last_launch_status();
+}
+
 chela_status_t launch_longconv(const void *x, const float *k_long, const float *w_short, int short_width,
                                void *z, int B, int L, int D, chela_dtype_t in_dtype,
-                               chela_dtype_t out_dtype, void *workspace, cudaStream_t stream, bool transposed_pair)
+                               chela_dtype_t out_dtype, void *workspace, cudaStream_t stream, bool transposed_pair,
+                               const void *spectrum)
 {
+    // spectrum: what launch_longconv_prepare wrote for these weights (k_long is then not read), else null
     // transposed_pair: z receives the rows as they leave the FFT kernel, [2][B][D][Ls] bf16 (hi plane, lo plane),
     // and the transpose back to token-major is skipped (the projections read this layout as a transposed operand)
     if (transposed_pair && !longconv_transposed_pair_supported(L)) return CHELA_ERR_UNSUPPORTED;
     const LongconvPlan p = longconv_plan(B, L, D);
     char *ws = (char *)workspace;
     float *at = (float *)(ws + p.off_at);
-    float2 *tw = (float2 *)(ws + p.off_tw);
-    float2 *spec = (float2 *)(ws + p.off_spec);
+    float2 *tw = spectrum ? (float2 *)spectrum : (float2 *)(ws + p.off_tw);
+    float2 *spec = spectrum ? (float2 *)((char *)spectrum + spectrum_off_spec(L)) : (float2 *)(ws + p.off_spec);
 
     dim3 g1((L + 63) / 64, (D + 31) / 32, B);
     const int wfast = w_short ? short_width : 0;
@@ -713,11 +740,11 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
                                                                      at, L, D, p.Ls);
     else
         conv_transpose_kernel<float><<<g1, 256, 0, stream>>>((const float *)x, w_short, short_width, at, L, D, p.Ls);
-    twiddle_kernel<<<(p.M + 255) / 256, 256, 0, stream>>>(tw, p.M);
+    if (!spectrum) twiddle_kernel<<<(p.M + 255) / 256, 256, 0, stream>>>(tw, p.M);
 
     // sizes 2^10 .. 2^14: the kernels with compile-time strides; other sizes: the generic kernel below
     const int spec_stride = p.M + 2;
-    if (launch_fft_conv_fast(0, const_cast<float *>(k_long), L, L, D, D, p.logM, tw, spec, spec_stride, stream) &&
+    if ((spectrum || launch_fft_conv_fast(0, const_cast<float *>(k_long), L, L, D, D, p.logM, tw, spec, spec_stride, stream)) &&
         launch_fft_conv_fast(1, at, p.Ls, L, D, B * D, p.logM, tw, spec, spec_stride, stream,
                              transposed_pair ? (__nv_bfloat16 *)z : nullptr, (size_t)B * D * p.Ls)) {
         if (transposed_pair) return last_launch_status();
@@ -731,7 +758,7 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(fft_conv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return CHELA_ERR_CUDA;
-    fft_conv_kernel<0><<<D, threads, smem, stream>>>(const_cast<float *>(k_long), L, L, D, p.M, p.logM, tw, spec, spec_stride);
+    if (!spectrum) fft_conv_kernel<0><<<D, threads, smem, stream>>>(const_cast<float *>(k_long), L, L, D, p.M, p.logM, tw, spec, spec_stride);
     fft_conv_kernel<1><<<B * D, threads, smem, stream>>>(at, p.Ls, L, D, p.M, p.logM, tw, spec, spec_stride);
     return finish_longconv(at, z, B, L, D, p.Ls, out_dtype, stream);
 }

@@ -128,3 +128,29 @@ def test_queued_mixer_calls_are_deterministic(B, L, D, H, chunk):
     assert chela.async_status(ws) == chela.OK
     for o in outs:
         assert torch.equal(first, o)
+
+
+@pytest.mark.parametrize("B,L,D,H", [(2, 1500, 128, 2), (1, 300, 64, 1), (1, 2048, 256, 4)])
+def test_prepared_spectra_give_the_same_mixer_and_long_convolution(B, L, D, H):
+    """chela_longconv_prepare + the *_prepared_fwd calls: the kernel spectra computed once for constant weights.  Same
+    kernels on the same spectra, so the outputs equal those of the unprepared calls bit for bit, and the oracle's
+    within the bound."""
+    import torch
+    m = inputs.mixer(11, B, L, D)
+    x, ws_, kl = to_device(m["x"], "bf16"), dev_f32(m["w_short"]), dev_f32(m["k_long"])
+    wq, wk, wv = (to_device(m[n], "bf16") for n in ("w_q", "w_k", "w_v"))
+    spec = chela.longconv_prepare(kl)
+    z0 = chela.longconv_fwd(x, kl, ws_)
+    z1 = chela.longconv_prepared_fwd(x, spec, ws_)
+    assert torch.equal(z0, z1)
+    assert rel_err(to_numpy(z1), oracle.longconv_fft(oracle.shortconv(m["x"], m["w_short"]), m["k_long"])) <= 2e-5
+    o0 = chela.mixer_fwd(x, ws_, kl, wq, wk, wv, H)
+    o1 = chela.mixer_prepared_fwd(x, ws_, spec, wq, wk, wv, H)
+    o2 = chela.mixer_prepared_fwd(x, ws_, spec, wq, wk, wv, H)   # the buffer is read, never written
+    assert torch.equal(o0, o1) and torch.equal(o1, o2)
+    assert rel_err(to_numpy(o1), oracle.mixer(m["x"], m["w_short"], m["k_long"], m["w_q"], m["w_k"], m["w_v"], H)) <= TOL
+    # a buffer that is too small, and the missing spectrum, are refused before anything is launched
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    assert chela.lib().chela_longconv_prepare(kl.data_ptr(), L, D, small.data_ptr(), small.numel(), None) == chela.ERR_WORKSPACE
+    with pytest.raises(chela.ChelaError):
+        chela.mixer_prepared_fwd(x, ws_, None, wq, wk, wv, H)
