@@ -22,9 +22,9 @@
 // traffic stays the algorithmic Q + K + V + O (measured), with no second kernel and no workspace.
 //
 // Warps (16): 0,1,4,5 output rows (add the halves, scale, normaliser, TMA store; 0,1 take the even own chunks, 4,5 the
-// odd ones); 8,9,12 score rows (mask, bf16, shared tile: a third of the live 64 x 64 triangle each); 10,11,14,15 state
-// rows (two warps per half of the columns); one issuing thread in each of 2 (G1), 3 (G2), 6 (G3 and the K^T V of chunks
-// that are not owned) and 7 (TMA producer).  A lone thread issues a tcgen05.mma about every 50 to 80 cycles and pays
+// odd ones); 2,3,6 score rows (mask, bf16, shared tile: a third of the live 64 x 64 triangle each); 10,11,14,15 state
+// rows (two warps per half of the columns); one issuing thread in each of 8 (G1), 9 (G2), 12 (G3 and the K^T V of chunks
+// that are not owned) and 13 (TMA producer).  A lone thread issues a tcgen05.mma about every 50 to 80 cycles and pays
 // the latency of every instruction between them, hence several issuers and no divisions in their loops.
 // Roles meet only through mbarriers, every wait bounded: on a timeout the CTA records CHELA_ERR_TIMEOUT, waits
 // (bounded) for its loads and products in flight, frees its TMEM and returns.

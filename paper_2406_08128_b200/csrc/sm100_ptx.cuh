@@ -45,14 +45,19 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within `limit` cycles, or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag, long long limit = kWaitCycles)
+// Bounded wait: false if the phase did not complete within `limit` cycles, or another role gave up.  The spin is out
+// of line: the roles of these kernels run long straight-line code, and every inlined spin loop is instruction-cache
+// footprint on their fast path.
+static __device__ __noinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, const volatile int *abort_flag, long long limit)
 {
-    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity))
         if (clock64() - t0 > limit || (abort_flag && *abort_flag)) return false;
     return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag, long long limit = kWaitCycles)
+{
+    return mbar_try_wait(bar, parity) || mbar_wait_spin(bar, parity, abort_flag, limit);
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
