@@ -235,6 +235,59 @@ def run_mixer_mode(args):
                                            "the long convolution (fp32 FFT on the plain ALUs) is inside the time"}}))
 
 
+def run_probe_mode(args):
+    """--probe NAME: a few calls of one small operation (the case the committed ncu summaries of that kernel were
+    captured on); prints one JSON line with its time.  NAME: shortconv, linattn_d128, decode_step, mixer_gated."""
+    import torch
+    from paper_2406_08128_b200 import build as _build, chela
+    _build.build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device=dev).manual_seed(7)
+    rnd = lambda *shape, s=1.0: (torch.randn(shape, device=dev, generator=gen) * s)
+    name = args.probe
+    if name == "shortconv":       # config 3's activations: 67 MB in, 67 MB out
+        x, w = rnd(4, 16384, 512).to(torch.bfloat16), rnd(512, 3, s=3 ** -0.5)
+        y = torch.empty_like(x)
+        step, work = (lambda: chela.shortconv_fwd(x, w, out=y)), "shortconv B=4 L=16384 D=512 width 3, bf16"
+    elif name == "linattn_d128":  # plain bf16, d = 128: 32768 tokens x 8 heads
+        q, k, v = (rnd(2, 16384, 8, 128, s=0.125).to(torch.bfloat16) for _ in range(3))
+        o = torch.empty(2, 16384, 8, 128, device=dev)
+        ws = torch.zeros(chela.linattn_workspace_bytes(2, 8, 16384, 128, 128, 128), dtype=torch.uint8, device=dev)
+        step, work = (lambda: chela.linattn_fwd(q, k, v, chunk=128, out=o, workspace=ws)), "linattn_fwd B=2 L=16384 H=8 d=128, bf16 in, fp32 out"
+    elif name == "decode_step":   # one token per sequence against the carried state
+        q, k, v = (rnd(256, 16, 64, s=0.125).to(torch.bfloat16) for _ in range(3))
+        states = [torch.zeros(256, 16, 64, 64, device=dev) for _ in range(3)]
+        o, it = torch.empty(256, 16, 64, device=dev), [0]
+
+        def step():
+            chela.linattn_step(q, k, v, states[it[0] % 3], out=o)
+            it[0] += 1
+        work = "linattn_step B=256 H=16 d=64, fp32 state"
+    elif name == "mixer_gated":   # a quarter of config 3
+        mb, ml, md, mh = 1, 16384, 512, 8
+        x = rnd(mb, ml, md).to(torch.bfloat16)
+        w_s = rnd(md, 3, s=3 ** -0.5)
+        k_l = rnd(md, ml) * torch.exp(-0.001 * torch.arange(ml, device=dev))[None, :]
+        w = [rnd(md, md, s=md ** -0.5).to(torch.bfloat16) for _ in range(5)]
+        ws = torch.zeros(chela.mixer_gated_workspace_bytes(mb, ml, md, mh, 64), dtype=torch.uint8, device=dev)
+        spec, o = chela.longconv_prepare(k_l), torch.empty(mb, ml, md, device=dev)
+        step = lambda: chela.mixer_prepared_fwd(x, w_s, spec, w[0], w[1], w[2], mh, w_a=w[3], w_o=w[4], out=o, workspace=ws)
+        work = "gated mixer B=1 L=16384 D=512 H=8, bf16 in, fp32 out, spectra prepared"
+    else:
+        raise SystemExit("unknown probe %r" % name)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    print(json.dumps({"probe": name, "workload": work, "steps": args.steps, "ms_per_step": e0.elapsed_time(e1) / args.steps}))
+
+
 def run_backward_mode(args):
     """--backward: one step = one chela_linattn_bwd call at the timed workload (normaliser on); one JSON line."""
     import torch
@@ -285,7 +338,12 @@ def main():
     ap.add_argument("--mixer", default=None, metavar="B,L,D,H,chunk",
                     help="time the whole token mixer (short conv, long conv, Q/K/V, attention) on this shape instead, "
                          "e.g. 4,16384,512,8,64 (config 3) or 8,8192,1024,8,128 (config 4); single GPU")
+    ap.add_argument("--probe", default=None, metavar="NAME",
+                    help="run a few calls of one small operation (shortconv, linattn_d128, decode_step, mixer_gated): the cases "
+                         "the committed ncu summaries were captured on")
     args = ap.parse_args()
+    if args.probe:
+        return run_probe_mode(args)
     if args.backward:
         run_backward_mode(args)
         return
