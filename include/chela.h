@@ -99,7 +99,9 @@ chela_status_t chela_shortconv_reparam(const float *w1, int width1, const float 
  * The product is evaluated with fp32 FFTs of size >= 2L (zero padded), so it is the causal
  * linear convolution, not the circular one.
  * x : [B, L, D] in_dtype.  k_long : [D, L] fp32.  w_short : [D, short_width] fp32 or NULL.
- * z : [B, L, D] out_dtype.  Supported: L <= 16384, D a multiple of 8.
+ * z : [B, L, D] out_dtype.  Supported: L <= 262144, D a multiple of 8.  Up to L = 16384 a row is transformed inside
+ * one SM's shared memory; longer rows are cut into blocks of 16384 tokens whose spectra pass through the workspace
+ * (2 x the row bytes more), one forward and one inverse transform per block and the block products in between.
  */
 size_t chela_longconv_workspace_bytes(int B, int L, int D, chela_dtype_t in_dtype,
                                       chela_dtype_t out_dtype);
@@ -254,7 +256,7 @@ chela_status_t chela_linattn_static_ws_status(cudaStream_t stream);
  *   O = per-head Norm(causal linear attention), head h = columns [h*D/H, (h+1)*D/H), scale 1.
  * x, o : [B, L, D] (in_dtype / out_dtype).  Dense weights : [D_in, D_out] row-major, in_dtype.
  * qk_diag scalers : [D], in_dtype.  Biases : [D] fp32 or NULL.  w_short : [D, short_width] fp32.
- * k_long : [D, L] fp32.  Supported: D/H in {64, 128}, chunk in {64, 128}, L <= 16384.
+ * k_long : [D, L] fp32.  Supported: D/H in {64, 128}, chunk in {64, 128}, L <= 262144.
  */
 size_t chela_mixer_workspace_bytes(int B, int L, int D, int H, int chunk, chela_dtype_t in_dtype);
 chela_status_t chela_mixer_fwd(const void *x, const float *w_short, int short_width,

@@ -6,6 +6,7 @@
 using namespace chela;
 
 namespace {
+constexpr int kLongconvMaxL = 262144;   // 16 blocks of the blocked long convolution
 
 bool dtype_ok(chela_dtype_t t) { return t == CHELA_F32 || t == CHELA_BF16; }
 
@@ -130,14 +131,14 @@ size_t chela_longconv_workspace_bytes(int B, int L, int D, chela_dtype_t, chela_
 
 size_t chela_longconv_spectrum_bytes(int L, int D)
 {
-    if (L < 1 || L > 16384 || D < 1 || D % 8 != 0) return 0;
+    if (L < 1 || L > kLongconvMaxL || D < 1 || D % 8 != 0) return 0;
     return longconv_spectrum_bytes(L, D);
 }
 
 chela_status_t chela_longconv_prepare(const float *k_long, int L, int D, void *spectrum, size_t spectrum_bytes, cudaStream_t stream)
 {
     if (!k_long || !spectrum || L < 1 || D < 1 || !aligned16(spectrum)) return CHELA_ERR_INVALID_ARG;
-    if (L > 16384 || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
+    if (L > kLongconvMaxL || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
     if (spectrum_bytes < longconv_spectrum_bytes(L, D)) return CHELA_ERR_WORKSPACE;
     return launch_longconv_prepare(k_long, L, D, spectrum, stream);
 }
@@ -149,7 +150,7 @@ chela_status_t chela_longconv_prepared_fwd(const void *x, const void *spectrum, 
     if (!x || !spectrum || !z || B < 1 || L < 1 || D < 1 || !dtype_ok(in_dtype) || !dtype_ok(out_dtype))
         return CHELA_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(z) || !aligned16(workspace) || !aligned16(spectrum)) return CHELA_ERR_INVALID_ARG;
-    if (L > 16384 || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
+    if (L > kLongconvMaxL || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
     if (w_short && (short_width < 1 || short_width > 16)) return CHELA_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < longconv_workspace_bytes(B, L, D)) return CHELA_ERR_WORKSPACE;
     return launch_longconv(x, nullptr, w_short, short_width, z, B, L, D, in_dtype, out_dtype, workspace, stream, false, spectrum);
@@ -163,7 +164,7 @@ chela_status_t chela_longconv_fwd(const void *x, const float *k_long, const floa
     if (!x || !k_long || !z || B < 1 || L < 1 || D < 1 || !dtype_ok(in_dtype) || !dtype_ok(out_dtype))
         return CHELA_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(z) || !aligned16(workspace)) return CHELA_ERR_INVALID_ARG;
-    if (L > 16384 || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
+    if (L > kLongconvMaxL || D % 8 != 0) return CHELA_ERR_UNSUPPORTED;
     if (w_short && (short_width < 1 || short_width > 16)) return CHELA_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < longconv_workspace_bytes(B, L, D)) return CHELA_ERR_WORKSPACE;
     return launch_longconv(x, k_long, w_short, short_width, z, B, L, D, in_dtype, out_dtype, workspace, stream);
@@ -321,7 +322,7 @@ chela_status_t mixer_impl(const void *x, const float *w_short, int short_width, 
         return CHELA_ERR_INVALID_ARG;
     if (D % H != 0) return CHELA_ERR_INVALID_ARG;
     const int d = D / H;
-    if ((d != 64 && d != 128) || (chunk != 64 && chunk != 128) || L > 16384 || short_width < 1 || short_width > 16)
+    if ((d != 64 && d != 128) || (chunk != 64 && chunk != 128) || L > kLongconvMaxL || short_width < 1 || short_width > 16)
         return CHELA_ERR_UNSUPPORTED;
     const MixerPlan p = mixer_plan(B, L, D, H, chunk, gated);
     if (!workspace || workspace_bytes < p.total) return CHELA_ERR_WORKSPACE;

@@ -588,6 +588,125 @@ __global__ void __launch_bounds__(1024) fft_conv_kernel(float *__restrict__ rows
     }
 }
 
+
+// ---- rows longer than one shared-memory FFT: the causal convolution by blocks of kBlockLen tokens (Eq. 6) ----------
+//
+// With x = (x_0, x_1, ...) and k = (k_0, k_1, ...) cut into blocks of kBlockLen, output block m is
+//   y_m = sum_{i+j=m} low(x_i * k_j) + sum_{i+j=m-1} high(x_i * k_j),
+// low/high = the two halves of the 2 kBlockLen-point linear convolution of two blocks.  Moving the high half onto the
+// low half is a rotation by half a period, i.e. a factor (-1)^f on the spectrum, so one inverse transform per output
+// block suffices:  y_m = low( IFFT( sum_{i+j=m} X_i K_j + (-1)^f sum_{i+j=m-1} X_i K_j ) ).
+// Block spectra go through global memory in the layout of fft_conv_kernel's mode 0 (M + 1 entries per block: position
+// p holds frequency bitrev(p), entry M the Nyquist term).
+constexpr int kBlockLen = 16384, kBlockM = 16384, kBlockLogM = 14;
+
+// spectrum of block j = blockIdx.y of row blockIdx.x; rows[row * row_stride + t], t < L
+__global__ void __launch_bounds__(1024) fft_block_spectrum_kernel(const float *__restrict__ rows, size_t row_stride, int L, int nb,
+                                                                  const float2 *__restrict__ tw_global, float2 *__restrict__ spec)
+{
+    constexpr int M = kBlockM, logM = kBlockLogM;
+    extern __shared__ __align__(16) float2 s[];
+    float2 *t1 = s + M, *t2 = t1 + 128;
+    for (int j = threadIdx.x; j < 128; j += blockDim.x) {
+        t1[j] = tw_global[j];
+        t2[j] = tw_global[128 * j];
+    }
+    const Twiddles tw = {t1, t2};
+    const int j = blockIdx.y;
+    const size_t row = blockIdx.x;
+    const float *x = rows + row * row_stride + (size_t)j * kBlockLen;
+    const int len = min(kBlockLen, L - j * kBlockLen);
+    for (int n = threadIdx.x; n < M; n += blockDim.x) {
+        const int t = 2 * n;
+        s[phys(n)] = make_float2(t < len ? x[t] : 0.f, t + 1 < len ? x[t + 1] : 0.f);
+    }
+    __syncthreads();
+    fft_forward_dif(s, tw, M, logM);
+    float2 *out = spec + (row * nb + j) * (size_t)(M + 2);
+    for (int pf = threadIdx.x; pf < M; pf += blockDim.x) {
+        const int f = bitrev(pf, logM);
+        if (f > (M >> 1)) continue;
+        const int pm = bitrev((M - f) & (M - 1), logM);
+        const float2 Cf = s[phys(pf)], Cm = s[phys(pm)];
+        const float2 E = make_float2(0.5f * (Cf.x + Cm.x), 0.5f * (Cf.y - Cm.y));
+        const float2 O = make_float2(0.5f * (Cf.y + Cm.y), -0.5f * (Cf.x - Cm.x));
+        const float2 wO = cmul(tw(f), O);
+        if (f == 0) {
+            out[0] = make_float2(E.x + O.x, 0.f);
+            out[M] = make_float2(E.x - O.x, 0.f);
+        } else {
+            out[pf] = cadd(E, wO);
+            out[pm] = cconj(csub(E, wO));
+        }
+    }
+}
+
+// output block m = blockIdx.y of row blockIdx.x, written over rows[row * row_stride + m * kBlockLen ...]
+__global__ void __launch_bounds__(1024) fft_block_combine_kernel(float *__restrict__ rows, size_t row_stride, int L, int D, int nb,
+                                                                 const float2 *__restrict__ tw_global,
+                                                                 const float2 *__restrict__ xspec, const float2 *__restrict__ kspec)
+{
+    constexpr int M = kBlockM, logM = kBlockLogM;
+    extern __shared__ __align__(16) float2 s[];
+    float2 *t1 = s + M, *t2 = t1 + 128;
+    for (int j = threadIdx.x; j < 128; j += blockDim.x) {
+        t1[j] = tw_global[j];
+        t2[j] = tw_global[128 * j];
+    }
+    __syncthreads();
+    const Twiddles tw = {t1, t2};
+    const int m = blockIdx.y;
+    const size_t row = blockIdx.x;
+    const size_t stride = (size_t)(M + 2);
+    const float2 *X = xspec + row * nb * stride, *K = kspec + (row % D) * nb * stride;
+    for (int pf = threadIdx.x; pf < M; pf += blockDim.x) {
+        const int f = bitrev(pf, logM);
+        if (f > (M >> 1)) continue;
+        const int pm = bitrev((M - f) & (M - 1), logM);
+        const float sgn = (f & 1) ? -1.f : 1.f;   // M - f has the parity of f
+        float2 Yf = make_float2(0.f, 0.f), Ym = make_float2(0.f, 0.f);
+        if (f == 0) {   // entries 0 (DC) and M (Nyquist), both real and of even frequency
+            for (int i = 0; i <= m; ++i) {
+                Yf.x += X[i * stride].x * K[(m - i) * stride].x;
+                Ym.x += X[i * stride + M].x * K[(m - i) * stride + M].x;
+            }
+            for (int i = 0; i < m; ++i) {
+                Yf.x += X[i * stride].x * K[(m - 1 - i) * stride].x;
+                Ym.x += X[i * stride + M].x * K[(m - 1 - i) * stride + M].x;
+            }
+        } else {
+            for (int i = 0; i <= m; ++i) {
+                Yf = cadd(Yf, cmul(X[i * stride + pf], K[(m - i) * stride + pf]));
+                Ym = cadd(Ym, cmul(X[i * stride + pm], K[(m - i) * stride + pm]));
+            }
+            float2 Hf = make_float2(0.f, 0.f), Hm = make_float2(0.f, 0.f);
+            for (int i = 0; i < m; ++i) {
+                Hf = cadd(Hf, cmul(X[i * stride + pf], K[(m - 1 - i) * stride + pf]));
+                Hm = cadd(Hm, cmul(X[i * stride + pm], K[(m - 1 - i) * stride + pm]));
+            }
+            Yf = make_float2(Yf.x + sgn * Hf.x, Yf.y + sgn * Hf.y);
+            Ym = make_float2(Ym.x + sgn * Hm.x, Ym.y + sgn * Hm.y);
+        }
+        // packed spectrum of the real result, as in fft_conv_kernel's mode 1
+        const float2 wf = tw(f);
+        const float2 Ep = make_float2(0.5f * (Yf.x + Ym.x), 0.5f * (Yf.y - Ym.y));
+        const float2 Dp = make_float2(0.5f * (Yf.x - Ym.x), 0.5f * (Yf.y + Ym.y));
+        const float2 Op = cmulc(Dp, wf);
+        s[phys(pf)] = make_float2(Ep.x - Op.y, Ep.y + Op.x);
+        if (pm != pf) s[phys(pm)] = make_float2(Ep.x + Op.y, -Ep.y + Op.x);
+    }
+    __syncthreads();
+    fft_inverse_dit(s, tw, M, logM);
+    const float inv = 1.0f / (float)M;
+    float *y = rows + row * row_stride + (size_t)m * kBlockLen;
+    const int len = min(kBlockLen, L - m * kBlockLen);
+    for (int n = threadIdx.x; 2 * n < len; n += blockDim.x) {
+        const float2 p = s[phys(n)];
+        y[2 * n] = p.x * inv;
+        if (2 * n + 1 < len) y[2 * n + 1] = p.y * inv;
+    }
+}
+
 }  // namespace
 
 namespace {
@@ -646,21 +765,34 @@ chela_status_t launch_shortconv_reparam(const float *w1, int width1, const float
 
 namespace {
 struct LongconvPlan {
-    int M, logM, Ls;
-    size_t off_at, off_tw, off_spec, total;
+    int M, logM, Ls, nb;   // nb > 1: the blocked path (L > kBlockLen), M = kBlockM points per block
+    size_t off_at, off_tw, off_spec, off_xspec, total;
 };
 LongconvPlan longconv_plan(int B, int L, int D)
 {
     LongconvPlan p;
-    p.M = next_pow2(L) < 16 ? 16 : next_pow2(L);
+    p.nb = (L + kBlockLen - 1) / kBlockLen;
+    if (p.nb < 1) p.nb = 1;
+    p.M = p.nb > 1 ? kBlockM : (next_pow2(L) < 16 ? 16 : next_pow2(L));
     p.logM = 0;
     while ((1 << p.logM) < p.M) ++p.logM;
     p.Ls = (int)align_up((size_t)L, 8);
     p.off_at = 0;
     p.off_tw = align_up(p.off_at + (size_t)B * D * p.Ls * sizeof(float), 256);
     p.off_spec = align_up(p.off_tw + (size_t)p.M * sizeof(float2), 256);
-    p.total = align_up(p.off_spec + (size_t)D * (p.M + 2) * sizeof(float2), 256);   // rows of M + 1 entries, 16-byte aligned
+    // kernel spectra: rows of M + 1 entries, 16-byte aligned, one per (channel, block)
+    p.off_xspec = align_up(p.off_spec + (size_t)D * p.nb * (p.M + 2) * sizeof(float2), 256);
+    // blocked path only: the spectra of the data blocks
+    p.total = p.nb > 1 ? align_up(p.off_xspec + (size_t)B * D * p.nb * (p.M + 2) * sizeof(float2), 256) : p.off_xspec;
     return p;
+}
+const size_t kBlockSmem = (size_t)(kBlockM + 256) * sizeof(float2);
+chela_status_t block_kernels_ready()
+{
+    if (cudaFuncSetAttribute(fft_block_spectrum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBlockSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(fft_block_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBlockSmem) != cudaSuccess)
+        return CHELA_ERR_CUDA;
+    return CHELA_OK;
 }
 }  // namespace
 
@@ -670,7 +802,7 @@ static size_t spectrum_off_spec(int L) { return align_up((size_t)longconv_plan(1
 size_t longconv_spectrum_bytes(int L, int D)
 {
     const LongconvPlan p = longconv_plan(1, L, D);
-    return align_up(spectrum_off_spec(L) + (size_t)D * (p.M + 2) * sizeof(float2), 256);
+    return align_up(spectrum_off_spec(L) + (size_t)D * p.nb * (p.M + 2) * sizeof(float2), 256);
 }
 int longconv_row_stride(int L) { return (int)align_up((size_t)L, 8); }
 // the FFT kernels that can write bf16 pair rows cover 2^10 .. 2^14 points
@@ -698,6 +830,11 @@ chela_status_t launch_longconv_prepare(const float *k_long, int L, int D, void *
     float2 *tw = (float2 *)spectrum;
     float2 *spec = (float2 *)((char *)spectrum + spectrum_off_spec(L));
     twiddle_kernel<<<(p.M + 255) / 256, 256, 0, stream>>>(tw, p.M);
+    if (p.nb > 1) {
+        if (block_kernels_ready() != CHELA_OK) return CHELA_ERR_CUDA;
+        fft_block_spectrum_kernel<<<dim3(D, p.nb), 1024, kBlockSmem, stream>>>(k_long, (size_t)L, L, p.nb, tw, spec);
+        return last_launch_status();
+    }
     const int spec_stride = p.M + 2;
     if (launch_fft_conv_fast(0, const_cast<float *>(k_long), L, L, D, D, p.logM, tw, spec, spec_stride, stream)) return last_launch_status();
     const size_t smem = (size_t)(p.M + 256) * sizeof(float2);
@@ -742,6 +879,15 @@ chela_status_t launch_longconv(const void *x, const float *k_long, const float *
         conv_transpose_kernel<float><<<g1, 256, 0, stream>>>((const float *)x, w_short, short_width, at, L, D, p.Ls);
     if (!spectrum) twiddle_kernel<<<(p.M + 255) / 256, 256, 0, stream>>>(tw, p.M);
 
+    if (p.nb > 1) {   // longer than one shared-memory row: block spectra through global memory
+        if (transposed_pair) return CHELA_ERR_UNSUPPORTED;
+        if (block_kernels_ready() != CHELA_OK) return CHELA_ERR_CUDA;
+        float2 *xspec = (float2 *)(ws + p.off_xspec);
+        if (!spectrum) fft_block_spectrum_kernel<<<dim3(D, p.nb), 1024, kBlockSmem, stream>>>(k_long, (size_t)L, L, p.nb, tw, spec);
+        fft_block_spectrum_kernel<<<dim3(B * D, p.nb), 1024, kBlockSmem, stream>>>(at, (size_t)p.Ls, L, p.nb, tw, xspec);
+        fft_block_combine_kernel<<<dim3(B * D, p.nb), 1024, kBlockSmem, stream>>>(at, (size_t)p.Ls, L, D, p.nb, tw, xspec, spec);
+        return finish_longconv(at, z, B, L, D, p.Ls, out_dtype, stream);
+    }
     // sizes 2^10 .. 2^14: the kernels with compile-time strides; other sizes: the generic kernel below
     const int spec_stride = p.M + 2;
     if ((spectrum || launch_fft_conv_fast(0, const_cast<float *>(k_long), L, L, D, D, p.logM, tw, spec, spec_stride, stream)) &&

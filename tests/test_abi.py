@@ -76,7 +76,7 @@ def test_invalid_arguments_rejected_without_gpu(lib):
     assert L.chela_shortconv_fwd(one, one, null, two, 1, 8, 8, 17, 1, 1, null) == chela.ERR_UNSUPPORTED
     assert L.chela_shortconv_fwd(one, one, null, two, 1, 8, 12, 3, 1, 1, null) == chela.ERR_UNSUPPORTED
     # long conv: length limit and workspace
-    assert L.chela_longconv_fwd(one, one, null, 0, two, 1, 32768, 8, 1, 0, two, 1 << 40, null) == chela.ERR_UNSUPPORTED
+    assert L.chela_longconv_fwd(one, one, null, 0, two, 1, 262145, 8, 1, 0, two, 1 << 40, null) == chela.ERR_UNSUPPORTED
     assert L.chela_longconv_fwd(one, one, null, 0, two, 1, 64, 8, 1, 0, null, 0, null) == chela.ERR_WORKSPACE
     assert L.chela_longconv_fwd(one, one, null, 0, two, 1, 64, 8, 1, 0, two, 16, null) == chela.ERR_WORKSPACE
     # mixer: D not divisible by H, head dim unsupported, workspace too small

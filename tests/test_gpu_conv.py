@@ -48,6 +48,28 @@ def test_longconv_against_direct_and_fft_oracle(B, L, D, fused_short):
     assert np.allclose(z[:, 0], k_long[:, 0] * a[:, 0], rtol=1e-4, atol=1e-4)
 
 
+@pytest.mark.parametrize("B,L,D", [(1, 16385, 8), (1, 32768, 8), (2, 40000, 16), (1, 65536, 8), (1, 100000, 8)])
+@pytest.mark.parametrize("fused_short", [False, True])
+def test_longconv_longer_than_one_shared_memory_row(B, L, D, fused_short):
+    """Rows beyond 16384 tokens go block by block with the block spectra in the workspace (Eq. 6 has no length limit);
+    also through the prepared-spectra entry point."""
+    m = inputs.mixer(900 + L, B, L, D, dtype="bf16", decay=0.0002)
+    x, k_long, w_short = m["x"], m["k_long"], m["w_short"]
+    ws = dev_f32(w_short) if fused_short else None
+    z = to_numpy(chela.longconv_fwd(to_device(x, "bf16"), dev_f32(k_long), ws))
+    a = oracle.shortconv(x, w_short, act=True) if fused_short else x.astype(np.float64)
+    ref = oracle.longconv_fft(a, k_long)
+    assert rel_err(z, ref) <= 2e-5
+    # every block boundary carries the tails of the blocks before it: check the samples around each on their own
+    for t0 in range(16384, L, 16384):
+        sl = slice(t0 - 4, min(L, t0 + 4))
+        assert np.abs(z[:, sl] - ref[:, sl]).max() <= 2e-5 * np.abs(ref).max()
+    assert np.allclose(z[:, 0], k_long[:, 0] * a[:, 0], rtol=1e-4, atol=1e-4)
+    spec = chela.longconv_prepare(dev_f32(k_long))
+    z2 = to_numpy(chela.longconv_prepared_fwd(to_device(x, "bf16"), spec, ws))
+    assert np.array_equal(z2, z)
+
+
 def test_longconv_f32_input_and_bf16_output():
     B, L, D = 2, 300, 16
     m = inputs.mixer(7, B, L, D, dtype="f32")

@@ -94,6 +94,32 @@ def test_gated_mixer(B, L, D, H, chunk, dtype):
     assert rel_err(to_numpy(u), ref) <= TOL
 
 
+@pytest.mark.parametrize("seed,B,L,D,H,chunk", [(12, 4, 16384, 512, 8, 64), (13, 8, 8192, 1024, 8, 128)])
+def test_gated_mixer_configs_3_and_4_full_size_sampled_rows(seed, B, L, D, H, chunk):
+    """The gated call (Eqs. 8, 9, 13, 14) at the full sizes of configs 3 and 4; the oracle checks the first and last batch row."""
+    m = inputs.mixer(seed, B, L, D)
+    rng = np.random.default_rng(seed + 100)
+    w_a, w_o = (inputs.round_storage(rng.standard_normal((D, D), dtype=np.float32) / np.sqrt(D) / 12, "bf16") for _ in range(2))
+    b_a, b_o = (rng.standard_normal(D, dtype=np.float32) * 0.5 for _ in range(2))
+    dev = lambda a: to_device(a, "bf16")
+    u = to_numpy(chela.mixer_gated_fwd(dev(m["x"]), dev_f32(m["w_short"]), dev_f32(m["k_long"]), dev(m["w_q"]), dev(m["w_k"]),
+                                       dev(m["w_v"]), dev(w_a), dev(w_o), H, chunk=chunk, b_a=dev_f32(b_a), b_o=dev_f32(b_o)))
+    assert np.isfinite(u).all()
+    for b in (0, B - 1):
+        ref = oracle.mixer_gated(m["x"][b:b + 1], m["w_short"], m["k_long"], m["w_q"], m["w_k"], m["w_v"], w_a, w_o, H,
+                                 b_a=b_a, b_o=b_o)
+        assert rel_err(u[b:b + 1], ref) <= TOL, b
+
+
+@pytest.mark.parametrize("B,L,D,H", [(1, 32768, 128, 2), (2, 40000, 128, 1)])
+def test_mixer_on_sequences_longer_than_one_fft_row(B, L, D, H):
+    """L > 16384: the long convolution goes block by block; the rest of the layer is the same path."""
+    m = inputs.mixer(21, B, L, D, decay=0.0003)
+    got = run_mixer(m, H, 64)
+    ref = oracle.mixer(m["x"], m["w_short"], m["k_long"], m["w_q"], m["w_k"], m["w_v"], H)
+    assert rel_err(got, ref) <= TOL
+
+
 def test_mixer_call_can_be_captured_in_a_cuda_graph():
     import torch
     B, L, D, H = 1, 2048, 512, 8
