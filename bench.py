@@ -209,6 +209,10 @@ def run_mixer_mode(args):
     out = torch.empty(mb, ml, md, device=dev)
     spec = chela.longconv_prepare(k_l)   # the long kernels' spectra: weights do not change between steps
     step = lambda: chela.mixer_prepared_fwd(x, w_s, spec, w_q, w_k, w_v, mh, chunk=mc, out=out, workspace=ws)
+    if args.gated:   # Eqs. 8, 13, 14: two more projections, gates applied in the attention kernel's store
+        w_a, w_o = [(torch.randn(md, md, device=dev, generator=gen) / md ** 0.5 / 12).to(torch.bfloat16) for _ in range(2)]
+        ws = torch.zeros(chela.mixer_gated_workspace_bytes(mb, ml, md, mh, mc), dtype=torch.uint8, device=dev)
+        step = lambda: chela.mixer_prepared_fwd(x, w_s, spec, w_q, w_k, w_v, mh, w_a=w_a, w_o=w_o, chunk=mc, out=out, workspace=ws)
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -223,7 +227,7 @@ def run_mixer_mode(args):
     ms = e0.elapsed_time(e1) / args.steps
     peaks, peak_kind = measured_peaks()
     d_head = md // mh
-    flops_tok = mixer_flops_per_token(md, mh)
+    flops_tok = mixer_flops_per_token(md, mh, gated=args.gated)
     achieved = flops_tok * mb * ml / (ms * 1e-3) / 1e12
     print(json.dumps({"metric": "mixer_fwd_tokens_per_s", "value": mb * ml / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
                       "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
@@ -338,6 +342,7 @@ def main():
     ap.add_argument("--mixer", default=None, metavar="B,L,D,H,chunk",
                     help="time the whole token mixer (short conv, long conv, Q/K/V, attention) on this shape instead, "
                          "e.g. 4,16384,512,8,64 (config 3) or 8,8192,1024,8,128 (config 4); single GPU")
+    ap.add_argument("--gated", action="store_true", help="with --mixer: the gated call (two more projections, gates in the attention store)")
     ap.add_argument("--probe", default=None, metavar="NAME",
                     help="run a few calls of one small operation (shortconv, linattn_d128, decode_step, mixer_gated): the cases "
                          "the committed ncu summaries were captured on")
