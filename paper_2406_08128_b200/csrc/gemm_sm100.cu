@@ -194,18 +194,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                     // (test hook: the first hand-back of CTA 0 left out, so that the issuer's wait for it runs out)
                     if (lane == 0 && !(wc.skip_arrival && blockIdx.x == 0 && ti == 0 && warp == 0)) mbar_arrive(bar_tempty0 + 8 * buf);
                 }
-                // the staging buffer is free once the store that last used it has been read (two boxes ago with
-                // ping-pong buffers, the previous box with one)
-                if (lane == 0) {
-                    if (Smem::kStagingBufs == 2) bulk_wait_read1();
-                    else bulk_wait_read0();
-                }
-                __syncwarp();
-                const int sb = Smem::kStagingBufs == 2 ? (nbox & 1) : 0;
-                uint8_t *hi = stg + sb * (2 * 32 * 128), *lo = hi + 32 * 128;
+                // bias, activation and the hi/lo split first, into registers: the store of the previous box is still
+                // reading the staging buffer meanwhile
+                uint32_t wh[8][4], wl[8][4];
 #pragma unroll
                 for (int j8 = 0; j8 < 8; ++j8) {
-                    uint32_t wh[4], wl[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const int col = j8 * 8 + e * 2;
@@ -219,15 +212,27 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                             x1 = activate(x1, act);
                         }
                         const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
-                        wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                        wh[j8][e] = *reinterpret_cast<const uint32_t *>(&hh);
                         if (kYPair) {
                             const float2 hf = __bfloat1622float2(hh);
-                            wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                            wl[j8][e] = pack_bf16(x0 - hf.x, x1 - hf.y);
                         }
                     }
+                }
+                // the staging buffer is free once the store that last used it has been read (two boxes ago with
+                // ping-pong buffers, the previous box with one)
+                if (lane == 0) {
+                    if (Smem::kStagingBufs == 2) bulk_wait_read1();
+                    else bulk_wait_read0();
+                }
+                __syncwarp();
+                const int sb = Smem::kStagingBufs == 2 ? (nbox & 1) : 0;
+                uint8_t *hi = stg + sb * (2 * 32 * 128), *lo = hi + 32 * 128;
+#pragma unroll
+                for (int j8 = 0; j8 < 8; ++j8) {
                     const uint32_t off = sw128(lane, j8);
-                    *reinterpret_cast<uint4 *>(hi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
-                    if (kYPair) *reinterpret_cast<uint4 *>(lo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                    *reinterpret_cast<uint4 *>(hi + off) = make_uint4(wh[j8][0], wh[j8][1], wh[j8][2], wh[j8][3]);
+                    if (kYPair) *reinterpret_cast<uint4 *>(lo + off) = make_uint4(wl[j8][0], wl[j8][1], wl[j8][2], wl[j8][3]);
                 }
                 fence_proxy_async();
                 __syncwarp();
