@@ -382,7 +382,7 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             tmem_ld32(tmem_warp + col, t);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < kCols; ++j) sv[j] += t[j];
+            for (int j = 0; j < kCols; j += 2) add2(sv[j], sv[j + 1], t[j], t[j + 1]);
         };
         bool ok = true;
         if (lane == 0) {   // both accumulators start free
@@ -411,8 +411,10 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                         const float x0 = sv[c8 * 8 + e * 2], x1 = sv[c8 * 8 + e * 2 + 1];
                         const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
                         const float2 hf = __bfloat1622float2(hh);
+                        float l0, l1;
+                        sub2(l0, l1, x0, x1, hf.x, hf.y);
                         wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
-                        wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                        wl[e] = pack_bf16(l0, l1);
                     }
                     const uint32_t off = sw128(r, c0 / 8 + c8);
                     *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
@@ -467,19 +469,19 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 tmem_ld32(tmem_warp + kColOS + 128 * buf + 64 + 32 * hc, lo);
                 tmem_ld_wait();
 #pragma unroll
-                for (int c = 0; c < 32; ++c) acc[32 * hc + c] += lo[c];
+                for (int c = 0; c < 32; c += 2) add2(acc[32 * hc + c], acc[32 * hc + c + 1], lo[c], lo[c + 1]);
             }
             zero_lo();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_of + 8 * buf);   // the output rows are out of TMEM
-            float ss = 0.f;
+            // the row is scaled and normalised in one multiplication: o = acc * scale / sqrt(scale^2 mean(acc^2) + eps)
+            float ss0 = 0.f, ss1 = 0.f;
 #pragma unroll
-            for (int c = 0; c < kD; ++c) {
-                acc[c] *= scale;
-                ss = fmaf(acc[c], acc[c], ss);
-            }
-            const float inv = norm ? rsqrtf(ss * (1.0f / kD) + eps) : 1.0f;
+            for (int c = 0; c < kD; c += 2) sqacc2(ss0, ss1, acc[c], acc[c + 1]);
+            const float inv = norm ? scale * rsqrtf((ss0 + ss1) * (scale * scale * (1.0f / kD)) + eps) : scale;
+#pragma unroll
+            for (int c = 0; c < kD; c += 2) mul2(acc[c], acc[c + 1], acc[c], acc[c + 1], inv);
             // this warp's 32 rows x 128 bytes of the set's staging tile, one 128-byte wide box after the other
             uint8_t *sO = smem + SM::offO + buf * kTile;
 #pragma unroll
@@ -490,13 +492,13 @@ linattn_sm100_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
 #pragma unroll
                     for (int c = 0; c < 32; c += 4)
                         *reinterpret_cast<float4 *>(sO + sw128(r, c / 4)) =
-                            make_float4(acc[32 * bx + c] * inv, acc[32 * bx + c + 1] * inv, acc[32 * bx + c + 2] * inv, acc[32 * bx + c + 3] * inv);
+                            make_float4(acc[32 * bx + c], acc[32 * bx + c + 1], acc[32 * bx + c + 2], acc[32 * bx + c + 3]);
                 } else {
 #pragma unroll
                     for (int c = 0; c < kD; c += 8)
                         *reinterpret_cast<uint4 *>(sO + sw128(r, c / 8)) =
-                            make_uint4(pack_bf16(acc[c] * inv, acc[c + 1] * inv), pack_bf16(acc[c + 2] * inv, acc[c + 3] * inv),
-                                       pack_bf16(acc[c + 4] * inv, acc[c + 5] * inv), pack_bf16(acc[c + 6] * inv, acc[c + 7] * inv));
+                            make_uint4(pack_bf16(acc[c], acc[c + 1]), pack_bf16(acc[c + 2], acc[c + 3]),
+                                       pack_bf16(acc[c + 4], acc[c + 5]), pack_bf16(acc[c + 6], acc[c + 7]));
                 }
                 fence_proxy_async();
                 __syncwarp();

@@ -225,6 +225,28 @@ __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_
 // ---- small device helpers ---------------------------------------------------------------------
 
 // byte offset of element (row, 16-byte chunk) inside a 128-byte-swizzled [rows] x 128 B tile
+// Two-wide fp32 arithmetic (one instruction for a pair of lanes' values): a += b, a *= s, acc += a * a.
+__device__ __forceinline__ void add2(float &a0, float &a1, float b0, float b1)
+{
+    asm("{ .reg .b64 x, y; mov.b64 x, {%0, %1}; mov.b64 y, {%2, %3}; add.rn.f32x2 x, x, y; mov.b64 {%0, %1}, x; }"
+        : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void sub2(float &d0, float &d1, float a0, float a1, float b0, float b1)
+{
+    asm("{ .reg .b64 x, y; mov.b64 x, {%2, %3}; mov.b64 y, {%4, %5}; sub.rn.f32x2 x, x, y; mov.b64 {%0, %1}, x; }"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void mul2(float &d0, float &d1, float a0, float a1, float s)
+{
+    asm("{ .reg .b64 x, y; mov.b64 x, {%2, %3}; mov.b64 y, {%4, %4}; mul.rn.f32x2 x, x, y; mov.b64 {%0, %1}, x; }"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(s));
+}
+__device__ __forceinline__ void sqacc2(float &s0, float &s1, float a0, float a1)
+{
+    asm("{ .reg .b64 x, y; mov.b64 x, {%2, %3}; mov.b64 y, {%0, %1}; fma.rn.f32x2 y, x, x, y; mov.b64 {%0, %1}, y; }"
+        : "+f"(s0), "+f"(s1) : "f"(a0), "f"(a1));
+}
+
 __device__ __forceinline__ uint32_t sw128(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
