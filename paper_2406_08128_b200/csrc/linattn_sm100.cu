@@ -403,13 +403,26 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     bulk_wait_read0();      // this warp's previous output boxes have left shared memory
                 }
                 __syncwarp();
-                float ss = 0.f;
+                float inv;
+                if (kGrad) {   // the pull-back below needs the scaled row r itself
+                    float ss = 0.f;
 #pragma unroll
-                for (int j = 0; j < kD; ++j) {
-                    acc[j] *= scale;
-                    ss = fmaf(acc[j], acc[j], ss);
+                    for (int j = 0; j < kD; ++j) {
+                        acc[j] *= scale;
+                        ss = fmaf(acc[j], acc[j], ss);
+                    }
+                    inv = norm ? rsqrtf(ss * (1.0f / kD) + eps) : 1.0f;
+                } else {
+                    // scaled and normalised in one multiplication, o = acc * scale / sqrt(scale^2 mean(acc^2) + eps),
+                    // with two-wide fp32 instructions; the stores below then take the row as it is
+                    float ss0 = 0.f, ss1 = 0.f;
+#pragma unroll
+                    for (int j = 0; j < kD; j += 2) sqacc2(ss0, ss1, acc[j], acc[j + 1]);
+                    const float f = norm ? scale * rsqrtf((ss0 + ss1) * (scale * scale * (1.0f / kD)) + eps) : scale;
+#pragma unroll
+                    for (int j = 0; j < kD; j += 2) mul2(acc[j], acc[j + 1], acc[j], acc[j + 1], f);
+                    inv = 1.0f;
                 }
-                const float inv = norm ? rsqrtf(ss * (1.0f / kD) + eps) : 1.0f;
                 uint8_t *sO = smem + SM::offO;
                 if (kGrad) {
                     // acc = r (scaled); o = r inv; G = scale (d_o - o <o, d_o> / d) inv, stored as hi and lo planes
