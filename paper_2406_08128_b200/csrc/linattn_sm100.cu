@@ -293,8 +293,10 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const float x0 = sv[c8 * 8 + e * 2], x1 = sv[c8 * 8 + e * 2 + 1];
                     const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
                     const float2 hf = __bfloat1622float2(hh);
+                    float l0, l1;
+                    sub2(l0, l1, x0, x1, hf.x, hf.y);
                     wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
-                    wl[e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+                    wl[e] = pack_bf16(l0, l1);
                 }
                 const uint32_t off = sw128(r, c8);
                 *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
