@@ -232,7 +232,7 @@ void chela_debug_wait_control(long long limit_cycles, int skip_arrival);
  *     split sequence, up to one group per SM: B*H = 1 with L above about 130 000 tokens needs more than 8 MiB on a
  *     148-SM part and is refused.
  *   - The first call on each device looks up the device address of the built-in array (with that device
- *     current) and caches it; make that first call during set-up, before any stream capture.
+ *     current) and caches it; make that first call during set-up.
  *   - The call itself calls no cudaMalloc / cudaFree and no allocating library routine.
  *   - All calls on one GPU share the one array, which keeps the previous call's contents.  Nothing in it
  *     needs to start at zero except the status word, which each launch clears on `stream` itself.  Two
