@@ -249,9 +249,9 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         };
         if (has_init) {
             if (upper) {
-#pragma unroll
+#pragma unroll 1
                 for (int x = 0; x < 2; ++x)
-#pragma unroll
+#pragma unroll 1
                     for (int half = 0; half < 2; ++half) {
                         float sv[64];
 #pragma unroll
@@ -366,9 +366,9 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 }
             } else if (i + 1 < nchunks) {
                 // ---- state rows d_k = r (from OS_a) and d_k = 64 + r (from S_b): bf16 hi + lo -> shared --------
-#pragma unroll
+#pragma unroll 1
                 for (int x = 0; x < 2; ++x)
-#pragma unroll
+#pragma unroll 1
                     for (int half = 0; half < 2; ++half) {
                         float sv[64];
                         const uint32_t col = (x == 0 ? kColOS : kColSb) + 64 * half;
@@ -383,9 +383,9 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 if (lane == 0) mbar_arrive(bar_s);
             } else if (state_out && g == G - 1) {
                 // last chunk of the sequence: the fp32 state leaves the SM once, for the caller
-#pragma unroll
+#pragma unroll 1
                 for (int x = 0; x < 2; ++x)
-#pragma unroll
+#pragma unroll 1
                     for (int half = 0; half < 2; ++half) {
                         float sv[64];
                         const uint32_t col = (x == 0 ? kColOS : kColSb) + 64 * half;
