@@ -303,6 +303,27 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
             }
         };
+        // the same for one half of the row (32 columns: pieces 4 * hf .. 4 * hf + 3), for the per-chunk loop below
+        auto write_state_half = [&](const float(&sv)[32], int hf) {
+            uint8_t *sHi = smem + SM::offShi, *sLo = smem + SM::offSlo;
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {
+                uint32_t wh[4], wl[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float x0 = sv[c8 * 8 + e * 2], x1 = sv[c8 * 8 + e * 2 + 1];
+                    const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                    const float2 hf2 = __bfloat1622float2(hh);
+                    float l0, l1;
+                    sub2(l0, l1, x0, x1, hf2.x, hf2.y);
+                    wh[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                    wl[e] = pack_bf16(l0, l1);
+                }
+                const uint32_t off = sw128(r, 4 * hf + c8);
+                *reinterpret_cast<uint4 *>(sHi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+            }
+        };
         if (has_init) {
             // initial state of the group: sum of the preceding groups' K^T V, into TMEM rows 64..127 and
             // into the G2 operand tiles
@@ -481,10 +502,14 @@ linattn_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             } else {
                 // ---- state row d_k: bf16 hi + lo -> shared (MN-major B operand of the next chunk's G2) ------
                 if (i + 1 < nchunks) {
-                    tmem_ld32(tmem_warp + kColOS, *reinterpret_cast<float(*)[32]>(&acc[0]));
-                    tmem_ld32(tmem_warp + kColOS + 32, *reinterpret_cast<float(*)[32]>(&acc[32]));
-                    tmem_ld_wait();
-                    write_state_tiles(acc);
+                    // (a loop over the two halves, not unrolled: the per-chunk code of these warps stays small)
+#pragma unroll 1
+                    for (int hf = 0; hf < 2; ++hf) {
+                        float sv[32];
+                        tmem_ld32(tmem_warp + kColOS + 32 * hf, sv);
+                        tmem_ld_wait();
+                        write_state_half(sv, hf);
+                    }
                     fence_proxy_async();
                     tc_fence_before();
                     __syncwarp();
