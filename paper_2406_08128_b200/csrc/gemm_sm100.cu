@@ -44,6 +44,36 @@ struct Smem {
     static_assert(bytes <= 232448, "shared memory per CTA");
 };
 
+// One box of the epilogue: 64 accumulator values of a row -> bias, activation ACT, bf16 (hi) and the rounding remainder
+// (lo).  The activation is a template argument and the caller branches once per box: with a run-time switch per element
+// the box's code is three times as long and the epilogue warps wait for instruction fetches.
+template <int ACT, bool kYPair>
+__device__ __forceinline__ void pack_box(const float (&acc)[64], const float *__restrict__ bias, uint32_t (&wh)[8][4], uint32_t (&wl)[8][4])
+{
+#pragma unroll
+    for (int j8 = 0; j8 < 8; ++j8) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int col = j8 * 8 + e * 2;
+            float x0 = acc[col], x1 = acc[col + 1];
+            if (bias) {
+                x0 += bias[col];
+                x1 += bias[col + 1];
+            }
+            if (ACT) {
+                x0 = activate(x0, ACT);
+                x1 = activate(x1, ACT);
+            }
+            const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+            wh[j8][e] = *reinterpret_cast<const uint32_t *>(&hh);
+            if (kYPair) {
+                const float2 hf = __bfloat1622float2(hh);
+                wl[j8][e] = pack_bf16(x0 - hf.x, x1 - hf.y);
+            }
+        }
+    }
+}
+
 // kATrans: A is given transposed, [B][K][Lt] per plane (the long convolution's row layout: channel-major, tokens
 // contiguous); its tiles are then MN-major like W's, two 64-token atoms per 128-row tile, and row tile m0 lies in
 // batch m0 / Lt at token m0 % Lt (Lt a multiple of 128).
@@ -197,28 +227,10 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tm_a_hi, const __grid_cons
                 // bias, activation and the hi/lo split first, into registers: the store of the previous box is still
                 // reading the staging buffer meanwhile
                 uint32_t wh[8][4], wl[8][4];
-#pragma unroll
-                for (int j8 = 0; j8 < 8; ++j8) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int col = j8 * 8 + e * 2;
-                        float x0 = acc[col], x1 = acc[col + 1];
-                        if (bias) {
-                            x0 += bias[n0 + c * 64 + col];
-                            x1 += bias[n0 + c * 64 + col + 1];
-                        }
-                        if (act) {
-                            x0 = activate(x0, act);
-                            x1 = activate(x1, act);
-                        }
-                        const __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
-                        wh[j8][e] = *reinterpret_cast<const uint32_t *>(&hh);
-                        if (kYPair) {
-                            const float2 hf = __bfloat1622float2(hh);
-                            wl[j8][e] = pack_bf16(x0 - hf.x, x1 - hf.y);
-                        }
-                    }
-                }
+                const float *bias_box = bias ? bias + n0 + c * 64 : nullptr;
+                if (act == 0) pack_box<0, kYPair>(acc, bias_box, wh, wl);
+                else if (act == 1) pack_box<1, kYPair>(acc, bias_box, wh, wl);
+                else pack_box<2, kYPair>(acc, bias_box, wh, wl);
                 // the staging buffer is free once the store that last used it has been read (two boxes ago with
                 // ping-pong buffers, the previous box with one)
                 if (lane == 0) {
