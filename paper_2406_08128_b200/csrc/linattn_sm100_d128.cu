@@ -176,24 +176,26 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 {
                     const uint32_t pt_hi = sbase + SM::offPT, pt_lo = pt_hi + kTile;
                     const uint32_t v_hi = desc_lo(tile(i, 0, 4), kTile);
-                    // OS_a: [P^T | K_a]; S_b: [P^T | K_b] with the lower lanes write-disabled
-                    const uint32_t a_a = desc_lo(pt_hi, tile(i, 0, 1) - pt_hi), a_b = desc_lo(pt_hi, tile(i, 0, 3) - pt_hi);
+                    // OS_a: [P^T | K_a] (output rows in lanes 0..63, state rows d_k < 64 in lanes 64..127); S_b: [K_b | next tile]
+                    // with the upper lanes write-disabled: state rows d_k >= 64 in lanes 0..63, so that the output warps
+                    // convert that half of the state while the score warps convert the other
+                    const uint32_t a_a = desc_lo(pt_hi, tile(i, 0, 1) - pt_hi), a_b = desc_lo(tile(i, 0, 3), kTile);
                     const uint32_t first = (i > 0 || has_init) ? 1u : 0u;
 #pragma unroll
                     for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColOS, a_a + 128 * k, v_hi + 128 * k, idescG3, (first || k > 0) ? 1u : 0u);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColSb, a_b + 128 * k, v_hi + 128 * k, idescG3, (first || k > 0) ? 1u : 0u, 2);
+                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColSb, a_b + 128 * k, v_hi + 128 * k, idescG3, (first || k > 0) ? 1u : 0u, 1);
                     if (kPair) {
                         const uint32_t v_lo = desc_lo(tile(i, 1, 4), kTile);
-                        const uint32_t a2_a = desc_lo(pt_lo, tile(i, 1, 1) - pt_lo), a2_b = desc_lo(pt_lo, tile(i, 1, 3) - pt_lo);
+                        const uint32_t a2_a = desc_lo(pt_lo, tile(i, 1, 1) - pt_lo), a2_b = desc_lo(tile(i, 1, 3), kTile);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColOS, a_a + 128 * k, v_lo + 128 * k, idescG3, 1);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColOS, a2_a + 128 * k, v_hi + 128 * k, idescG3, 1);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColSb, a_b + 128 * k, v_lo + 128 * k, idescG3, 1, 2);
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColSb, a_b + 128 * k, v_lo + 128 * k, idescG3, 1, 1);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColSb, a2_b + 128 * k, v_hi + 128 * k, idescG3, 1, 2);
+                        for (int k = 0; k < 4; ++k) umma_bf16(tmem + kColSb, a2_b + 128 * k, v_hi + 128 * k, idescG3, 1, 1);
                     }
                     umma_commit(bar_o);
                 }
@@ -247,10 +249,12 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                 *reinterpret_cast<uint4 *>(sLo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
             }
         };
+        // state rows of this thread: d_k = 64 * xs + r, xs = 0 for the score warps (accumulator OS_a, lanes 64..127), 1 for the
+        // output warps (accumulator S_b, lanes 0..63)
+        const int xs = upper ? 0 : 1;
         if (has_init) {
-            if (upper) {
-#pragma unroll 1
-                for (int x = 0; x < 2; ++x)
+            {
+                const int x = xs;
 #pragma unroll 1
                     for (int half = 0; half < 2; ++half) {
                         float sv[64];
@@ -322,7 +326,37 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
             ok = __all_sync(0xffffffffu, mbar_wait(bar_o, i & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
+            // ---- state rows d_k = 64 * xs + r of this thread: bf16 hi + lo -> shared (B operand of the next chunk's G2) ----
+            auto convert_state_rows = [&]() {
+#pragma unroll 1
+                for (int half = 0; half < 2; ++half) {
+                    float sv[64];
+                    const uint32_t col = (xs == 0 ? kColOS : kColSb) + 64 * half;
+                    tmem_ld32(tmem_warp + col, *reinterpret_cast<float(*)[32]>(&sv[0]));
+                    tmem_ld32(tmem_warp + col + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+                    tmem_ld_wait();
+                    write_state_tiles(sv, xs, half);
+                }
+                fence_proxy_async();
+            };
+            // last chunk of the sequence: the fp32 state leaves the SM once, for the caller
+            auto store_state_rows = [&]() {
+#pragma unroll 1
+                for (int half = 0; half < 2; ++half) {
+                    float sv[64];
+                    const uint32_t col = (xs == 0 ? kColOS : kColSb) + 64 * half;
+                    tmem_ld32(tmem_warp + col, *reinterpret_cast<float(*)[32]>(&sv[0]));
+                    tmem_ld32(tmem_warp + col + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+                    tmem_ld_wait();
+                    float4 *dst = reinterpret_cast<float4 *>(state_out + (size_t)bh * kD * kD + (size_t)(64 * xs + r) * kD + 64 * half);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) dst[j] = make_float4(sv[4 * j], sv[4 * j + 1], sv[4 * j + 2], sv[4 * j + 3]);
+                }
+            };
             if (!upper) {
+                // their half of the state first (the next chunk's G2 waits for it), then the output rows
+                if (i + 1 < nchunks) convert_state_rows();
+                else if (state_out && g == G - 1) store_state_rows();
                 // ---- output row t (128 values): scale, normaliser -> swizzled staging -> TMA store ------------
                 float acc[kD];
 #pragma unroll
@@ -365,37 +399,12 @@ linattn_sm100_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                     bulk_commit();
                 }
             } else if (i + 1 < nchunks) {
-                // ---- state rows d_k = r (from OS_a) and d_k = 64 + r (from S_b): bf16 hi + lo -> shared --------
-#pragma unroll 1
-                for (int x = 0; x < 2; ++x)
-#pragma unroll 1
-                    for (int half = 0; half < 2; ++half) {
-                        float sv[64];
-                        const uint32_t col = (x == 0 ? kColOS : kColSb) + 64 * half;
-                        tmem_ld32(tmem_warp + col, *reinterpret_cast<float(*)[32]>(&sv[0]));
-                        tmem_ld32(tmem_warp + col + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
-                        tmem_ld_wait();
-                        write_state_tiles(sv, x, half);
-                    }
-                fence_proxy_async();
+                convert_state_rows();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_s);
             } else if (state_out && g == G - 1) {
-                // last chunk of the sequence: the fp32 state leaves the SM once, for the caller
-#pragma unroll 1
-                for (int x = 0; x < 2; ++x)
-#pragma unroll 1
-                    for (int half = 0; half < 2; ++half) {
-                        float sv[64];
-                        const uint32_t col = (x == 0 ? kColOS : kColSb) + 64 * half;
-                        tmem_ld32(tmem_warp + col, *reinterpret_cast<float(*)[32]>(&sv[0]));
-                        tmem_ld32(tmem_warp + col + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
-                        tmem_ld_wait();
-                        float4 *dst = reinterpret_cast<float4 *>(state_out + (size_t)bh * kD * kD + (size_t)(64 * x + r) * kD + 64 * half);
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) dst[j] = make_float4(sv[4 * j], sv[4 * j + 1], sv[4 * j + 2], sv[4 * j + 3]);
-                    }
+                store_state_rows();
             }
         }
         if (!ok && lane == 0) {
