@@ -429,6 +429,18 @@ __global__ void __launch_bounds__(NTHR) fft_conv_fast_kernel(float *__restrict__
     const bool aligned = (reinterpret_cast<size_t>(x) & 7) == 0;
     float2 *kspec = spec + (size_t)(MODE == 1 ? row % D : row) * spec_stride;
     __syncthreads();
+    // With one slot per thread the middle passes do not need the whole CTA to meet: the pass at sub-length 4096 works
+    // inside blocks of 4096 points, which belong to groups of 256 consecutive threads before and after it, and the pass
+    // at sub-length 256 and the contiguous pass work inside blocks of 256 points = 16 consecutive threads of one warp.
+    constexpr bool kOneSlot = NSLOT == NTHR;
+    auto sync_4096_group = [&]() {
+        if (kOneSlot && NTHR > 256) asm volatile("bar.sync %0, 256;" ::"r"(1 + (int)(threadIdx.x >> 8)) : "memory");
+        else __syncthreads();
+    };
+    auto sync_256_group = [&]() {
+        if (kOneSlot) __syncwarp();
+        else __syncthreads();
+    };
 
     // ---- forward ----
 #pragma unroll 1
@@ -437,12 +449,12 @@ __global__ void __launch_bounds__(NTHR) fft_conv_fast_kernel(float *__restrict__
     if (LEN1 == 4096) {   // sub-length left by the first pass: 4096 or 256
 #pragma unroll 1
         for (int g = threadIdx.x; g < NSLOT; g += NTHR) r16_pass<4096, false>(s, g, tb);
-        __syncthreads();
+        sync_4096_group();
     }
     if (LEN1 >= 256) {
 #pragma unroll 1
         for (int g = threadIdx.x; g < NSLOT; g += NTHR) r16_pass<256, false>(s, g, tb);
-        __syncthreads();
+        sync_256_group();
     }
 #pragma unroll 1
     for (int g = threadIdx.x; g < NSLOT; g += NTHR) contiguous_pass<false>(s, g);
@@ -457,12 +469,14 @@ __global__ void __launch_bounds__(NTHR) fft_conv_fast_kernel(float *__restrict__
     // ---- inverse ----
 #pragma unroll 1
     for (int g = threadIdx.x; g < NSLOT; g += NTHR) contiguous_pass<true>(s, g);
-    __syncthreads();
     if (LEN1 >= 256) {
+        sync_256_group();
 #pragma unroll 1
         for (int g = threadIdx.x; g < NSLOT; g += NTHR) r16_pass<256, true>(s, g, tb);
+        if (LEN1 == 4096) sync_4096_group();
+        else __syncthreads();
+    } else
         __syncthreads();
-    }
     if (LEN1 == 4096) {
 #pragma unroll 1
         for (int g = threadIdx.x; g < NSLOT; g += NTHR) r16_pass<4096, true>(s, g, tb);
