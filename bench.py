@@ -418,6 +418,8 @@ def main():
     ms_total = ev0.elapsed_time(ev1)
     if chela.async_status(ws) != chela.OK:
         raise RuntimeError("device-side wait timed out during the timed region")
+    # the clock the hardware counts (SM cycles over global-timer nanoseconds), right after the timed region
+    sm_mhz_counted = chela.debug_sm_clock_mhz()
     # keep the GPU under the same load a little longer if the timed region was too short to sample clocks
     clocks = sampler.summary(t_wall0, t_wall1)
     if clocks["samples"] < 5:
@@ -428,6 +430,7 @@ def main():
             torch.cuda.synchronize()
         clocks = sampler.summary(t_wall0, time.perf_counter())
         clocks["note"] = "timed region too short for NVML polling: window extended over an identical untimed burst"
+    clocks["sm_mhz_counted"] = sm_mhz_counted
     ms_step = max_over_ranks(ms_total, world, dev) / args.steps
     value = job_tokens_per_s(ms_step, world, TOTAL_TOKENS)
 
@@ -531,9 +534,15 @@ def main():
         # ---- every L of the sweep, same kernel and launch path ---------------------------------------
         sweep = []
         for L in SWEEP_L:
+            tw0 = time.perf_counter()
             ms = timed(lambda: step(L), 30, warm=5)
+            ck = sampler.summary(tw0, time.perf_counter())   # the SM clock NVML reports for this point (warm-up included)
+            # and the clock the hardware counts right after it: SM cycles over global-timer nanoseconds.  The two differ:
+            # NVML was seen to report the maximum clock with no throttle reason while the counted clock had dropped to
+            # 1400 MHz after a few hundred milliseconds of load, and the shapes with fewer sequences than SMs follow it.
             sweep.append({"L": L, "B": TOTAL_TOKENS // L, "ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
-                          "hbm_frac": alg_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]})
+                          "hbm_frac": alg_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "sm_mhz_nvml": ck["sm_mhz"],
+                          "sm_mhz_counted": chela.debug_sm_clock_mhz(), "clock_reasons": ck["reasons"]})
         line["sweep"] = sweep
         line["sweep_linearity"] = sweep_linearity(sweep)
         # ---- d = 128 (config 4's head size) plain bf16 linear attention at the same token count: H = 8 ----------

@@ -214,6 +214,16 @@ chela_status_t chela_async_status(const void *workspace, cudaStream_t stream);
 void chela_debug_wait_control(long long limit_cycles, int skip_arrival);
 
 /*
+ * Measurement aid (the paper has no counterpart): the SM clock as the hardware counts it.  Enqueues one CTA of one
+ * thread on `stream` that spins for spin_cycles SM cycles (clamped to [10 000, 2 000 000]) and writes two 64-bit
+ * integers to the device buffer `out16` (16 bytes, 8-byte aligned): the SM cycles that passed and the nanoseconds of
+ * the GPU's global timer over the same interval.  cycles * 1000 / nanoseconds = MHz.  Run right after a timed region it
+ * shows the clock that region ended at; the driver's management interface was seen to report the maximum clock while
+ * this ratio read 1400 MHz after a few hundred milliseconds of load.
+ */
+chela_status_t chela_debug_sm_clock(void *out16, long long spin_cycles, cudaStream_t stream);
+
+/*
  * chela_linattn_fwd without a caller-provided workspace and without any allocation.  (The paper has no
  * counterpart: this is a packaging variant of the entry point above, same kernels, same results.)
  *

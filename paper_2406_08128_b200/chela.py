@@ -49,6 +49,7 @@ _SIGNATURES = {
                                  _c_size_t, _vp]),
     "chela_async_status": (_c_int, [_vp, _vp]),
     "chela_debug_wait_control": (None, [ctypes.c_longlong, _c_int]),
+    "chela_debug_sm_clock": (_c_int, [_vp, ctypes.c_longlong, _vp]),
     "chela_linattn_static_ws_status": (_c_int, [_vp]),
     "chela_linattn_fwd_static_ws": (_c_int, [_vp, _vp, _vp, _vp] + [_c_int] * 6 + [_c_int, _c_int, _c_int, _c_float,
                                              _c_float, _vp]),
@@ -317,6 +318,14 @@ def mixer_prepared_fwd(x, w_short, spectrum, w_q, w_k, w_v, H, w_a=None, w_o=Non
 def debug_wait_control(limit_cycles=0, skip_arrival=0) -> None:
     """chela_debug_wait_control: the wait limit (SM cycles, 0 = default) and the skipped-arrival test hook."""
     lib().chela_debug_wait_control(int(limit_cycles), int(skip_arrival))
+
+
+def debug_sm_clock_mhz(spin_cycles=400000, device=None) -> float:
+    """chela_debug_sm_clock on the current stream: the SM clock in MHz as SM cycles over global-timer nanoseconds."""
+    out = torch.zeros(2, dtype=torch.int64, device=device if device is not None else torch.device("cuda", torch.cuda.current_device()))
+    _check(lib().chela_debug_sm_clock(_ptr(out), int(spin_cycles), _stream()), "chela_debug_sm_clock")
+    cycles, ns = (int(x) for x in out.cpu())
+    return cycles * 1000.0 / max(ns, 1)
 
 
 def linattn_static_ws_status() -> int:

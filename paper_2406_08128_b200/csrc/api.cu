@@ -57,6 +57,29 @@ WaitCtl current_wait_ctl() { return WaitCtl{g_wait_limit_cycles, g_skip_arrival}
 
 extern "C" {
 
+namespace {
+__global__ void sm_clock_probe_kernel(long long *out, long long spin_cycles)
+{
+    unsigned long long g0, g1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g0));
+    const long long c0 = clock64();
+    long long c1 = c0;
+    while (c1 - c0 < spin_cycles) c1 = clock64();   // bounded by spin_cycles
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g1));
+    out[0] = c1 - c0;
+    out[1] = (long long)(g1 - g0);
+}
+}  // namespace
+
+chela_status_t chela_debug_sm_clock(void *out16, long long spin_cycles, cudaStream_t stream)
+{
+    if (!out16 || (reinterpret_cast<uintptr_t>(out16) & 7u)) return CHELA_ERR_INVALID_ARG;
+    if (spin_cycles < 10000) spin_cycles = 10000;
+    if (spin_cycles > 2000000) spin_cycles = 2000000;
+    sm_clock_probe_kernel<<<1, 1, 0, stream>>>((long long *)out16, spin_cycles);
+    return last_launch_status();
+}
+
 void chela_debug_wait_control(long long limit_cycles, int skip_arrival)
 {
     g_wait_limit_cycles = limit_cycles > 0 ? limit_cycles : 2000000000LL;

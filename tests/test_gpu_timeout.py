@@ -66,3 +66,9 @@ def test_projection_wait_runs_out_and_the_next_call_is_clean():
     assert chela.async_status(ws) == chela.OK
     ref = oracle.dense(a, w)
     assert rel_err(to_numpy(got), ref) <= 2e-2
+
+
+def test_sm_clock_probe_reports_a_plausible_clock():
+    """chela_debug_sm_clock: SM cycles over global-timer nanoseconds, a few hundred microseconds of spinning."""
+    mhz = chela.debug_sm_clock_mhz()
+    assert 300.0 < mhz < 3000.0, mhz
