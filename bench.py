@@ -545,6 +545,18 @@ def main():
                           "sm_mhz_counted": chela.debug_sm_clock_mhz(), "clock_reasons": ck["reasons"]})
         line["sweep"] = sweep
         line["sweep_linearity"] = sweep_linearity(sweep)
+        # The same points again, each after a one-second pause: back to back, the counted SM clock falls from point to
+        # point (1965 -> 1680 -> 1400-1580 MHz while NVML reports 1965), and the shapes with fewer sequences than SMs
+        # follow it; rested, every point starts from the same clock state.  Both sets are printed; neither is the headline.
+        rested = []
+        for L in SWEEP_L:
+            time.sleep(1.0)
+            ms = timed(lambda: step(L), 30, warm=5)
+            rested.append({"L": L, "B": TOTAL_TOKENS // L, "ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
+                           "hbm_frac": alg_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                           "sm_mhz_counted": chela.debug_sm_clock_mhz()})
+        line["sweep_rested"] = rested
+        line["sweep_rested_linearity"] = sweep_linearity(rested)
         # ---- d = 128 (config 4's head size) plain bf16 linear attention at the same token count: H = 8 ----------
         n128 = TOTAL_TOKENS * 8 * 128
         q8, k8, v8 = (flat[j][:n128].view(16, TOTAL_TOKENS // 16, 8, 128) for j in range(3))
