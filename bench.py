@@ -562,13 +562,16 @@ def main():
         q8, k8, v8 = (flat[j][:n128].view(16, TOTAL_TOKENS // 16, 8, 128) for j in range(3))
         o8 = out_flat[:n128].view(16, TOTAL_TOKENS // 16, 8, 128)
         ws8 = torch.zeros(chela.linattn_workspace_bytes(16, 8, TOTAL_TOKENS // 16, 128, 128, 128), dtype=torch.uint8, device=dev)
+        time.sleep(1.0)   # like the rested sweep: from the clock state of an idle GPU; the counted clock is printed
         ms = timed(lambda: chela.linattn_fwd(q8, k8, v8, chunk=128, out_dtype=chela.F32, out=o8, workspace=ws8), 20, warm=5)
+        mhz128 = chela.debug_sm_clock_mhz()
         if chela.async_status(ws8) != chela.OK:
             raise RuntimeError("device-side wait timed out in the d = 128 extra")
         b128 = TOTAL_TOKENS * 8 * (3 * 128 * 2 + 128 * 4)
         line["linattn_d128"] = {"B": 16, "L": TOTAL_TOKENS // 16, "H": 8, "d": 128, "ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
-                                "hbm_frac": b128 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                "note": "plain bf16 in, fp32 out, d_k = d_v = 128; algorithmic bytes 1280 per token-head"}
+                                "hbm_frac": b128 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "sm_mhz_counted": mhz128,
+                                "note": "plain bf16 in, fp32 out, d_k = d_v = 128; algorithmic bytes 1280 per token-head; "
+                                        "measured after a one-second pause"}
         del ws8
         # ---- config 2: B=8, H=8, L=4096 (134 MB in + 67 MB out; four rotating buffer sets exceed L2) ----
         sets = []
@@ -584,9 +587,15 @@ def main():
             chela.linattn_fwd(q, k, v, chunk=64, out_dtype=chela.F32, out=o, workspace=ws)
 
         ms = timed(c2, 40)
+        mhz_c2 = chela.debug_sm_clock_mhz()
+        time.sleep(1.0)
+        ms_rested = timed(c2, 40)
         c2_bytes = BYTES_PER_TOKEN_HEAD * 8 * 4096 * 8
         line["config2"] = {"ms": ms, "tokens_per_s": 8 * 4096 / (ms * 1e-3),
-                           "hbm_frac": c2_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                           "hbm_frac": c2_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "sm_mhz_counted": mhz_c2,
+                           "ms_rested": ms_rested, "hbm_frac_rested": c2_bytes / (ms_rested * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                           "sm_mhz_counted_rested": chela.debug_sm_clock_mhz(),
+                           "note": "ms: right after the other extras; ms_rested: after a one-second pause"}
         if chela.async_status(ws) != chela.OK:
             raise RuntimeError("device-side wait timed out in the extras")
         del sets
