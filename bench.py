@@ -620,12 +620,13 @@ def main():
             mo = torch.empty(mb, ml, md, device=dev)
             spec = chela.longconv_prepare(k_l)   # the long kernels' spectra, once: the weights do not change between calls
             ms = timed(lambda: chela.mixer_prepared_fwd(x, w_s, spec, w_q, w_k, w_v, mh, chunk=mc, out=mo, workspace=mws), 20, warm=5)
+            mhz_mixer = chela.debug_sm_clock_mhz()
             ms_unprepared = timed(lambda: chela.mixer_fwd(x, w_s, k_l, w_q, w_k, w_v, mh, chunk=mc, out=mo, workspace=mws), 10, warm=3)
             if chela.async_status(mws) != chela.OK:
                 raise RuntimeError("device-side wait timed out in the mixer")
             d_head = md // mh
             flops_tok = mixer_flops_per_token(md, mh)
-            mixers.append({"B": mb, "L": ml, "D": md, "H": mh, "chunk": mc, "attention_tile_tokens": 64, "ms": ms, "ms_spectra_recomputed_every_call": ms_unprepared,
+            mixers.append({"B": mb, "L": ml, "D": md, "H": mh, "chunk": mc, "attention_tile_tokens": 64, "ms": ms, "sm_mhz_counted": mhz_mixer, "ms_spectra_recomputed_every_call": ms_unprepared,
                            "call": "chela_mixer_prepared_fwd (kernel spectra prepared once with chela_longconv_prepare)",
                            "tokens_per_s": mb * ml / (ms * 1e-3),
                            "tensor_frac": flops_tok * mb * ml / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
@@ -672,10 +673,11 @@ def main():
         d_o = (torch.randn(q_.shape, device=dev, generator=gen)).to(torch.bfloat16)
         bws = torch.zeros(int(chela.lib().chela_linattn_bwd_workspace_bytes(q_.shape[0], H, L_MAIN, D, D)), dtype=torch.uint8, device=dev)
         ms = timed(lambda: chela.linattn_bwd(q_, k_, v_, d_o, workspace=bws), 10, warm=3)
+        mhz_bwd = chela.debug_sm_clock_mhz()
         if chela.async_status(bws) != chela.OK:
             raise RuntimeError("device-side wait timed out in the backward pass")
         bwd_alg = TOTAL_TOKENS * H * D * (4 * 2 + 3 * 4)   # read q, k, v, d_o (bf16), write dq, dk, dv (fp32): 20 B per element
-        line["backward"] = {"ms": ms, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
+        line["backward"] = {"ms": ms, "sm_mhz_counted": mhz_bwd, "tokens_per_s": TOTAL_TOKENS / (ms * 1e-3),
                             "roofline": {"bound": "hbm", "achieved": bwd_alg / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                          "frac": bwd_alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_kind,
                                          "algorithmic_bytes_per_call": bwd_alg},
